@@ -1,0 +1,188 @@
+/*
+ * lococo.h - C ABI of the LoCoCo chunk-step library for NVIDIA B200 (sm_100a).
+ *
+ * The library implements the per-chunk hot path of "LoCoCo: Dropping In
+ * Convolutions for Long Context Compression" (arXiv 2406.05317):
+ *   Algorithm 2, Step 3   chunk attention over [compressed cache, causal chunk] (Eq. 1)
+ *   Algorithm 2, Step 4   mixing logits by a 1-D multi-channel convolution over the
+ *                         concatenated [cache; chunk] states (Eq. 6), ReLU
+ *                         (Section 3.2.1), sum normalisation (Eq. 7)
+ *   Algorithm 2, Step 5   the M cache slots rebuilt as weighted blends of all
+ *                         cache and chunk tokens, same weights for K and V (Eq. 4, Eq. 5)
+ *   Algorithm 2, loop     attention with the old cache, then fill or compress
+ * for batch x heads independent (sequence, head) units.  Notation follows the
+ * paper: M cache slots, B chunk size, k conv kernel width, d head dimension.
+ *
+ * Conventions
+ *   - Every pointer named "device" is a CUDA device pointer on the current device,
+ *     owned by the caller; the library allocates and frees no device memory and keeps
+ *     no pointer after a call returns, except the workspace given to
+ *     lococo_set_workspace (which also holds the packed conv weights).
+ *   - Tensors are 4-D views [batch, heads, tokens, d] with d contiguous, described by
+ *     a lococo_tensor; strides are in elements.  Base pointers and all strides in bytes
+ *     must be multiples of 16.
+ *   - `stream` is a cudaStream_t passed as void* (NULL = the default stream).  Calls
+ *     enqueue work and return; they do not synchronise unless stated.
+ *   - Every entry point returns a lococo_status.  Argument errors are detected on the
+ *     host before anything is launched.  Nothing throws, aborts or prints.
+ *   - Storage types: LOCOCO_F32 (computed with fp32 FMA) and LOCOCO_BF16 (bf16
+ *     operands, fp32 accumulation, fp32 softmax and normalisation).
+ */
+#ifndef LOCOCO_H_
+#define LOCOCO_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    LOCOCO_OK = 0,
+    LOCOCO_ERR_INVALID_ARG = 1,       /* NULL / misaligned pointer, bad size, k even, ... */
+    LOCOCO_ERR_UNSUPPORTED_SHAPE = 2, /* a shape the kernels do not cover */
+    LOCOCO_ERR_WORKSPACE = 3,         /* workspace missing or too small, weights not set */
+    LOCOCO_ERR_CUDA = 4,              /* a CUDA runtime call failed */
+    LOCOCO_ERR_TIMEOUT = 5            /* a bounded device-side wait ran out */
+} lococo_status;
+
+typedef enum { LOCOCO_F32 = 0, LOCOCO_BF16 = 1 } lococo_dtype;
+
+/* Which kernels serve a call. AUTO: tensor-core (tcgen05) kernels where the shape and
+ * dtype allow, CUDA-core kernels otherwise. */
+typedef enum { LOCOCO_PATH_AUTO = 0, LOCOCO_PATH_SIMT = 1, LOCOCO_PATH_TENSOR = 2 } lococo_path;
+
+typedef struct {
+    int32_t batch;            /* sequences processed together */
+    int32_t heads;            /* attention heads per sequence */
+    int32_t head_dim;         /* d: 64 or 128 */
+    int32_t M;                /* cache slots (Section 3.2) */
+    int32_t k;                /* conv kernel width, odd (Section 3.2.1; 21 in the paper) */
+    int32_t c_in;             /* conv input channels: d (keys) or 2*d (keys stacked on values, Eq. 6) */
+    int32_t weights_per_head; /* 0: one weight set [M,c_in,k] shared by the heads (Section 4.1);
+                                 1: one set per head [heads,M,c_in,k] */
+    int32_t dtype;            /* lococo_dtype of Q, K, V, O, the cache and the weights */
+    float softmax_scale;      /* 0 selects 1/sqrt(d) (Eq. 1) */
+    float norm_eps;           /* added to the denominator of Eq. 7 */
+    int32_t max_chunk;        /* largest chunk length b any call will pass */
+    int32_t path;             /* lococo_path */
+} lococo_config;
+
+/* Strided view [batch, heads, tokens, d]; element (n,h,t,c) is at
+ * ptr + n*stride_batch + h*stride_head + t*stride_token + c (in elements). */
+typedef struct {
+    void* ptr; /* device */
+    int64_t stride_batch, stride_head, stride_token;
+} lococo_tensor;
+
+typedef struct lococo_handle lococo_handle;
+
+/* Validates the configuration and returns a host-side handle. No device work. */
+lococo_status lococo_create(const lococo_config* config, lococo_handle** out);
+lococo_status lococo_destroy(lococo_handle* handle);
+
+/* Bytes of device scratch the handle needs (packed weights, mixing logits, partial
+ * blends, status word). */
+lococo_status lococo_workspace_bytes(const lococo_handle* handle, size_t* out);
+/* Gives the handle its scratch: device memory, 256-byte aligned, at least
+ * lococo_workspace_bytes; it must stay valid until lococo_destroy or the next
+ * lococo_set_workspace.  Clears the device status word on `stream`. */
+lococo_status lococo_set_workspace(lococo_handle* handle, void* device_ptr, size_t bytes, void* stream);
+
+/* Conv weights of Eq. 6: G [heads|1, M, c_in, k] and optional bias [heads|1, M]
+ * (NULL = none), device pointers in the configured dtype, contiguous.  They are
+ * re-packed into the workspace, so the workspace must be set first and G may be
+ * released after the stream reaches this point. */
+lococo_status lococo_set_weights(lococo_handle* handle, const void* G_device, const void* bias_device,
+                                 void* stream);
+
+/*
+ * Algorithm 2, the branch after Step 3.  With c = cache_len:
+ *   c + b <= M : fill - chunk rows are appended at cache rows c..c+b-1;
+ *   otherwise  : Steps 4 and 5 on the S = c + b real entries [cache; chunk]:
+ *       A[i,j] = bias_i + sum_ch sum_t G[i,ch,t] * Z[j+t-(k-1)/2, ch]   (zero outside [0,S))
+ *       R = max(A, 0);  s_i = sum_j R[i,j] + eps;  w = R / s              (Eq. 7)
+ *       K_out[i,:] = sum_j w[i,j] XK[j,:];  V_out likewise                (Eq. 4, Eq. 5)
+ *     with Z = XK (c_in = d) or [XK | XV] along channels (c_in = 2d).
+ * K_cache/V_cache hold M rows per unit of which the first c are valid; the outputs
+ * may alias them.  new_cache_len (host, optional) receives c + b or M.
+ * W_out (device, optional, fp32 [batch, heads, M, c+b]) receives w of a compress step.
+ */
+lococo_status lococo_compress_step(lococo_handle* handle, lococo_tensor K_cache, lococo_tensor V_cache,
+                                   int32_t cache_len, lococo_tensor K_chunk, lococo_tensor V_chunk, int32_t b,
+                                   lococo_tensor K_cache_out, lococo_tensor V_cache_out,
+                                   int32_t* new_cache_len, float* W_out, void* stream);
+
+/*
+ * Algorithm 2, Step 3 (Eq. 1): the b chunk queries attend over the c cache entries
+ * (all visible) followed by the chunk (query r sees chunk keys 0..r), softmax over
+ * keys with scale softmax_scale.  lse (device, optional, fp32 [batch, heads, b])
+ * receives the log-sum-exp of the scaled logits.
+ */
+lococo_status lococo_chunk_attention(lococo_handle* handle, lococo_tensor Q_chunk, lococo_tensor K_cache,
+                                     lococo_tensor V_cache, int32_t cache_len, lococo_tensor K_chunk,
+                                     lococo_tensor V_chunk, int32_t b, lococo_tensor O_chunk, float* lse,
+                                     void* stream);
+
+/* Bytes of the `saved` buffer lococo_process_sequence fills for a later backward pass:
+ * the cache before every step, and the attention log-sum-exp. */
+lococo_status lococo_saved_bytes(const lococo_handle* handle, int32_t L, int32_t B, size_t* out);
+
+/*
+ * Algorithm 2 over L tokens in chunks of B (the last chunk may be short): for each
+ * chunk, lococo_chunk_attention with the cache as it stands, then lococo_compress_step.
+ * Q, K, V, O hold L tokens; K_cache/V_cache (M rows per unit) and *cache_len_inout
+ * (host) carry the cache state in and out, so a sequence can be suspended and resumed
+ * between calls.  saved (device, optional) is laid out as lococo_saved_bytes describes.
+ */
+lococo_status lococo_process_sequence(lococo_handle* handle, lococo_tensor Q, lococo_tensor K, lococo_tensor V,
+                                      int32_t L, int32_t B, lococo_tensor O, lococo_tensor K_cache,
+                                      lococo_tensor V_cache, int32_t* cache_len_inout, void* saved, void* stream);
+
+/* Bytes of device staging lococo_process_sequence_host needs for L tokens. */
+lococo_status lococo_host_staging_bytes(const lococo_handle* handle, int32_t L, size_t* out);
+
+/*
+ * lococo_process_sequence on HOST buffers: contiguous [batch, heads, L, d] Q, K, V are
+ * copied to the device staging area, the loop runs from an empty cache, and O plus the
+ * final cache ([batch, heads, M, d] each, optional) are copied back.  Host buffers
+ * should be pinned for the copies to be asynchronous.  Synchronises `stream` before
+ * returning; final_cache_len (host) receives the fill count.
+ */
+lococo_status lococo_process_sequence_host(lococo_handle* handle, const void* Q_host, const void* K_host,
+                                           const void* V_host, int32_t L, int32_t B, void* O_host,
+                                           void* K_cache_host, void* V_cache_host, int32_t* final_cache_len,
+                                           void* device_staging, size_t staging_bytes, void* stream);
+
+/*
+ * Gradients of  loss = <dO, O> + <dK_cache_final, K_cache_final> + <dV_cache_final, V_cache_final>
+ * through lococo_process_sequence started from an empty cache (the training use of
+ * Algorithm 2; Section 3.2.1: the conv parameters are trained end to end).
+ * Q, K, V, O: the forward's tensors; saved: what that forward wrote.
+ * dQ, dK, dV (configured dtype) are overwritten; dG (fp32 [heads|1, M, c_in, k]) and
+ * dbias (fp32 [heads|1, M], optional) are accumulated (+=), summed over the units that
+ * share a weight set.  dK_cache_final/dV_cache_final may have ptr == NULL (zero).
+ * scratch: device memory of lococo_backward_scratch_bytes.
+ */
+lococo_status lococo_backward_scratch_bytes(const lococo_handle* handle, int32_t L, int32_t B, size_t* out);
+lococo_status lococo_process_sequence_backward(lococo_handle* handle, lococo_tensor Q, lococo_tensor K,
+                                               lococo_tensor V, lococo_tensor O, int32_t L, int32_t B,
+                                               const void* saved, lococo_tensor dO,
+                                               lococo_tensor dK_cache_final, lococo_tensor dV_cache_final,
+                                               lococo_tensor dQ, lococo_tensor dK, lococo_tensor dV, float* dG,
+                                               float* dbias, void* scratch, size_t scratch_bytes, void* stream);
+
+/* Synchronises `stream` and reads the device status word: LOCOCO_OK, or
+ * LOCOCO_ERR_TIMEOUT if a bounded wait inside a kernel gave up (results invalid). */
+lococo_status lococo_get_last_device_status(lococo_handle* handle, int32_t* out, void* stream);
+
+/* Number of kernels this handle has launched so far (host-side counter). */
+lococo_status lococo_launch_count(const lococo_handle* handle, int64_t* out);
+
+const char* lococo_status_string(lococo_status status);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* LOCOCO_H_ */
