@@ -1,0 +1,32 @@
+// Host-side state behind a lococo_handle, and the hooks of the tensor-core path.
+#pragma once
+
+#include "common.cuh"
+
+struct lococo_handle {
+    lococo_config cfg{};
+    int units = 0;          // batch * heads
+    size_t elt = 0;         // bytes per stored element
+    float scale = 0.f;      // softmax scale in effect
+    bool use_tensor = false;
+    bool weights_set = false;
+    bool has_bias = false;
+    char* ws = nullptr;     // caller-owned device workspace
+    size_t ws_need = 0;
+    size_t off_status = 0, off_gpack = 0, off_bias = 0, off_s = 0, off_UK = 0, off_UV = 0, off_R = 0;
+    size_t off_gimage = 0, off_part = 0, off_counter = 0;  // tensor-core path
+    int64_t launches = 0;
+};
+
+namespace lococo {
+
+// Tensor-core (tcgen05) path, tensor_forward.cu.
+bool tensor_config_supported(const lococo_config* c);
+void tensor_layout_workspace(lococo_handle* h, size_t* off);
+int tensor_pack_weights(lococo_handle* h, const void* G, cudaStream_t st);
+bool tensor_compress_supported(const lococo_handle* h, const CompressParams& p);
+int tensor_compress(lococo_handle* h, const CompressParams& p, cudaStream_t st);
+bool tensor_attention_supported(const lococo_handle* h, const AttnParams& p);
+int tensor_attention(lococo_handle* h, const AttnParams& p, cudaStream_t st);
+
+}  // namespace lococo
