@@ -1,0 +1,268 @@
+"""Parity of the CUDA path (through the C ABI) with the float64 CPU oracle, element by
+element on the same seeded inputs."""
+import numpy as np
+import pytest
+import torch
+
+from paper_2406_05317_b200 import workloads as wl
+from tests.helpers import assert_close, to_device, to_host, torch_dtype
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def api():
+    from paper_2406_05317_b200 import api as _api
+    return _api
+
+
+@pytest.fixture(scope="module")
+def orc():
+    from oracle import lococo_oracle
+    return lococo_oracle
+
+
+def make_ctx(api, w, path=0, bias=False, norm_eps=1e-6, max_chunk=None):
+    ctx = api.Lococo(w.batch, w.heads, w.d, w.M, w.k, max_chunk or w.B, dtype=torch_dtype(w.dtype), c_in=w.c_in,
+                     weights_per_head=w.weights_per_head, norm_eps=norm_eps, path=path)
+    G, bvec = wl.make_weights(w, with_bias=bias)
+    ctx.set_weights(to_device(G, w.dtype), None if bvec is None else to_device(bvec, w.dtype))
+    return ctx, G, bvec
+
+
+def run_sequence(api, w, path=0, bias=False):
+    """GPU process_sequence on workload w; returns numpy O, Kc, Vc, c."""
+    ctx, G, bvec = make_ctx(api, w, path, bias)
+    Q, K, V = wl.make_qkv(w)
+    dQ, dK, dV = (to_device(x, w.dtype) for x in (Q, K, V))
+    O = torch.empty_like(dQ)
+    Kc = torch.zeros(w.batch, w.heads, w.M, w.d, dtype=dQ.dtype, device="cuda")
+    Vc = torch.zeros_like(Kc)
+    c = ctx.process_sequence(dQ, dK, dV, w.B, O, Kc, Vc, 0)
+    torch.cuda.synchronize()
+    assert ctx.device_status() == api.OK
+    assert ctx.launch_count() > 0
+    return to_host(O), to_host(Kc), to_host(Vc), c
+
+
+_oracle_cache = {}
+
+
+def oracle_sequence(orc, w, bias=False):
+    """The oracle on workload w (cached: the same workload is checked on several paths)."""
+    key = (w, bias)
+    if key not in _oracle_cache:
+        Q, K, V = wl.make_qkv(w)
+        G, bvec = wl.make_weights(w, with_bias=bias)
+        _oracle_cache[key] = orc.process_batch(Q, K, V, G, w.B, bias=bvec)[:4]
+    return _oracle_cache[key]
+
+
+def check_sequence(api, orc, w, path=0, bias=False):
+    O, Kc, Vc, c = run_sequence(api, w, path, bias)
+    Or, Kr, Vr, cr = oracle_sequence(orc, w, bias)
+    assert (cr == c).all()
+    assert_close(O, Or, w.dtype, f"{w.name} O")
+    assert_close(Kc[:, :, :c], Kr[:, :, :c], w.dtype, f"{w.name} K cache")
+    assert_close(Vc[:, :, :c], Vr[:, :, :c], w.dtype, f"{w.name} V cache")
+
+
+# ---------------------------------------------------------------- whole loop
+@pytest.mark.parametrize("path", [0, 1])
+def test_cfg1_tiny_fp32_full(api, orc, path):
+    check_sequence(api, orc, wl.CONFIGS["cfg1"], path)
+
+
+@pytest.mark.parametrize("path", [0, 1])
+@pytest.mark.parametrize("c_mult", [1, 2])
+def test_cfg2_slice(api, orc, path, c_mult):
+    # Llama-2-7B inference shape, 3 of the 32 heads, all 8 chunks
+    check_sequence(api, orc, wl.CONFIGS["cfg2"].slice(heads=3, c_in_mult=c_mult), path)
+
+
+@pytest.mark.parametrize("path", [0, 1])
+def test_cfg3_slice(api, orc, path):
+    # streaming shape: 2 sequences x 2 heads, 32 chunks (2 fills + 30 compress steps)
+    check_sequence(api, orc, wl.CONFIGS["cfg3"].slice(batch=2, heads=2, L=2048), path)
+
+
+@pytest.mark.parametrize("path", [0, 1])
+def test_cfg4_slice(api, orc, path):
+    # fine-tuning shape M=512, shortened chunks so the oracle finishes in seconds:
+    # B=1024 keeps S = 1536 spanning several tiles of every kernel
+    check_sequence(api, orc, wl.CONFIGS["cfg4"].slice(heads=2, B=1024, L=3072), path)
+
+
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+def test_ragged_everything(api, orc, dtype):
+    # sizes that are multiples of nothing: M=40, B=37, L=301 (last chunk short), k=7,
+    # bias, per-head weights, c_in = 2d
+    w = wl.Workload("ragged", 9, batch=2, heads=3, d=64, M=40, B=37, k=7, L=301, dtype=dtype,
+                    weights_per_head=True, qkv_scale=1.0, g_std=0.05, c_in_mult=2)
+    check_sequence(api, orc, w, 0, bias=True)
+
+
+def test_short_sequence_is_full_attention(api, orc):
+    # L <= M: only the fill branch runs
+    w = wl.Workload("short", 10, batch=1, heads=2, d=128, M=128, B=48, k=21, L=100, dtype="bf16",
+                    weights_per_head=False, qkv_scale=1.0)
+    check_sequence(api, orc, w, 0)
+
+
+def test_suspend_resume_bit_identical(api):
+    w = wl.CONFIGS["cfg2"].slice(heads=2, L=2048)
+    ctx, G, _ = make_ctx(api, w)
+    Q, K, V = (to_device(x, w.dtype) for x in wl.make_qkv(w))
+
+    def run(splits):
+        O = torch.empty_like(Q)
+        Kc = torch.zeros(w.batch, w.heads, w.M, w.d, dtype=Q.dtype, device="cuda")
+        Vc = torch.zeros_like(Kc)
+        c, t0 = 0, 0
+        for n in splits:
+            sl = slice(t0, t0 + n)
+            c = ctx.process_sequence(Q[:, :, sl], K[:, :, sl], V[:, :, sl], w.B, O[:, :, sl], Kc, Vc, c)
+            t0 += n
+        torch.cuda.synchronize()
+        return O, Kc, Vc, c
+
+    a, b = run([2048]), run([1024, 1024])
+    assert a[3] == b[3]
+    for x, y in zip(a[:3], b[:3]):
+        assert torch.equal(x, y)
+
+
+# ---------------------------------------------------------------- single calls
+@pytest.mark.parametrize("dtype,d,M,k,c,b,c_mult,per_head,bias", [
+    ("f32", 64, 16, 5, 16, 16, 1, False, False),
+    ("f32", 128, 24, 3, 10, 30, 2, True, True),
+    ("bf16", 128, 128, 21, 128, 512, 1, True, False),
+    ("bf16", 128, 128, 21, 0, 512, 2, False, False),
+    ("bf16", 128, 128, 21, 128, 64, 1, False, True),
+    ("bf16", 64, 72, 9, 50, 171, 1, False, False),
+    ("bf16", 128, 512, 21, 512, 700, 1, False, False),
+])
+def test_compress_step_and_weights(api, orc, dtype, d, M, k, c, b, c_mult, per_head, bias):
+    w = wl.Workload("step", 11, batch=1, heads=2, d=d, M=M, B=b, k=k, L=b, dtype=dtype, weights_per_head=per_head,
+                    qkv_scale=1.0, c_in_mult=c_mult)
+    ctx, G, bvec = make_ctx(api, w, bias=bias)
+    _, Kn, Vn = wl.make_qkv(w)
+    wc = w.slice(L=max(c, 1), seed0=77)
+    _, Kc, Vc = wl.make_qkv(wc)
+    Kc_full = np.zeros((w.batch, w.heads, M, d), np.float32)
+    Vc_full = np.zeros_like(Kc_full)
+    Kc_full[:, :, :c], Vc_full[:, :, :c] = Kc[:, :, :c], Vc[:, :, :c]
+    dKc, dVc, dKn, dVn = (to_device(x, dtype) for x in (Kc_full, Vc_full, Kn, Vn))
+    Ko, Vo = torch.zeros_like(dKc), torch.zeros_like(dVc)
+    S = c + b
+    W = torch.zeros(w.batch, w.heads, M, S, dtype=torch.float32, device="cuda")
+    new_len = ctx.compress_step(dKc, dVc, c, dKn, dVn, Ko, Vo, W)
+    torch.cuda.synchronize()
+    assert new_len == M and ctx.device_status() == api.OK
+    Ko_h, Vo_h, W_h = to_host(Ko), to_host(Vo), to_host(W)
+    for n in range(w.batch):
+        for h in range(w.heads):
+            XK = np.vstack([Kc_full[n, h, :c], Kn[n, h]])
+            XV = np.vstack([Vc_full[n, h, :c], Vn[n, h]])
+            Kr, Vr, wr, _, _ = orc.compress(XK, XV, G[h if per_head else 0],
+                                            bias=None if bvec is None else bvec[h if per_head else 0],
+                                            want_weights=True)
+            assert_close(Ko_h[n, h], Kr, dtype, "K slots")
+            assert_close(Vo_h[n, h], Vr, dtype, "V slots")
+            assert_close(W_h[n, h], wr, dtype, "mixing weights")
+            assert np.abs(W_h[n, h].sum(1) - 1).max() <= 1e-3       # Eq. 7: rows sum to one
+    # in-place update gives the same slots
+    ctx.compress_step(dKc, dVc, c, dKn, dVn)
+    torch.cuda.synchronize()
+    assert torch.equal(dKc, Ko) and torch.equal(dVc, Vo)
+
+
+@pytest.mark.parametrize("dtype,d,c,b", [("f32", 64, 16, 16), ("f32", 128, 0, 45), ("bf16", 128, 128, 512),
+                                         ("bf16", 128, 0, 512), ("bf16", 128, 128, 1), ("bf16", 64, 37, 203),
+                                         ("bf16", 128, 512, 1100)])
+def test_chunk_attention(api, orc, dtype, d, c, b):
+    M = max(c, 16)
+    w = wl.Workload("attn", 12, batch=2, heads=2, d=d, M=M, B=b, k=3, L=b, dtype=dtype, weights_per_head=False,
+                    qkv_scale=1.0)
+    ctx = api.Lococo(w.batch, w.heads, d, M, 3, b, dtype=torch_dtype(dtype))
+    Q, Kn, Vn = wl.make_qkv(w)
+    _, Kc, Vc = wl.make_qkv(w.slice(L=M, seed0=5))
+    dQ, dKn, dVn, dKc, dVc = (to_device(x, dtype) for x in (Q, Kn, Vn, Kc, Vc))
+    O = torch.empty_like(dQ)
+    lse = torch.empty(w.batch, w.heads, b, dtype=torch.float32, device="cuda")
+    ctx.chunk_attention(dQ, dKc, dVc, c, dKn, dVn, O, lse)
+    torch.cuda.synchronize()
+    O_h, lse_h = to_host(O), to_host(lse)
+    for n in range(w.batch):
+        for h in range(w.heads):
+            Or, lr = orc.attention(Q[n, h], np.vstack([Kc[n, h, :c], Kn[n, h]]), np.vstack([Vc[n, h, :c], Vn[n, h]]), c)
+            assert_close(O_h[n, h], Or, dtype, "O")
+            assert np.abs(lse_h[n, h] - lr).max() <= (2e-2 if dtype == "bf16" else 1e-4 * max(1, np.abs(lr).max()))
+
+
+def test_strided_views_and_fill_to_other_buffer(api, orc):
+    # Q/K/V as slices of one packed [batch, tokens, 3, heads, d] projection output
+    w = wl.Workload("strided", 13, batch=2, heads=2, d=64, M=32, B=24, k=5, L=120, dtype="bf16",
+                    weights_per_head=False, qkv_scale=1.0)
+    ctx, G, _ = make_ctx(api, w)
+    Q, K, V = wl.make_qkv(w)
+    packed = torch.empty(w.batch, w.L, 3, w.heads, w.d, dtype=torch.bfloat16, device="cuda")
+    for i, x in enumerate((Q, K, V)):
+        packed[:, :, i] = to_device(x, "bf16").permute(0, 2, 1, 3)
+    q, k, v = (packed[:, :, i].permute(0, 2, 1, 3) for i in range(3))
+    assert not q.is_contiguous()
+    O = torch.empty(w.batch, w.L, w.heads, w.d, dtype=torch.bfloat16, device="cuda").permute(0, 2, 1, 3)
+    Kc = torch.zeros(w.batch, w.heads, w.M, w.d, dtype=torch.bfloat16, device="cuda")
+    Vc = torch.zeros_like(Kc)
+    ctx.process_sequence(q, k, v, w.B, O, Kc, Vc, 0)
+    torch.cuda.synchronize()
+    Or, Kr, Vr, cr, _ = orc.process_batch(Q, K, V, G, w.B)
+    assert_close(to_host(O), Or, "bf16", "O (strided)")
+    assert_close(to_host(Kc), Kr, "bf16", "K cache")
+    # fill branch into a different output buffer carries the old rows over
+    Kc2, Vc2 = torch.zeros_like(Kc), torch.zeros_like(Vc)
+    Ko, Vo = torch.full_like(Kc, 7.0), torch.full_like(Vc, 7.0)
+    Kc2[:, :, :5], Vc2[:, :, :5] = 1.0, 2.0
+    n = ctx.compress_step(Kc2, Vc2, 5, k[:, :, :10], v[:, :, :10], Ko, Vo)
+    torch.cuda.synchronize()
+    assert n == 15
+    assert torch.equal(Ko[:, :, :5], Kc2[:, :, :5]) and torch.equal(Ko[:, :, 5:15], k[:, :, :10])
+    assert torch.equal(Vo[:, :, 5:15], v[:, :, :10]) and (Ko[:, :, 15:] == 7.0).all()
+
+
+def test_host_entry_point_matches_device_entry_point(api):
+    w = wl.CONFIGS["cfg2"].slice(heads=2, L=1536)
+    ctx, G, _ = make_ctx(api, w)
+    Q, K, V = wl.make_qkv(w)
+    hq, hk, hv = (to_device(x, w.dtype).cpu().pin_memory() for x in (Q, K, V))
+    ho = torch.empty_like(hq).pin_memory()
+    hkc = torch.empty(w.batch, w.heads, w.M, w.d, dtype=hq.dtype).pin_memory()
+    hvc = torch.empty_like(hkc).pin_memory()
+    staging = torch.empty(ctx.host_staging_bytes(w.L), dtype=torch.uint8, device="cuda")
+    c = ctx.process_sequence_host(hq, hk, hv, w.B, ho, staging, hkc, hvc)
+    dq, dk, dv = hq.cuda(), hk.cuda(), hv.cuda()
+    O = torch.empty_like(dq)
+    Kc = torch.zeros(w.batch, w.heads, w.M, w.d, dtype=dq.dtype, device="cuda")
+    Vc = torch.zeros_like(Kc)
+    c2 = ctx.process_sequence(dq, dk, dv, w.B, O, Kc, Vc, 0)
+    torch.cuda.synchronize()
+    assert c == c2 == w.M
+    assert torch.equal(ho, O.cpu()) and torch.equal(hkc, Kc.cpu()) and torch.equal(hvc, Vc.cpu())
+
+
+def test_runtime_argument_errors_launch_nothing(api):
+    w = wl.CONFIGS["cfg1"]
+    ctx, G, _ = make_ctx(api, w)
+    x = torch.zeros(1, 1, 16, 64, device="cuda")
+    before = ctx.launch_count()
+    with pytest.raises(api.LococoError) as e:
+        ctx.compress_step(x, x.clone(), 17, x.clone(), x.clone())
+    assert e.value.status == api.ERR_INVALID_ARG
+    with pytest.raises(api.LococoError):
+        ctx.chunk_attention(x, x.clone(), x.clone(), 0, x.clone(), x.clone(), x)       # O aliases Q
+    big = torch.zeros(1, 1, 32, 64, device="cuda")
+    with pytest.raises(api.LococoError):
+        ctx.chunk_attention(big, x, x.clone(), 0, big.clone(), big.clone(), big.clone())  # b > max_chunk
+    with pytest.raises(api.LococoError):
+        ctx.compress_step(x[:, :, :, 1:], x.clone(), 0, x.clone(), x.clone())             # misaligned view
+    assert ctx.launch_count() == before
