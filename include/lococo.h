@@ -180,6 +180,17 @@ lococo_status lococo_get_last_device_status(lococo_handle* handle, int32_t* out,
 /* Number of kernels this handle has launched so far (host-side counter). */
 lococo_status lococo_launch_count(const lococo_handle* handle, int64_t* out);
 
+/*
+ * Optional timing of single kernel classes with CUDA events recorded on the launching
+ * stream around each launch.  kind 0: the kernel that evaluates Eq. 6 (the conv
+ * contraction, with whatever is fused into it); kind 1: the chunk-attention kernel (Eq. 1).
+ * lococo_profile_enable(h, 1) starts a fresh recording, (h, 0) stops it;
+ * lococo_profile_read waits for the recorded events and returns the summed duration in
+ * milliseconds and the number of launches of that kind since the recording started.
+ */
+lococo_status lococo_profile_enable(lococo_handle* handle, int32_t on);
+lococo_status lococo_profile_read(lococo_handle* handle, int32_t kind, double* total_ms, int64_t* launches);
+
 const char* lococo_status_string(lococo_status status);
 
 #ifdef __cplusplus

@@ -53,6 +53,8 @@ _SIGNATURES = {
                                          ctypes.c_size_t, _P],
     "lococo_get_last_device_status": [_P, ctypes.POINTER(_I), _P],
     "lococo_launch_count": [_P, ctypes.POINTER(ctypes.c_int64)],
+    "lococo_profile_enable": [_P, _I],
+    "lococo_profile_read": [_P, _I, ctypes.POINTER(ctypes.c_double), ctypes.POINTER(ctypes.c_int64)],
 }
 for _name, _args in _SIGNATURES.items():
     _fn = getattr(_lib, _name)
@@ -210,3 +212,13 @@ class Lococo:
         out = ctypes.c_int64()
         _check(_lib.lococo_launch_count(self._h, ctypes.byref(out)), "lococo_launch_count")
         return out.value
+
+    def profile(self, on: bool):
+        """Start (or stop) recording per-kernel CUDA-event timings."""
+        _check(_lib.lococo_profile_enable(self._h, int(on)), "lococo_profile_enable")
+
+    def profile_read(self, kind: int):
+        """(total milliseconds, launches) of kernel class `kind` (0: conv, 1: attention)."""
+        ms, n = ctypes.c_double(), ctypes.c_int64()
+        _check(_lib.lococo_profile_read(self._h, kind, ctypes.byref(ms), ctypes.byref(n)), "lococo_profile_read")
+        return ms.value, n.value

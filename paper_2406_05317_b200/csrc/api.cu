@@ -94,6 +94,7 @@ lococo_status compress_impl(lococo_handle* h, View kc, View vc, int c, View kn, 
     p.UK = reinterpret_cast<float*>(h->ws + h->off_UK);
     p.UV = reinterpret_cast<float*>(h->ws + h->off_UV);
     p.W_out = W_out;
+    p.prof = h->prof.on ? &h->prof : nullptr;
     if (h->use_tensor && tensor_compress_supported(h, p)) return count(h, tensor_compress(h, p, st));
     return count(h, simt_compress(cfg.dtype, p, st));
 }
@@ -108,6 +109,7 @@ lococo_status attention_impl(lococo_handle* h, View q, View kc, View vc, int c, 
     p.heads = cfg.heads; p.units = h->units; p.d = cfg.head_dim; p.b = b; p.c = c;
     p.scale = h->scale;
     p.lse = lse; p.lse_stride = lse_stride;
+    p.prof = h->prof.on ? &h->prof : nullptr;
     if (h->use_tensor && tensor_attention_supported(h, p)) return count(h, tensor_attention(h, p, st));
     return count(h, simt_attention(cfg.dtype, p, st));
 }
@@ -118,7 +120,61 @@ bool chunk_args_ok(const lococo_handle* h, int c, int b) {
 
 }  // namespace
 
+namespace lococo {
+
+void Profiler::begin(int kind, cudaStream_t st) {
+    if (used == recs.size()) {
+        Rec r{nullptr, nullptr, kind};
+        if (cudaEventCreate(&r.a) != cudaSuccess || cudaEventCreate(&r.b) != cudaSuccess) { on = false; return; }
+        recs.push_back(r);
+    }
+    recs[used].kind = kind;
+    cudaEventRecord(recs[used].a, st);
+}
+void Profiler::end(cudaStream_t st) {
+    if (used < recs.size()) cudaEventRecord(recs[used++].b, st);
+}
+void Profiler::release() {
+    for (Rec& r : recs) { cudaEventDestroy(r.a); cudaEventDestroy(r.b); }
+    recs.clear();
+    used = 0;
+}
+void prof_begin(void* p, int kind, cudaStream_t st) {
+    if (p && static_cast<Profiler*>(p)->on) static_cast<Profiler*>(p)->begin(kind, st);
+}
+void prof_end(void* p, cudaStream_t st) {
+    if (p && static_cast<Profiler*>(p)->on) static_cast<Profiler*>(p)->end(st);
+}
+
+}  // namespace lococo
+
 extern "C" {
+
+lococo_status lococo_profile_enable(lococo_handle* h, int32_t on) {
+    if (!h) return LOCOCO_ERR_INVALID_ARG;
+    h->prof.on = on != 0;
+    h->prof.used = 0;
+    return LOCOCO_OK;
+}
+
+lococo_status lococo_profile_read(lococo_handle* h, int32_t kind, double* total_ms, int64_t* launches) {
+    if (!h || !total_ms || !launches || kind < 0 || kind >= PROF_KINDS) return LOCOCO_ERR_INVALID_ARG;
+    double ms = 0.0;
+    int64_t n = 0;
+    for (size_t i = 0; i < h->prof.used; ++i) {
+        const Profiler::Rec& r = h->prof.recs[i];
+        if (r.kind != kind) continue;
+        if (cudaEventSynchronize(r.b) != cudaSuccess) return LOCOCO_ERR_CUDA;
+        float t = 0.f;
+        if (cudaEventElapsedTime(&t, r.a, r.b) != cudaSuccess) return LOCOCO_ERR_CUDA;
+        ms += t;
+        ++n;
+    }
+    *total_ms = ms;
+    *launches = n;
+    return LOCOCO_OK;
+}
+
 
 const char* lococo_status_string(lococo_status s) {
     switch (s) {
@@ -165,6 +221,7 @@ lococo_status lococo_create(const lococo_config* c, lococo_handle** out) {
 
 lococo_status lococo_destroy(lococo_handle* h) {
     if (!h) return LOCOCO_ERR_INVALID_ARG;
+    h->prof.release();
     delete h;
     return LOCOCO_OK;
 }

@@ -57,6 +57,7 @@ struct CompressParams {
     float* UK;             // [units][M][d] unnormalised blends
     float* UV;
     float* W_out;          // optional [units][M][S]
+    void* prof;            // host only: Profiler* or nullptr
 };
 
 // Parameters of one chunk attention (Algorithm 2, Step 3) for all units.
@@ -67,6 +68,7 @@ struct AttnParams {
     float scale;
     float* lse;        // optional [units][lse_stride]
     int64_t lse_stride;
+    void* prof;        // host only: Profiler* or nullptr
 };
 
 struct FillParams {
@@ -79,6 +81,10 @@ int simt_pack_weights(int dtype, const void* G, void* packed, int sets, int M, i
 int simt_fill(int dtype, const FillParams& p, cudaStream_t st);
 int simt_compress(int dtype, const CompressParams& p, cudaStream_t st);
 int simt_attention(int dtype, const AttnParams& p, cudaStream_t st);
+// Brackets the launches between them with an event pair when p is a live Profiler*.
+void prof_begin(void* p, int kind, cudaStream_t st);
+void prof_end(void* p, cudaStream_t st);
+
 int simt_convert_bias(int dtype, const void* bias, float* out, int n, cudaStream_t st);
 
 }  // namespace lococo

@@ -1,7 +1,23 @@
 // Host-side state behind a lococo_handle, and the hooks of the tensor-core path.
 #pragma once
 
+#include <vector>
+
 #include "common.cuh"
+
+namespace lococo {
+// Optional CUDA-event timing of individual kernel classes, on the launching stream.
+enum ProfKind { PROF_CONV = 0, PROF_ATTENTION = 1, PROF_KINDS = 2 };
+struct Profiler {
+    struct Rec { cudaEvent_t a, b; int kind; };
+    bool on = false;
+    std::vector<Rec> recs;  // event pairs, reused across profile runs
+    size_t used = 0;
+    void begin(int kind, cudaStream_t st);
+    void end(cudaStream_t st);
+    void release();
+};
+}  // namespace lococo
 
 struct lococo_handle {
     lococo_config cfg{};
@@ -16,6 +32,7 @@ struct lococo_handle {
     size_t off_status = 0, off_gpack = 0, off_bias = 0, off_s = 0, off_UK = 0, off_UV = 0, off_R = 0;
     size_t off_gimage = 0, off_part = 0, off_counter = 0;  // tensor-core path
     int64_t launches = 0;
+    lococo::Profiler prof;
 };
 
 namespace lococo {

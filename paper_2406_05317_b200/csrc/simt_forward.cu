@@ -357,7 +357,10 @@ static int compress_typed(const CompressParams& p, cudaStream_t st) {
     {
         dim3 grid((p.S + CT - 1) / CT, (p.M + CT - 1) / CT, p.units);
         const size_t smem = sizeof(float) * ((size_t)(CT + p.k - 1) * (CCH + 1) + (size_t)CT * (CCH + 1));
-        if (checked([&] { conv_relu_kernel<T><<<grid, 256, smem, st>>>(p); }) < 0) return -1;
+        prof_begin(p.prof, 0, st);
+        const int rc = checked([&] { conv_relu_kernel<T><<<grid, 256, smem, st>>>(p); });
+        prof_end(p.prof, st);
+        if (rc < 0) return -1;
         ++launches;
     }
     {
@@ -395,8 +398,11 @@ int simt_compress(int dtype, const CompressParams& p, cudaStream_t st) {
 template <typename T>
 static int attention_typed(const AttnParams& p, cudaStream_t st) {
     dim3 grid((p.b + 31) / 32, p.units);
-    if (p.d == 128) return checked([&] { attention_kernel<T, 128><<<grid, 128, 0, st>>>(p); });
-    return checked([&] { attention_kernel<T, 64><<<grid, 128, 0, st>>>(p); });
+    prof_begin(p.prof, 1, st);
+    const int rc = p.d == 128 ? checked([&] { attention_kernel<T, 128><<<grid, 128, 0, st>>>(p); })
+                              : checked([&] { attention_kernel<T, 64><<<grid, 128, 0, st>>>(p); });
+    prof_end(p.prof, st);
+    return rc;
 }
 
 int simt_attention(int dtype, const AttnParams& p, cudaStream_t st) {
