@@ -1,0 +1,327 @@
+"""Benchmark of the LoCoCo chunk loop (Algorithm 2) on the Llama-2-7B-shaped layer.
+
+One step = one pass of the whole hot path (chunk attention, conv logits, ReLU,
+normalisation, both blends, for all 8 chunks) over one 4096-token sequence of a
+32-head layer.  Prints ONE JSON line.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import tempfile
+import time
+from pathlib import Path
+
+ROOT = Path(__file__).resolve().parent
+if str(ROOT) not in sys.path:
+    sys.path.insert(0, str(ROOT))
+
+METRIC = "chunk-step tokens/sec per layer (32 heads)"
+UNIT = "tokens/s"
+WORKLOAD = "cfg2"
+
+
+# ------------------------------------------------------------------ algorithmic work
+def conv_flops(S, M, C, k):
+    return 2.0 * S * M * C * k
+
+
+def blend_flops(S, M, d):
+    return 4.0 * M * S * d
+
+
+def attn_flops(b, c, d):
+    return 4.0 * b * (c + (b + 1) / 2.0) * d
+
+
+def chunk_schedule(L, B, M):
+    """(cache_len, b, compress?) for every chunk of Algorithm 2 from an empty cache."""
+    out, c = [], 0
+    for t0 in range(0, L, B):
+        b = min(B, L - t0)
+        comp = c + b > M
+        out.append((c, b, comp))
+        c = M if comp else c + b
+    return out
+
+
+def sequence_flops(w):
+    """Algorithmic flops of one (sequence, head) unit: conv, blends, attention."""
+    conv = blend = attn = 0.0
+    for c, b, comp in chunk_schedule(w.L, w.B, w.M):
+        attn += attn_flops(b, c, w.d)
+        if comp:
+            conv += conv_flops(c + b, w.M, w.c_in, w.k)
+            blend += blend_flops(c + b, w.M, w.d)
+    return conv, blend, attn
+
+
+def measured_peaks():
+    p = ROOT / "MEASURED_PEAKS.json"
+    if p.exists():
+        j = json.loads(p.read_text())
+        return {"bf16_tflops": j["bf16_tflops"], "hbm_gbs": j["hbm_gbs"], "source": "measured"}
+    return {"bf16_tflops": 1590.0, "hbm_gbs": 6650.0, "source": "fallback"}
+
+
+# ------------------------------------------------------------------ clocks
+class ClockSampler:
+    FIELDS = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+              "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+              "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index: int):
+        self.gpu, self.proc, self.path = gpu_index, None, None
+
+    def start(self):
+        try:
+            fd, self.path = tempfile.mkstemp(suffix=".csv")
+            os.close(fd)
+            self.proc = subprocess.Popen(["nvidia-smi", "-i", str(self.gpu), f"--query-gpu={self.FIELDS}",
+                                          "--format=csv,noheader,nounits", "-lms", "100"],
+                                         stdout=open(self.path, "w"), stderr=subprocess.DEVNULL)
+        except Exception:
+            self.proc = None
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["unavailable"]}
+        time.sleep(0.15)
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        sm, mx, reasons = [], [], set()
+        for line in open(self.path).read().splitlines():
+            f = [x.strip() for x in line.split(",")]
+            if len(f) < 9:
+                continue
+            try:
+                sm.append(float(f[1]))
+                mx.append(float(f[2]))
+            except ValueError:
+                continue
+            for name, val in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"), f[5:9]):
+                if val.lower().startswith("active"):
+                    reasons.add(name)
+        os.unlink(self.path)
+        if not sm:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["no samples"]}
+        sm.sort()
+        return {"sm_mhz": sm[len(sm) // 2], "sm_max_mhz": max(mx), "reasons": sorted(reasons), "samples": len(sm)}
+
+
+# ------------------------------------------------------------------ the oracle arm
+def time_oracle(w, heads_sample, repeats=1):
+    """Times the float64 CPU oracle, as it stands, on `heads_sample` heads of the workload.
+    Returns (layer tokens/s scaled to all heads, seconds per sample run, threads)."""
+    from oracle import lococo_oracle as orc
+    from paper_2406_05317_b200 import workloads as wl
+    ws = w.slice(heads=heads_sample)
+    Q, K, V = wl.make_qkv(ws)
+    G, _ = wl.make_weights(ws)
+    times = []
+    for _ in range(repeats):
+        t = time.perf_counter()
+        orc.process_batch(Q, K, V, G, ws.B)
+        times.append(time.perf_counter() - t)
+    dt = sum(times) / len(times)
+    layer_seconds = dt * (w.heads / heads_sample)
+    return w.batch * w.L / layer_seconds, times, orc.threads()
+
+
+def run_reference(args):
+    """--impl reference: the CPU oracle on the host cores, same metric and workload."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    from oracle import lococo_oracle as orc
+    from paper_2406_05317_b200 import workloads as wl
+    w = wl.CONFIGS[WORKLOAD]
+    threads = orc.threads()
+    heads_sample = max(1, min(w.heads, threads))
+    ws = w.slice(heads=heads_sample)
+    Q, K, V = wl.make_qkv(ws)
+    G, _ = wl.make_weights(ws)
+    for _ in range(args.warmup):
+        orc.process_batch(Q, K, V, G, ws.B)
+    t = time.perf_counter()
+    for _ in range(args.steps):
+        orc.process_batch(Q, K, V, G, ws.B)
+    dt = (time.perf_counter() - t) / args.steps
+    layer_ms = dt * 1e3 * (w.heads / heads_sample)
+    value = w.batch * w.L / (layer_ms / 1e3)
+    sample = f"{heads_sample} of {w.heads} heads, all {w.n_chunks} chunks, scaled by {w.heads}/{heads_sample}"
+    print(json.dumps({
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": layer_ms, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": f"{WORKLOAD}: Llama-2-7B-shaped layer, 32 heads, d=128, M=128, B=512, k=21, L=4096, "
+                               "batch 1, per-head conv weights"},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": threads, "kind": "oracle", "sample": sample},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+    }))
+
+
+# ------------------------------------------------------------------ our arm
+def run_ours(args):
+    import torch
+    import torch.distributed as dist
+
+    from paper_2406_05317_b200 import api, sharding, workloads as wl
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    torch.cuda.set_device(local_rank)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+    w = wl.CONFIGS[WORKLOAD]
+    tdt = torch.bfloat16
+
+    # weak scaling: every rank runs one whole sequence of its own (sequence index = rank)
+    seq = list(sharding.weak_scaling_sequences(world, rank))[0]
+    Qh, Kh, Vh = (torch.from_numpy(x[None]).to(tdt).pin_memory() for x in wl.make_sequence(w, seq))
+    G, _ = wl.make_weights(w)
+    ctx = api.Lococo(w.batch, w.heads, w.d, w.M, w.k, w.B, dtype=tdt, c_in=w.c_in, weights_per_head=w.weights_per_head)
+    ctx.set_weights(torch.from_numpy(G).cuda().to(tdt))
+    Q, K, V = Qh.cuda(), Kh.cuda(), Vh.cuda()
+    O = torch.empty_like(Q)
+    Kc = torch.zeros(w.batch, w.heads, w.M, w.d, dtype=tdt, device="cuda")
+    Vc = torch.zeros_like(Kc)
+    Oh = torch.empty_like(Qh).pin_memory()
+    Kch = torch.empty(w.batch, w.heads, w.M, w.d, dtype=tdt).pin_memory()
+    Vch = torch.empty_like(Kch).pin_memory()
+    staging = torch.empty(ctx.host_staging_bytes(w.L), dtype=torch.uint8, device="cuda")
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")   # larger than the 126 MB L2
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    def step_device():
+        flush.fill_(1)
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record()
+        ctx.process_sequence(Q, K, V, w.B, O, Kc, Vc, 0)
+        b.record()
+        return a, b
+
+    def step_host():
+        flush.fill_(1)
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record()
+        ctx.process_sequence_host(Qh, Kh, Vh, w.B, Oh, staging, Kch, Vch)
+        b.record()
+        return a, b
+
+    for _ in range(args.warmup):
+        step_device()
+    barrier()
+    sampler = ClockSampler(local_rank)
+    if rank == 0:
+        sampler.start()
+    launches0 = ctx.launch_count()
+    events = [step_device() for _ in range(args.steps)]
+    barrier()
+    launches = ctx.launch_count() - launches0
+    clocks = sampler.stop() if rank == 0 else None
+    local_ms = sum(a.elapsed_time(b) for a, b in events)
+    assert ctx.device_status() == api.OK
+
+    # per-kernel timing of the same steps (CUDA events on the launching stream, in the library)
+    ctx.profile(True)
+    for _ in range(args.steps):
+        step_device()
+    torch.cuda.synchronize()
+    conv_ms, conv_n = ctx.profile_read(0)
+    attn_ms, attn_n = ctx.profile_read(1)
+    ctx.profile(False)
+
+    # end to end through the host-buffer entry point
+    for _ in range(min(args.warmup, 3)):
+        step_host()
+    barrier()
+    e2e_steps = max(1, min(args.steps, 10))
+    ev = [step_host() for _ in range(e2e_steps)]
+    barrier()
+    e2e_local_ms = sum(a.elapsed_time(b) for a, b in ev) * (args.steps / e2e_steps)
+
+    tokens = float(w.batch * w.L * args.steps)
+    total_ms, total_tokens = sharding.aggregate_throughput(dist if world > 1 else None, local_ms, tokens)
+    e2e_ms, _ = sharding.aggregate_throughput(dist if world > 1 else None, e2e_local_ms, tokens)
+    if rank != 0:
+        if world > 1:
+            dist.destroy_process_group()
+        return
+
+    peaks = measured_peaks()
+    conv_f, blend_f, attn_f = sequence_flops(w)
+    units = w.batch * w.heads
+    n_comp = sum(1 for _, _, comp in chunk_schedule(w.L, w.B, w.M) if comp)
+    fused = bool(getattr(api, "TENSOR_PATH_FUSES_BLEND", False))
+    dom_flops_per_seq = units * (conv_f + (blend_f if fused else 0.0))
+    conv_per_launch_ms = conv_ms / max(conv_n, 1)
+    flops_per_launch = dom_flops_per_seq / n_comp
+    achieved = flops_per_launch / (conv_per_launch_ms * 1e-3) / 1e12 if conv_n else None
+    step_flops = units * (conv_f + blend_f + attn_f)
+    seq_bytes = 4.0 * units * w.L * w.d * 2 + units * 2 * w.M * w.d * 2 + w.heads * w.M * w.c_in * w.k * 2
+    roof_ms = max(step_flops / (peaks["bf16_tflops"] * 1e12), seq_bytes / (peaks["hbm_gbs"] * 1e9)) * 1e3
+
+    out = {
+        "metric": METRIC, "value": total_tokens / (total_ms * 1e-3), "unit": UNIT, "n_gpus": world,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": total_ms / args.steps,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+        "config": {"workload": f"{WORKLOAD}: Llama-2-7B-shaped layer, 32 heads, d=128, M=128, B=512, k=21, L=4096, "
+                               "batch 1 per GPU, per-head conv weights, c_in=d",
+                   "l2": "256 MB flush between timed steps", "chunks_per_step": w.n_chunks,
+                   "parallelism": f"sequences x{world} (no collective)"},
+        "clocks": clocks,
+        "e2e": {"value": total_tokens / (e2e_ms * 1e-3), "unit": UNIT,
+                "h2d_bytes_per_step": 3 * Qh.numel() * 2, "d2h_bytes_per_step": (Oh.numel() + 2 * Kch.numel()) * 2},
+        "gpu_launches": launches,
+        "step_roofline": {"flops_per_step": step_flops, "bytes_per_step": seq_bytes, "roofline_ms": roof_ms,
+                          "frac": roof_ms / (total_ms / args.steps), "peak_source": peaks["source"] + " burst"},
+        "roofline": {"bound": "tensor", "kernel": "Eq. 6 conv" + (" + blends (fused)" if fused else ""),
+                     "achieved": achieved, "peak": peaks["bf16_tflops"], "unit": "TFLOP/s",
+                     "frac": (achieved / peaks["bf16_tflops"]) if achieved else None, "traffic": None,
+                     "peak_source": peaks["source"] + " burst", "launches": conv_n,
+                     "us_per_launch": conv_per_launch_ms * 1e3,
+                     "attention_us_per_launch": attn_ms / max(attn_n, 1) * 1e3},
+    }
+    if world == 1:
+        from oracle import lococo_oracle as orc
+        threads = orc.threads()
+        heads_sample = w.heads if threads >= 8 else max(1, min(w.heads, 2 * threads))
+        value, times, threads = time_oracle(w, heads_sample)
+        out["cpu_baseline"] = {"value": value, "unit": UNIT, "cores": threads, "kind": "oracle",
+                               "sample": f"{heads_sample} of {w.heads} heads, all {w.n_chunks} chunks, "
+                                         f"{times[0]:.1f} s, scaled by {w.heads}/{heads_sample}"}
+    print(json.dumps(out))
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()
