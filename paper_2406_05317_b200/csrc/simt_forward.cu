@@ -391,6 +391,12 @@ static int compress_typed(const CompressParams& p, cudaStream_t st) {
     return launches;
 }
 
+int simt_write_weights(const float* R, const float* s, float* W, int64_t rows, int S, cudaStream_t st) {
+    const int64_t total = rows * S;
+    const int blocks = (int)((total + 255) / 256 < 8192 ? (total + 255) / 256 : 8192);
+    return checked([&] { write_weights_kernel<<<blocks, 256, 0, st>>>(R, s, W, rows, S); });
+}
+
 int simt_compress(int dtype, const CompressParams& p, cudaStream_t st) {
     return dtype == LOCOCO_F32 ? compress_typed<float>(p, st) : compress_typed<__nv_bfloat16>(p, st);
 }

@@ -1,13 +1,396 @@
-// Tensor-core (tcgen05 / TMEM) kernels of the LoCoCo chunk step.
+// Tensor-core (tcgen05 / TMEM) kernels of the LoCoCo chunk step, bf16 storage, d = 128.
+//
+// compress_tc_kernel fuses Algorithm 2's Steps 4 and 5 for one tile of positions:
+//   1. the [cache; chunk] key and value rows of the tile (plus a (k-1)/2 halo) are staged
+//      once in shared memory, un-swizzled, as [8-channel group][row][8 channels];
+//   2. Eq. 6 runs as an implicit GEMM on the tensor cores: for every tap t,
+//      D[slot, pos] += G_t[slot, ch] * Z[pos + t, ch]; a tap is a row offset into the
+//      staged tile, which the un-swizzled layout allows at 16-byte granularity; the
+//      per-tap weight tiles stream from L2 through a ring fed by bulk async copies;
+//   3. the accumulator leaves TMEM once: bias, ReLU, the running row sum of Eq. 7, bf16
+//      rounding, and the result is written back to shared memory as the A operand of
+//   4. Eq. 4 / Eq. 5: U_K += R * X_K and U_V += R * X_V, which read the SAME staged tiles,
+//      now contracted over positions (MN-major B operand);
+// and the division by the row sum is applied after all tiles are summed (it commutes
+// with the blend), by finalize_parts_kernel.
+#include <algorithm>
+
 #include "handle.h"
+#include "tc_common.cuh"
 
 namespace lococo {
+namespace {
 
-bool tensor_config_supported(const lococo_config*) { return false; }
-void tensor_layout_workspace(lococo_handle*, size_t*) {}
-int tensor_pack_weights(lococo_handle*, const void*, cudaStream_t) { return 0; }
-bool tensor_compress_supported(const lococo_handle*, const CompressParams&) { return false; }
-int tensor_compress(lococo_handle*, const CompressParams&, cudaStream_t) { return -1; }
+using namespace tc;
+
+constexpr int kSlots = 128;              // slots per CTA (MMA M)
+constexpr int kD = 128;                  // head dimension
+constexpr int kStageBytes = 32768;       // one tap x 128 channels x 128 slots, bf16
+constexpr int kThreads = 160;            // 4 loader/epilogue warps + 1 control warp
+constexpr int kMaxSmem = 232448;         // 227 KB
+constexpr uint32_t kTmemCols = 512;
+constexpr uint32_t kColUK = 256, kColUV = 384;
+
+struct TcCompressParams {
+    CompressParams base;
+    const __nv_bfloat16* gimage;  // [sets][slot blocks][k][halves][16][128][8]
+    float* part_U;                // [units][slot blocks][parts][2][128][128]
+    float* part_s;                // [units][slot blocks][parts][128]
+    float* R_store;               // optional [units][M][S]
+    int* status;
+    int n_tile, tiles, parts, tiles_per_part, halves, stages, rows_pad, slot_blocks;
+};
+
+// G [sets][M][C][k] -> per (set, slot block, tap, 128-channel half) a 32 KB image of the
+// K-major un-swizzled MMA operand: [16 channel groups][128 slots][8 channels].
+__global__ void pack_image_kernel(const __nv_bfloat16* __restrict__ G, __nv_bfloat16* __restrict__ out, int sets, int M,
+                                  int C, int k) {
+    const int64_t total = (int64_t)sets * M * C * k;
+    const int SB = M / kSlots, halves = C / 128;
+    for (int64_t o = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; o < total; o += (int64_t)gridDim.x * blockDim.x) {
+        int64_t r = o;
+        const int e = r % 8; r /= 8;
+        const int i = r % kSlots; r /= kSlots;
+        const int q = r % 16; r /= 16;
+        const int half = r % halves; r /= halves;
+        const int t = r % k; r /= k;
+        const int sb = r % SB;
+        const int set = r / SB;
+        const int slot = sb * kSlots + i, ch = half * 128 + q * 8 + e;
+        out[o] = G[(((int64_t)set * M + slot) * C + ch) * k + t];
+    }
+}
+
+__global__ void __launch_bounds__(kThreads, 1) compress_tc_kernel(const __grid_constant__ TcCompressParams P) {
+    extern __shared__ __align__(128) uint8_t smem[];
+    const CompressParams& p = P.base;
+    const int part = blockIdx.x, sb = blockIdx.y, u = blockIdx.z;
+    const int n = u / p.heads, h = u % p.heads;
+    const int tid = threadIdx.x, warp = tid >> 5;
+    const int n_tile = P.n_tile, pad = (p.k - 1) / 2, rows = n_tile + p.k - 1;
+    const int NS = P.stages;
+    const uint32_t lbo_z = (uint32_t)P.rows_pad * 16u;
+
+    uint8_t* ring_ptr = smem;
+    uint8_t* zk_ptr = ring_ptr + (size_t)NS * kStageBytes;
+    uint8_t* zv_ptr = zk_ptr + 16 * lbo_z;
+    uint64_t* bars = reinterpret_cast<uint64_t*>(zv_ptr + 16 * lbo_z);
+    volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(bars + 2 * NS + 2);
+    volatile int* failed = reinterpret_cast<volatile int*>(tmem_slot + 1);
+    const uint32_t ring = smem_u32(ring_ptr), zk = smem_u32(zk_ptr), zv = smem_u32(zv_ptr);
+    const uint32_t bar_full = smem_u32(bars), bar_empty = bar_full + 8 * NS;
+    const uint32_t bar_acc = bar_empty + 8 * NS, bar_blend = bar_acc + 8;
+
+    if (tid == 128) {
+        for (int s = 0; s < NS; ++s) {
+            mbar_init(bar_full + 8 * s, 1);
+            mbar_init(bar_empty + 8 * s, 1);
+        }
+        mbar_init(bar_acc, 1);
+        mbar_init(bar_blend, 1);
+        *failed = 0;
+        fence_barrier_init();
+    }
+    if (warp == 4) {
+        __syncwarp();
+        tmem_alloc(smem_u32(const_cast<uint32_t*>(tmem_slot)), kTmemCols);
+        tmem_relinquish();
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem = *tmem_slot;
+
+    const int set = p.weights_per_head ? h : 0;
+    const __nv_bfloat16* gimg =
+        P.gimage + ((int64_t)set * P.slot_blocks + sb) * (int64_t)p.k * P.halves * (kStageBytes / 2);
+    const uint32_t idesc_conv = instr_desc_bf16(n_tile, false, false);
+    const uint32_t idesc_blend = instr_desc_bf16(kD, false, true);
+    const int slot = sb * kSlots + tid;  // meaningful for tid < 128
+    float bias_i = 0.f;
+    if (tid < kSlots && p.bias) bias_i = p.bias[(p.weights_per_head ? h * p.M : 0) + slot];
+    const __nv_bfloat16* safe = unit_base<__nv_bfloat16>(p.xk.chunk, n, h);
+
+    float ssum = 0.f;
+    uint32_t g = 0;  // ring iterations issued so far (control thread)
+    const int tile_begin = part * P.tiles_per_part;
+    const int tile_end = min(P.tiles, tile_begin + P.tiles_per_part);
+    int tile_it = 0;
+    for (int tile = tile_begin; tile < tile_end; ++tile, ++tile_it) {
+        const int j0 = tile * n_tile;
+        // ---- 1. stage the key and value rows j0-pad .. j0+n_tile+pad-1 (zeros outside [0,S))
+        for (int x = tid; x < rows * 16; x += kThreads) {
+            const int r = x >> 4, q = x & 15;
+            const int j = j0 - pad + r;
+            const bool valid = j >= 0 && j < p.S;
+            const __nv_bfloat16* sk = valid ? cat_row<__nv_bfloat16>(p.xk, n, h, j) + q * 8 : safe;
+            const __nv_bfloat16* sv = valid ? cat_row<__nv_bfloat16>(p.xv, n, h, j) + q * 8 : safe;
+            const uint32_t off = q * lbo_z + r * 16;
+            cp_async16(zk + off, sk, valid ? 16u : 0u);
+            cp_async16(zv + off, sv, valid ? 16u : 0u);
+        }
+        cp_async_wait_all();
+        fence_proxy_async();
+        __syncthreads();
+
+        // ---- 2. Eq. 6 as an implicit GEMM: one ring stage per (tap, 128-channel half)
+        if (tid == 128) {
+            const int total = p.k * P.halves;
+            auto load = [&](uint32_t gg, int it) {
+                const uint32_t s = gg % NS;
+                if (gg >= (uint32_t)NS) mbar_wait(bar_empty + 8 * s, ((gg / NS) - 1) & 1, P.status, failed, 1);
+                mbar_expect_tx(bar_full + 8 * s, kStageBytes);
+                bulk_load(ring + s * kStageBytes, gimg + (int64_t)it * (kStageBytes / 2), kStageBytes, bar_full + 8 * s);
+            };
+            const int npro = min(NS, total);
+            for (int i = 0; i < npro; ++i) load(g + i, i);
+            for (int it = 0; it < total; ++it) {
+                const uint32_t gg = g + it, s = gg % NS;
+                mbar_wait(bar_full + 8 * s, (gg / NS) & 1, P.status, failed, 2);
+                tc_fence_after();
+                const int t = it / P.halves, half = it % P.halves;
+                const uint32_t zbase = (half == 0 ? zk : zv) + t * 16;
+                const uint32_t abase = ring + s * kStageBytes;
+#pragma unroll
+                for (int kk = 0; kk < 8; ++kk) {
+                    const uint64_t ad = smem_desc(abase + kk * 2 * 2048, 2048, 128);
+                    const uint64_t bd = smem_desc(zbase + kk * 2 * lbo_z, lbo_z, 128);
+                    umma_ss(tmem, ad, bd, idesc_conv, (it | kk) != 0);
+                }
+                umma_commit(bar_empty + 8 * s);
+                if (it >= 1 && it - 1 + NS < total) load(gg - 1 + NS, it - 1 + NS);
+            }
+            umma_commit(bar_acc);
+            g += total;
+        }
+
+        // ---- 3. accumulator -> bias, ReLU, row sum (Eq. 7), bf16 -> A operand of the blends
+        if (warp < 4) {
+            mbar_wait(bar_acc, tile_it & 1, P.status, failed, 3);
+            tc_fence_after();
+            const uint32_t lane_addr = tmem + ((uint32_t)(warp * 32) << 16);
+            float* rstore = P.R_store ? P.R_store + ((int64_t)u * p.M + slot) * p.S : nullptr;
+            for (int c0 = 0; c0 < n_tile; c0 += 32) {
+                uint32_t v[32];
+                tmem_ld32(lane_addr + c0, v);
+                tmem_ld_wait();
+#pragma unroll
+                for (int e = 0; e < 32; e += 8) {
+                    uint32_t pk[4];
+#pragma unroll
+                    for (int x = 0; x < 8; x += 2) {
+                        const int ja = j0 + c0 + e + x;
+                        float ra = fmaxf(__uint_as_float(v[e + x]) + bias_i, 0.f);
+                        float rb = fmaxf(__uint_as_float(v[e + x + 1]) + bias_i, 0.f);
+                        if (ja >= p.S) ra = 0.f;
+                        if (ja + 1 >= p.S) rb = 0.f;
+                        const __nv_bfloat162 pr = __floats2bfloat162_rn(ra, rb);
+                        pk[x >> 1] = *reinterpret_cast<const uint32_t*>(&pr);
+                        const float fa = __low2float(pr), fb = __high2float(pr);
+                        ssum += fa + fb;
+                        if (rstore) {
+                            if (ja < p.S) rstore[ja] = fa;
+                            if (ja + 1 < p.S) rstore[ja + 1] = fb;
+                        }
+                    }
+                    *reinterpret_cast<uint4*>(ring_ptr + ((c0 + e) >> 3) * 2048 + tid * 16) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
+                }
+            }
+            fence_proxy_async();
+        }
+        tc_fence_before();
+        __syncthreads();
+
+        // ---- 4. Eq. 4, Eq. 5 (unnormalised): U_K += R X_K, U_V += R X_V from the staged tiles
+        if (tid == 128) {
+            tc_fence_after();
+            for (int kk = 0; kk < n_tile / 16; ++kk) {
+                const uint64_t ad = smem_desc(ring + kk * 2 * 2048, 2048, 128);
+                const uint32_t row0 = (uint32_t)(pad + kk * 16) * 16;
+                const uint64_t bk = smem_desc(zk + row0, 128, lbo_z);
+                const uint64_t bv = smem_desc(zv + row0, 128, lbo_z);
+                const uint32_t acc = (tile_it | kk) != 0;
+                umma_ss(tmem + kColUK, ad, bk, idesc_blend, acc);
+                umma_ss(tmem + kColUV, ad, bv, idesc_blend, acc);
+            }
+            umma_commit(bar_blend);
+        }
+        // the staged tiles and the ring are reused by the next tile only after the blends read them
+        mbar_wait(bar_blend, tile_it & 1, P.status, failed, 4);
+    }
+
+    // ---- partial blends and row sums of this CTA's tiles
+    if (warp < 4 && tile_it > 0) {
+        tc_fence_after();
+        const uint32_t lane_addr = tmem + ((uint32_t)(warp * 32) << 16);
+        const int64_t pidx = ((int64_t)u * P.slot_blocks + sb) * P.parts + part;
+        float* outK = P.part_U + (pidx * 2 + 0) * (kSlots * kD) + tid * kD;
+        float* outV = P.part_U + (pidx * 2 + 1) * (kSlots * kD) + tid * kD;
+#pragma unroll 1
+        for (int c0 = 0; c0 < kD; c0 += 32) {
+            uint32_t a[32], b[32];
+            tmem_ld32(lane_addr + kColUK + c0, a);
+            tmem_ld32(lane_addr + kColUV + c0, b);
+            tmem_ld_wait();
+#pragma unroll
+            for (int e = 0; e < 32; e += 4) {
+                *reinterpret_cast<uint4*>(outK + c0 + e) = make_uint4(a[e], a[e + 1], a[e + 2], a[e + 3]);
+                *reinterpret_cast<uint4*>(outV + c0 + e) = make_uint4(b[e], b[e + 1], b[e + 2], b[e + 3]);
+            }
+        }
+        P.part_s[pidx * kSlots + tid] = ssum;
+    }
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 4) {
+        __syncwarp();
+        tmem_dealloc(tmem, kTmemCols);
+    }
+}
+
+// cache = (sum of partial blends) / (sum of partial row sums + eps)   (Eq. 7 after Eq. 4-5)
+__global__ void finalize_parts_kernel(TcCompressParams P) {
+    const CompressParams& p = P.base;
+    const int u = blockIdx.y, n = u / p.heads, h = u % p.heads;
+    const int x = blockIdx.x * blockDim.x + threadIdx.x;
+    if (x >= p.M * kD) return;
+    const int i = x / kD, ch = x % kD, sb = i / kSlots, il = i % kSlots;
+    const int64_t base = ((int64_t)u * P.slot_blocks + sb) * P.parts;
+    float s = 0.f, uk = 0.f, uv = 0.f;
+    for (int pt = 0; pt < P.parts; ++pt) {
+        s += P.part_s[(base + pt) * kSlots + il];
+        uk += P.part_U[((base + pt) * 2 + 0) * (kSlots * kD) + il * kD + ch];
+        uv += P.part_U[((base + pt) * 2 + 1) * (kSlots * kD) + il * kD + ch];
+    }
+    s += p.eps;
+    const float inv = 1.f / s;
+    unit_base_mut<__nv_bfloat16>(p.k_out, n, h)[(int64_t)i * p.k_out.st + ch] = __float2bfloat16_rn(uk * inv);
+    unit_base_mut<__nv_bfloat16>(p.v_out, n, h)[(int64_t)i * p.v_out.st + ch] = __float2bfloat16_rn(uv * inv);
+    if (ch == 0) p.s[(int64_t)u * p.M + i] = s;
+}
+
+struct Plan {
+    int n_tile, tiles, parts, tiles_per_part, stages, rows_pad;
+    size_t smem;
+};
+
+int parts_cap(int units, int slot_blocks) {
+    const int pairs = units * slot_blocks;
+    return (600 + pairs - 1) / pairs;
+}
+
+size_t smem_bytes(int n_tile, int k, int stages) {
+    const int rows_pad = (n_tile + k - 1) | 1;
+    return (size_t)stages * kStageBytes + 2 * 16 * (size_t)rows_pad * 16 + (2 * stages + 2) * 8 + 16;
+}
+
+// Tile width and CTA count: fewest waves of 148 SMs, then least padded work.
+bool make_plan(int S, int k, int units, int slot_blocks, Plan* out) {
+    double best = 1e30;
+    const int cap = parts_cap(units, slot_blocks);
+    for (int n_tile = 160; n_tile >= 64; n_tile -= 32) {
+        int stages = 4;
+        while (stages >= 2 && smem_bytes(n_tile, k, stages) > (size_t)kMaxSmem) --stages;
+        if (stages < 2 || (size_t)stages * kStageBytes < (size_t)n_tile * kSlots * 2) continue;
+        const int tiles = (S + n_tile - 1) / n_tile;
+        for (int parts = 1; parts <= tiles && parts <= cap; ++parts) {
+            const int tpp = (tiles + parts - 1) / parts;
+            const int parts_eff = (tiles + tpp - 1) / tpp;
+            const long ctas = (long)units * slot_blocks * parts_eff;
+            const long waves = (ctas + 147) / 148;
+            const double cost = (double)waves * tpp * (n_tile + 24) + (stages < 4 ? 1.0 : 0.0);
+            if (cost < best) {
+                best = cost;
+                *out = Plan{n_tile, tiles, parts_eff, tpp, stages, (n_tile + k - 1) | 1, smem_bytes(n_tile, k, stages)};
+            }
+        }
+    }
+    return best < 1e30;
+}
+
+}  // namespace
+
+int simt_write_weights(const float* R, const float* s, float* W, int64_t rows, int S, cudaStream_t st);
+
+bool tensor_config_supported(const lococo_config* c) {
+    if (c->dtype != LOCOCO_BF16 || c->head_dim != kD) return false;
+    if (c->M % kSlots != 0) return false;
+    Plan pl;
+    return make_plan(c->M + c->max_chunk, c->k, c->batch * c->heads, c->M / kSlots, &pl);
+}
+
+void tensor_layout_workspace(lococo_handle* h, size_t* off) {
+    if (!h->use_tensor) return;
+    const lococo_config& c = h->cfg;
+    auto align = [](size_t x) { return (x + 255) / 256 * 256; };
+    const size_t sets = c.weights_per_head ? c.heads : 1;
+    const int SB = c.M / kSlots;
+    const int Smax = c.M + c.max_chunk;
+    const int max_parts = std::min(parts_cap(h->units, SB), (Smax + 63) / 64);
+    h->off_gimage = *off;
+    *off = align(*off + sets * (size_t)c.M * c.c_in * c.k * 2);
+    h->off_part = *off;
+    *off = align(*off + (size_t)h->units * SB * max_parts * (2 * kSlots * kD + kSlots) * sizeof(float));
+}
+
+int tensor_pack_weights(lococo_handle* h, const void* G, cudaStream_t st) {
+    const lococo_config& c = h->cfg;
+    const int sets = c.weights_per_head ? c.heads : 1;
+    const int64_t total = (int64_t)sets * c.M * c.c_in * c.k;
+    const int blocks = (int)std::min<int64_t>((total + 255) / 256, 8192);
+    pack_image_kernel<<<blocks, 256, 0, st>>>((const __nv_bfloat16*)G, (__nv_bfloat16*)(h->ws + h->off_gimage), sets, c.M,
+                                              c.c_in, c.k);
+    return cudaGetLastError() == cudaSuccess ? 1 : -1;
+}
+
+bool tensor_compress_supported(const lococo_handle* h, const CompressParams& p) {
+    Plan pl;
+    return h->use_tensor && p.S >= 1 && make_plan(p.S, p.k, p.units, p.M / kSlots, &pl);
+}
+
+int tensor_compress(lococo_handle* h, const CompressParams& p, cudaStream_t st) {
+    const int SB = p.M / kSlots;
+    Plan pl;
+    if (!make_plan(p.S, p.k, p.units, SB, &pl)) return -1;
+    static bool attr_set = false;
+    if (!attr_set) {
+        if (cudaFuncSetAttribute(compress_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxSmem) != cudaSuccess)
+            return -1;
+        attr_set = true;
+    }
+    const int Smax = h->cfg.M + h->cfg.max_chunk;
+    const int max_parts = std::min(parts_cap(h->units, SB), (Smax + 63) / 64);
+    if (pl.parts > max_parts) return -1;
+    TcCompressParams P{};
+    P.base = p;
+    P.gimage = reinterpret_cast<const __nv_bfloat16*>(h->ws + h->off_gimage);
+    P.part_U = reinterpret_cast<float*>(h->ws + h->off_part);
+    P.part_s = P.part_U + (size_t)p.units * SB * max_parts * 2 * kSlots * kD;
+    P.R_store = p.W_out ? p.R : nullptr;
+    P.status = reinterpret_cast<int*>(h->ws + h->off_status);
+    P.n_tile = pl.n_tile; P.tiles = pl.tiles; P.parts = pl.parts; P.tiles_per_part = pl.tiles_per_part;
+    P.halves = p.c_in / 128; P.stages = pl.stages; P.rows_pad = pl.rows_pad; P.slot_blocks = SB;
+    int launches = 0;
+    dim3 grid(pl.parts, SB, p.units);
+    prof_begin(p.prof, 0, st);
+    // the full 227 KB keeps one CTA per SM, so a CTA always finds its 512 TMEM columns free
+    compress_tc_kernel<<<grid, kThreads, kMaxSmem, st>>>(P);
+    const bool ok = cudaGetLastError() == cudaSuccess;
+    prof_end(p.prof, st);
+    if (!ok) return -1;
+    ++launches;
+    dim3 fgrid((p.M * kD + 255) / 256, p.units);
+    finalize_parts_kernel<<<fgrid, 256, 0, st>>>(P);
+    if (cudaGetLastError() != cudaSuccess) return -1;
+    ++launches;
+    if (p.W_out) {
+        const int r = simt_write_weights(p.R, p.s, p.W_out, (int64_t)p.units * p.M, p.S, st);
+        if (r < 0) return -1;
+        launches += r;
+    }
+    return launches;
+}
+
 bool tensor_attention_supported(const lococo_handle*, const AttnParams&) { return false; }
 int tensor_attention(lococo_handle*, const AttnParams&, cudaStream_t) { return -1; }
 
