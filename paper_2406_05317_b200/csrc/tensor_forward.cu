@@ -269,6 +269,221 @@ __global__ void finalize_parts_kernel(TcCompressParams P) {
     if (ch == 0) p.s[(int64_t)u * p.M + i] = s;
 }
 
+
+// ------------------------------------------------------------------ Eq. 1, chunk form
+// One CTA = 128 queries of one unit. Per 128-key tile of [cache; chunk]:
+//   S = Q K^T on the tensor cores (both operands K-major, staged un-swizzled),
+//   one thread per query row reads its S row from TMEM, applies the scale, the causal
+//   mask and the running-max update, and writes P (bf16) to shared memory,
+//   O_tile = P V on the tensor cores (V read MN-major from its staged tile),
+//   and the row's fp32 accumulator is rescaled and updated in registers.
+constexpr int kAttnThreads = 160;
+constexpr uint32_t kLboT = 129 * 16;               // byte stride between 8-channel groups of a staged 128-row tile
+constexpr uint32_t kTileBytes = 16 * kLboT;        // 33024
+constexpr uint32_t kPBytes = 16 * 2048;            // P tile: [16 key groups][128 rows][8 keys]
+constexpr uint32_t kAttnSmem = 5 * kTileBytes + kPBytes + 64;
+constexpr uint32_t kAttnTmemCols = 256;
+
+struct TcAttnParams {
+    AttnParams base;
+    int* status;
+};
+
+__global__ void __launch_bounds__(kAttnThreads, 1) attention_tc_kernel(const __grid_constant__ TcAttnParams P) {
+    extern __shared__ __align__(128) uint8_t smem[];
+    const AttnParams& p = P.base;
+    const int u = blockIdx.y, n = u / p.heads, h = u % p.heads;
+    const int tid = threadIdx.x, warp = tid >> 5;
+    const int r0 = blockIdx.x * 128;
+    const int S = p.c + p.b;
+
+    uint8_t* q_ptr = smem;
+    uint8_t* k_ptr = q_ptr + kTileBytes;       // two buffers
+    uint8_t* v_ptr = k_ptr + 2 * kTileBytes;   // two buffers
+    uint8_t* p_ptr = v_ptr + 2 * kTileBytes;
+    uint64_t* bars = reinterpret_cast<uint64_t*>(p_ptr + kPBytes);
+    volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(bars + 2);
+    volatile int* failed = reinterpret_cast<volatile int*>(tmem_slot + 1);
+    const uint32_t qs = smem_u32(q_ptr), ks = smem_u32(k_ptr), vs = smem_u32(v_ptr), ps = smem_u32(p_ptr);
+    const uint32_t bar_s = smem_u32(bars), bar_o = bar_s + 8;
+
+    if (tid == 128) {
+        mbar_init(bar_s, 1);
+        mbar_init(bar_o, 1);
+        *failed = 0;
+        fence_barrier_init();
+    }
+    if (warp == 4) {
+        __syncwarp();
+        tmem_alloc(smem_u32(const_cast<uint32_t*>(tmem_slot)), kAttnTmemCols);
+        tmem_relinquish();
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem = *tmem_slot;
+
+    const int last_row = min(r0 + 127, p.b - 1);
+    const int ncols = p.c + last_row + 1;           // columns any query of this tile can see
+    const int ntiles = (ncols + 127) / 128;
+    const __nv_bfloat16* safe = unit_base<__nv_bfloat16>(p.q, n, h);
+
+    auto load_kv = [&](int jt, int buf) {
+        const int j0 = jt * 128;
+        for (int x = tid; x < 128 * 16; x += kAttnThreads) {
+            const int r = x >> 4, q = x & 15;
+            const int j = j0 + r;
+            const bool valid = j < S;
+            const __nv_bfloat16* sk = valid ? cat_row<__nv_bfloat16>(p.xk, n, h, j) + q * 8 : safe;
+            const __nv_bfloat16* sv = valid ? cat_row<__nv_bfloat16>(p.xv, n, h, j) + q * 8 : safe;
+            const uint32_t off = buf * kTileBytes + q * kLboT + r * 16;
+            cp_async16(ks + off, sk, valid ? 16u : 0u);
+            cp_async16(vs + off, sv, valid ? 16u : 0u);
+        }
+    };
+    // queries of this tile (zeros beyond the chunk) and the first key/value tile
+    for (int x = tid; x < 128 * 16; x += kAttnThreads) {
+        const int r = x >> 4, q = x & 15;
+        const bool valid = r0 + r < p.b;
+        const __nv_bfloat16* sq = valid ? unit_base<__nv_bfloat16>(p.q, n, h) + (int64_t)(r0 + r) * p.q.st + q * 8 : safe;
+        cp_async16(qs + q * kLboT + r * 16, sq, valid ? 16u : 0u);
+    }
+    load_kv(0, 0);
+    asm volatile("cp.async.commit_group;" ::: "memory");
+
+    const uint32_t idesc_s = instr_desc_bf16(128, false, false);
+    const uint32_t idesc_o = instr_desc_bf16(128, false, true);
+    const int row = r0 + tid;                       // compute threads only
+    const bool live = tid < 128 && row < p.b;
+    const int vis = live ? p.c + row + 1 : 1;       // visible columns of this row
+    const float sc2 = p.scale * 1.4426950408889634f;
+    float acc[128];
+#pragma unroll
+    for (int e = 0; e < 128; ++e) acc[e] = 0.f;
+    float mrun = -INFINITY, lrun = 0.f;
+    const uint32_t lane_addr = tmem + ((uint32_t)((warp & 3) * 32) << 16);
+
+    for (int jt = 0; jt < ntiles; ++jt) {
+        const int buf = jt & 1;
+        if (jt + 1 < ntiles) {
+            load_kv(jt + 1, buf ^ 1);
+            asm volatile("cp.async.commit_group;" ::: "memory");
+            asm volatile("cp.async.wait_group 1;" ::: "memory");
+        } else {
+            asm volatile("cp.async.wait_group 0;" ::: "memory");
+        }
+        fence_proxy_async();
+        __syncthreads();
+        if (tid == 128) {
+            tc_fence_after();
+#pragma unroll
+            for (int kk = 0; kk < 8; ++kk) {
+                const uint64_t ad = smem_desc(qs + kk * 2 * kLboT, kLboT, 128);
+                const uint64_t bd = smem_desc(ks + buf * kTileBytes + kk * 2 * kLboT, kLboT, 128);
+                umma_ss(tmem, ad, bd, idesc_s, kk != 0);
+            }
+            umma_commit(bar_s);
+        }
+        float corr = 1.f;
+        if (warp < 4) {
+            mbar_wait(bar_s, jt & 1, P.status, failed, 5);
+            tc_fence_after();
+            const int j0 = jt * 128;
+            const bool need_mask = j0 + 128 > p.c + r0;
+            // pass 1: row maximum of the scaled, masked logits
+            float tmax = -INFINITY;
+#pragma unroll 1
+            for (int c0 = 0; c0 < 128; c0 += 32) {
+                uint32_t v[32];
+                tmem_ld32(lane_addr + c0, v);
+                tmem_ld_wait();
+#pragma unroll
+                for (int e = 0; e < 32; ++e) {
+                    const float s2 = __uint_as_float(v[e]) * sc2;
+                    if (!need_mask || j0 + c0 + e < vis) tmax = fmaxf(tmax, s2);
+                }
+            }
+            const float mnew = fmaxf(mrun, tmax);
+            corr = exp2f(mrun - mnew);
+            float lsum = 0.f;
+            // pass 2: P = exp2(s - m), bf16, into the A-operand layout [key group][row][8 keys]
+#pragma unroll 1
+            for (int c0 = 0; c0 < 128; c0 += 32) {
+                uint32_t v[32];
+                tmem_ld32(lane_addr + c0, v);
+                tmem_ld_wait();
+#pragma unroll
+                for (int e = 0; e < 32; e += 8) {
+                    uint32_t pk[4];
+#pragma unroll
+                    for (int x = 0; x < 8; x += 2) {
+                        const int ja = j0 + c0 + e + x;
+                        float pa = exp2f(__uint_as_float(v[e + x]) * sc2 - mnew);
+                        float pb = exp2f(__uint_as_float(v[e + x + 1]) * sc2 - mnew);
+                        if (need_mask && ja >= vis) pa = 0.f;
+                        if (need_mask && ja + 1 >= vis) pb = 0.f;
+                        const __nv_bfloat162 pr = __floats2bfloat162_rn(pa, pb);
+                        pk[x >> 1] = *reinterpret_cast<const uint32_t*>(&pr);
+                        lsum += __low2float(pr) + __high2float(pr);
+                    }
+                    *reinterpret_cast<uint4*>(p_ptr + ((c0 + e) >> 3) * 2048 + tid * 16) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
+                }
+            }
+            lrun = lrun * corr + lsum;
+            mrun = mnew;
+            fence_proxy_async();
+        }
+        tc_fence_before();
+        __syncthreads();
+        if (tid == 128) {
+            tc_fence_after();
+#pragma unroll
+            for (int kk = 0; kk < 8; ++kk) {
+                const uint64_t ad = smem_desc(ps + kk * 2 * 2048, 2048, 128);
+                const uint64_t bd = smem_desc(vs + buf * kTileBytes + kk * 16 * 16, 128, kLboT);
+                umma_ss(tmem + 128, ad, bd, idesc_o, kk != 0);
+            }
+            umma_commit(bar_o);
+        }
+        if (warp < 4) {
+            mbar_wait(bar_o, jt & 1, P.status, failed, 6);
+            tc_fence_after();
+#pragma unroll
+            for (int c0 = 0; c0 < 128; c0 += 32) {
+                uint32_t v[32];
+                tmem_ld32(lane_addr + 128 + c0, v);
+                tmem_ld_wait();
+#pragma unroll
+                for (int e = 0; e < 32; ++e) acc[c0 + e] = fmaf(acc[c0 + e], corr, __uint_as_float(v[e]));
+            }
+        } else {
+            // the control warp also holds back until the tile's MMAs are done: the next
+            // iteration overwrites the other key/value buffer only, but P and S are reused
+            mbar_wait(bar_o, jt & 1, P.status, failed, 7);
+        }
+    }
+    if (live) {
+        const float inv = 1.f / lrun;
+        __nv_bfloat16* orow = unit_base_mut<__nv_bfloat16>(p.o, n, h) + (int64_t)row * p.o.st;
+#pragma unroll
+        for (int e = 0; e < 128; e += 8) {
+            uint4 o;
+            o.x = pack_bf16(acc[e] * inv, acc[e + 1] * inv);
+            o.y = pack_bf16(acc[e + 2] * inv, acc[e + 3] * inv);
+            o.z = pack_bf16(acc[e + 4] * inv, acc[e + 5] * inv);
+            o.w = pack_bf16(acc[e + 6] * inv, acc[e + 7] * inv);
+            *reinterpret_cast<uint4*>(orow + e) = o;
+        }
+        if (p.lse) p.lse[(int64_t)u * p.lse_stride + row] = (mrun + log2f(lrun)) * 0.6931471805599453f;
+    }
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 4) {
+        __syncwarp();
+        tmem_dealloc(tmem, kAttnTmemCols);
+    }
+}
+
 struct Plan {
     int n_tile, tiles, parts, tiles_per_part, stages, rows_pad;
     size_t smem;
@@ -391,7 +606,26 @@ int tensor_compress(lococo_handle* h, const CompressParams& p, cudaStream_t st) 
     return launches;
 }
 
-bool tensor_attention_supported(const lococo_handle*, const AttnParams&) { return false; }
-int tensor_attention(lococo_handle*, const AttnParams&, cudaStream_t) { return -1; }
+bool tensor_attention_supported(const lococo_handle* h, const AttnParams& p) {
+    return h->use_tensor && p.d == kD && h->ws != nullptr;
+}
+
+int tensor_attention(lococo_handle* h, const AttnParams& p, cudaStream_t st) {
+    static bool attr_set = false;
+    if (!attr_set) {
+        if (cudaFuncSetAttribute(attention_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kAttnSmem) != cudaSuccess)
+            return -1;
+        attr_set = true;
+    }
+    TcAttnParams P{};
+    P.base = p;
+    P.status = reinterpret_cast<int*>(h->ws + h->off_status);
+    dim3 grid((p.b + 127) / 128, p.units);
+    prof_begin(p.prof, 1, st);
+    attention_tc_kernel<<<grid, kAttnThreads, kAttnSmem, st>>>(P);
+    const bool ok = cudaGetLastError() == cudaSuccess;
+    prof_end(p.prof, st);
+    return ok ? 1 : -1;
+}
 
 }  // namespace lococo
