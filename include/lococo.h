@@ -115,6 +115,42 @@ lococo_status lococo_compress_step(lococo_handle* handle, lococo_tensor K_cache,
                                    int32_t* new_cache_len, float* W_out, void* stream);
 
 /*
+ * The compress branch of lococo_compress_step for callers that cannot allocate device
+ * memory at all.  (The paper has no counterpart of this entry point; it computes exactly
+ * Steps 4 and 5 of Algorithm 2 as described above.)
+ *
+ * Who needs it: code that runs where cudaMalloc is off limits - a plugin inside a host
+ * application that owns every byte of device memory and hands out none, a process whose
+ * memory pool was sized up front and is full, or a latency-critical loop in which an
+ * allocation (a synchronising driver call) is not acceptable.  Such a caller cannot provide
+ * the workspace lococo_set_workspace asks for.  Here the scratch (packed weights, mixing
+ * logits, row sums, partial blends) sits in a fixed 8 MiB array compiled into the library,
+ * which every GPU that loads the library keeps resident until the process exits.  No
+ * handle is needed and nothing is allocated or freed, on the host or on the device.
+ *
+ * cfg describes the problem as for lococo_create (max_chunk, path and softmax_scale are
+ * ignored); G [heads|1, M, c_in, k] and bias (or NULL) are device pointers in cfg->dtype and
+ * are re-packed on every call.  The tensors are those of lococo_compress_step; the outputs may
+ * alias the cache inputs.  Only a real compress step is accepted (cache_len + b > M): the fill
+ * branch needs no scratch, use lococo_compress_step for it.
+ * Errors: LOCOCO_ERR_WORKSPACE when the scratch this problem needs, about
+ *   4*batch*heads*M*(cache_len+b) + 8*batch*heads*M*d + sizeof(G) bytes,
+ * exceeds the built-in limit (lococo_static_scratch_limit); LOCOCO_ERR_INVALID_ARG /
+ * LOCOCO_ERR_UNSUPPORTED_SHAPE as for the other calls, before anything is launched.
+ * The first call on each device looks up the device address of the array (a runtime
+ * query); make that call outside any stream capture.  All calls on a device share the one
+ * array: every byte a call reads it has written first, so nothing needs clearing between
+ * calls, but two calls whose kernels overlap on the GPU (different streams, no dependency)
+ * race on it - order them.
+ */
+lococo_status lococo_compress_step_static(const lococo_config* cfg, const void* G_device, const void* bias_device,
+                                          lococo_tensor K_cache, lococo_tensor V_cache, int32_t cache_len,
+                                          lococo_tensor K_chunk, lococo_tensor V_chunk, int32_t b,
+                                          lococo_tensor K_cache_out, lococo_tensor V_cache_out, void* stream);
+/* Size in bytes of the built-in scratch array used by lococo_compress_step_static. */
+lococo_status lococo_static_scratch_limit(size_t* out);
+
+/*
  * Algorithm 2, Step 3 (Eq. 1): the b chunk queries attend over the c cache entries
  * (all visible) followed by the chunk (query r sees chunk keys 0..r), softmax over
  * keys with scale softmax_scale.  lse (device, optional, fp32 [batch, heads, b])

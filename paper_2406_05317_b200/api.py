@@ -53,6 +53,8 @@ _SIGNATURES = {
                                          ctypes.c_size_t, _P],
     "lococo_get_last_device_status": [_P, ctypes.POINTER(_I), _P],
     "lococo_launch_count": [_P, ctypes.POINTER(ctypes.c_int64)],
+    "lococo_compress_step_static": [ctypes.POINTER(Config), _P, _P, _T, _T, _I, _T, _T, _I, _T, _T, _P],
+    "lococo_static_scratch_limit": [ctypes.POINTER(ctypes.c_size_t)],
     "lococo_profile_enable": [_P, _I],
     "lococo_profile_read": [_P, _I, ctypes.POINTER(ctypes.c_double), ctypes.POINTER(ctypes.c_int64)],
 }
@@ -99,6 +101,22 @@ def _stream() -> int:
 
 def _ptr(t: torch.Tensor | None):
     return None if t is None else t.data_ptr()
+
+
+def static_scratch_limit() -> int:
+    n = ctypes.c_size_t()
+    _check(_lib.lococo_static_scratch_limit(ctypes.byref(n)), "lococo_static_scratch_limit")
+    return n.value
+
+
+def compress_step_static(cfg: Config, G, bias, K_cache, V_cache, cache_len, K_chunk, V_chunk, K_out, V_out):
+    """Compress step (Algorithm 2 Steps 4-5) that allocates nothing: for callers that may not
+    call cudaMalloc, the scratch is a fixed array inside the library. Raises LococoError with
+    ERR_WORKSPACE when the problem does not fit that array."""
+    _check(_lib.lococo_compress_step_static(ctypes.byref(cfg), G.data_ptr(), _ptr(bias), _view(K_cache),
+                                            _view(V_cache), cache_len, _view(K_chunk), _view(V_chunk),
+                                            K_chunk.shape[2], _view(K_out), _view(V_out), _stream()),
+           "lococo_compress_step_static")
 
 
 class Lococo:
