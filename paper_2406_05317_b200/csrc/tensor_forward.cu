@@ -26,7 +26,7 @@ using namespace tc;
 constexpr int kSlots = 128;              // slots per CTA (MMA M)
 constexpr int kD = 128;                  // head dimension
 constexpr int kStageBytes = 32768;       // one tap x 128 channels x 128 slots, bf16
-constexpr int kThreads = 160;            // 4 loader/epilogue warps + 1 control warp
+constexpr int kThreads = 192;            // 4 loader/epilogue warps + MMA-issue warp + weight-producer warp
 constexpr int kMaxSmem = 232448;         // 227 KB
 constexpr uint32_t kTmemCols = 512;
 constexpr uint32_t kColUK = 256, kColUV = 384;
@@ -34,7 +34,7 @@ constexpr uint32_t kColUK = 256, kColUV = 384;
 struct TcCompressParams {
     CompressParams base;
     const __nv_bfloat16* gimage;  // [sets][slot blocks][k][halves][16][128][8]
-    float* part_U;                // [units][slot blocks][parts][2][128][128]
+    float* part_U;                // [units][slot blocks][parts][2][128 channels][128 slots]
     float* part_s;                // [units][slot blocks][parts][128]
     float* R_store;               // optional [units][M][S]
     int* status;
@@ -112,60 +112,80 @@ __global__ void __launch_bounds__(kThreads, 1) compress_tc_kernel(const __grid_c
     const __nv_bfloat16* safe = unit_base<__nv_bfloat16>(p.xk.chunk, n, h);
 
     float ssum = 0.f;
-    uint32_t g = 0;  // ring iterations issued so far (control thread)
+    uint32_t g = 0;  // ring stages used so far, over all tiles of this CTA
     const int tile_begin = part * P.tiles_per_part;
     const int tile_end = min(P.tiles, tile_begin + P.tiles_per_part);
     int tile_it = 0;
     for (int tile = tile_begin; tile < tile_end; ++tile, ++tile_it) {
         const int j0 = tile * n_tile;
-        // ---- 1. stage the key and value rows j0-pad .. j0+n_tile+pad-1 (zeros outside [0,S))
-        for (int x = tid; x < rows * 16; x += kThreads) {
-            const int r = x >> 4, q = x & 15;
-            const int j = j0 - pad + r;
-            const bool valid = j >= 0 && j < p.S;
-            const __nv_bfloat16* sk = valid ? cat_row<__nv_bfloat16>(p.xk, n, h, j) + q * 8 : safe;
-            const __nv_bfloat16* sv = valid ? cat_row<__nv_bfloat16>(p.xv, n, h, j) + q * 8 : safe;
-            const uint32_t off = q * lbo_z + r * 16;
-            cp_async16(zk + off, sk, valid ? 16u : 0u);
-            cp_async16(zv + off, sv, valid ? 16u : 0u);
+        // The weight producer (one thread of warp 5) runs ahead of everything else: a tile's
+        // first ring stages need no wait, the ring being drained at every tile boundary.
+        const int total = p.k * P.halves;
+        auto load_stage = [&](uint32_t gg, int it) {
+            const uint32_t s = gg % NS;
+            if (gg >= (uint32_t)NS) mbar_wait(bar_empty + 8 * s, ((gg / NS) - 1) & 1, P.status, failed, 1);
+            mbar_expect_tx(bar_full + 8 * s, kStageBytes);
+            bulk_load(ring + s * kStageBytes, gimg + (int64_t)it * (kStageBytes / 2), kStageBytes, bar_full + 8 * s);
+        };
+        const int npro = min(NS, total);
+        if (tid == 160) {
+            for (int i = 0; i < npro; ++i) load_stage(g + i, i);
         }
+        // ---- 1. stage the key and value rows j0-pad .. j0+n_tile+pad-1 (zeros outside [0,S))
+        // each thread owns one 8-channel group (q) and every (threads/16)-th row
+        auto stage_tile = [&](const CatView& xv_, uint32_t dst, int first, int step) {
+            const int q = first & 15;
+            const __nv_bfloat16* cbase = unit_base<__nv_bfloat16>(xv_.cache, n, h) + q * 8;
+            const __nv_bfloat16* kbase = unit_base<__nv_bfloat16>(xv_.chunk, n, h) + q * 8;
+            const uint32_t d0 = dst + q * lbo_z;
+            for (int r = first >> 4; r < rows; r += step) {
+                const int j = j0 - pad + r;
+                const bool valid = j >= 0 && j < p.S;
+                const __nv_bfloat16* src = !valid ? safe : (j < xv_.c ? cbase + (int64_t)j * xv_.cache.st
+                                                                       : kbase + (int64_t)(j - xv_.c) * xv_.chunk.st);
+                cp_async16(d0 + r * 16, src, valid ? 16u : 0u);
+            }
+        };
+        stage_tile(p.xk, zk, tid, kThreads / 16);
+        // the value tile is a conv input only when c_in = 2d; otherwise it is needed by the
+        // blend only and is staged by the epilogue warps while the conv runs
+        if (P.halves == 2) stage_tile(p.xv, zv, tid, kThreads / 16);
         cp_async_wait_all();
         fence_proxy_async();
         __syncthreads();
 
-        // ---- 2. Eq. 6 as an implicit GEMM: one ring stage per (tap, 128-channel half)
-        if (tid == 128) {
-            const int total = p.k * P.halves;
-            auto load = [&](uint32_t gg, int it) {
-                const uint32_t s = gg % NS;
-                if (gg >= (uint32_t)NS) mbar_wait(bar_empty + 8 * s, ((gg / NS) - 1) & 1, P.status, failed, 1);
-                mbar_expect_tx(bar_full + 8 * s, kStageBytes);
-                bulk_load(ring + s * kStageBytes, gimg + (int64_t)it * (kStageBytes / 2), kStageBytes, bar_full + 8 * s);
-            };
-            const int npro = min(NS, total);
-            for (int i = 0; i < npro; ++i) load(g + i, i);
+        // ---- 2. Eq. 6 as an implicit GEMM: one ring stage per (tap, 128-channel half).
+        // Producer and MMA issuer are different threads, so the tensor pipe always has
+        // several stages of MMAs queued while the next weight copies are in flight.
+        if (tid == 160) {
+            for (int it = npro; it < total; ++it) load_stage(g + it, it);
+        } else if (tid == 128) {
+            const uint64_t a0 = smem_desc(ring, 2048, 128);
+            const uint64_t bk0 = smem_desc(zk, lbo_z, 128), bv0 = smem_desc(zv, lbo_z, 128);
+            const uint32_t bstep = (2 * lbo_z) >> 4;
+            // stage index and phase, tap and channel half are tracked incrementally: no division here
+            uint32_t st = g % NS, ph = (g / NS) & 1, tap = 0, half = 0;
             for (int it = 0; it < total; ++it) {
-                const uint32_t gg = g + it, s = gg % NS;
-                mbar_wait(bar_full + 8 * s, (gg / NS) & 1, P.status, failed, 2);
+                mbar_wait(bar_full + 8 * st, ph, P.status, failed, 2);
                 tc_fence_after();
-                const int t = it / P.halves, half = it % P.halves;
-                const uint32_t zbase = (half == 0 ? zk : zv) + t * 16;
-                const uint32_t abase = ring + s * kStageBytes;
+                const uint64_t ad = a0 + st * (uint32_t)(kStageBytes >> 4);
+                const uint64_t bd = (half == 0 ? bk0 : bv0) + tap;   // tap t = row offset t (16 bytes per row)
 #pragma unroll
-                for (int kk = 0; kk < 8; ++kk) {
-                    const uint64_t ad = smem_desc(abase + kk * 2 * 2048, 2048, 128);
-                    const uint64_t bd = smem_desc(zbase + kk * 2 * lbo_z, lbo_z, 128);
-                    umma_ss(tmem, ad, bd, idesc_conv, (it | kk) != 0);
-                }
-                umma_commit(bar_empty + 8 * s);
-                if (it >= 1 && it - 1 + NS < total) load(gg - 1 + NS, it - 1 + NS);
+                for (int kk = 0; kk < 8; ++kk) umma_ss(tmem, ad + kk * 256u, bd + kk * bstep, idesc_conv, (it | kk) != 0);
+                umma_commit(bar_empty + 8 * st);
+                if (++half == (uint32_t)P.halves) { half = 0; ++tap; }
+                if (++st == (uint32_t)NS) { st = 0; ph ^= 1; }
             }
             umma_commit(bar_acc);
-            g += total;
         }
+        g += total;
 
         // ---- 3. accumulator -> bias, ReLU, row sum (Eq. 7), bf16 -> A operand of the blends
         if (warp < 4) {
+            if (P.halves == 1) {
+                stage_tile(p.xv, zv, tid, kSlots / 16);
+                cp_async_wait_all();
+            }
             mbar_wait(bar_acc, tile_it & 1, P.status, failed, 3);
             tc_fence_after();
             const uint32_t lane_addr = tmem + ((uint32_t)(warp * 32) << 16);
@@ -224,8 +244,9 @@ __global__ void __launch_bounds__(kThreads, 1) compress_tc_kernel(const __grid_c
         tc_fence_after();
         const uint32_t lane_addr = tmem + ((uint32_t)(warp * 32) << 16);
         const int64_t pidx = ((int64_t)u * P.slot_blocks + sb) * P.parts + part;
-        float* outK = P.part_U + (pidx * 2 + 0) * (kSlots * kD) + tid * kD;
-        float* outV = P.part_U + (pidx * 2 + 1) * (kSlots * kD) + tid * kD;
+        // stored channel-major ([channel][slot]) so that a warp's 32 lanes write 128 contiguous bytes
+        float* outK = P.part_U + (pidx * 2 + 0) * (kSlots * kD) + tid;
+        float* outV = P.part_U + (pidx * 2 + 1) * (kSlots * kD) + tid;
 #pragma unroll 1
         for (int c0 = 0; c0 < kD; c0 += 32) {
             uint32_t a[32], b[32];
@@ -233,9 +254,9 @@ __global__ void __launch_bounds__(kThreads, 1) compress_tc_kernel(const __grid_c
             tmem_ld32(lane_addr + kColUV + c0, b);
             tmem_ld_wait();
 #pragma unroll
-            for (int e = 0; e < 32; e += 4) {
-                *reinterpret_cast<uint4*>(outK + c0 + e) = make_uint4(a[e], a[e + 1], a[e + 2], a[e + 3]);
-                *reinterpret_cast<uint4*>(outV + c0 + e) = make_uint4(b[e], b[e + 1], b[e + 2], b[e + 3]);
+            for (int e = 0; e < 32; ++e) {
+                outK[(c0 + e) * kSlots] = __uint_as_float(a[e]);
+                outV[(c0 + e) * kSlots] = __uint_as_float(b[e]);
             }
         }
         P.part_s[pidx * kSlots + tid] = ssum;
@@ -259,8 +280,8 @@ __global__ void finalize_parts_kernel(TcCompressParams P) {
     float s = 0.f, uk = 0.f, uv = 0.f;
     for (int pt = 0; pt < P.parts; ++pt) {
         s += P.part_s[(base + pt) * kSlots + il];
-        uk += P.part_U[((base + pt) * 2 + 0) * (kSlots * kD) + il * kD + ch];
-        uv += P.part_U[((base + pt) * 2 + 1) * (kSlots * kD) + il * kD + ch];
+        uk += P.part_U[((base + pt) * 2 + 0) * (kSlots * kD) + ch * kSlots + il];
+        uv += P.part_U[((base + pt) * 2 + 1) * (kSlots * kD) + ch * kSlots + il];
     }
     s += p.eps;
     const float inv = 1.f / s;
@@ -503,7 +524,7 @@ size_t smem_bytes(int n_tile, int k, int stages) {
 bool make_plan(int S, int k, int units, int slot_blocks, Plan* out) {
     double best = 1e30;
     const int cap = parts_cap(units, slot_blocks);
-    for (int n_tile = 160; n_tile >= 64; n_tile -= 32) {
+    for (int n_tile = 224; n_tile >= 64; n_tile -= 32) {
         int stages = 4;
         while (stages >= 2 && smem_bytes(n_tile, k, stages) > (size_t)kMaxSmem) --stages;
         if (stages < 2 || (size_t)stages * kStageBytes < (size_t)n_tile * kSlots * 2) continue;
