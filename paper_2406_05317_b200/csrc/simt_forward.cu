@@ -391,6 +391,19 @@ static int compress_typed(const CompressParams& p, cudaStream_t st) {
     return launches;
 }
 
+// Eq. 6 + ReLU and the denominators of Eq. 7 only (the backward pass recomputes them).
+int simt_conv_rowsum(int dtype, const CompressParams& p, cudaStream_t st) {
+    if (p.k > kMaxTaps) return -1;
+    dim3 grid((p.S + CT - 1) / CT, (p.M + CT - 1) / CT, p.units);
+    const size_t smem = sizeof(float) * ((size_t)(CT + p.k - 1) * (CCH + 1) + (size_t)CT * (CCH + 1));
+    const int rc = dtype == LOCOCO_F32 ? checked([&] { conv_relu_kernel<float><<<grid, 256, smem, st>>>(p); })
+                                       : checked([&] { conv_relu_kernel<__nv_bfloat16><<<grid, 256, smem, st>>>(p); });
+    if (rc < 0) return -1;
+    const int rows = p.units * p.M;
+    if (checked([&] { rowsum_kernel<<<(rows + 7) / 8, 256, 0, st>>>(p.R, p.s, rows, p.S, p.eps); }) < 0) return -1;
+    return 2;
+}
+
 int simt_write_weights(const float* R, const float* s, float* W, int64_t rows, int S, cudaStream_t st) {
     const int64_t total = rows * S;
     const int blocks = (int)((total + 255) / 256 < 8192 ? (total + 255) / 256 : 8192);
