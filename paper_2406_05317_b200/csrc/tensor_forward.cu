@@ -270,25 +270,41 @@ __global__ void __launch_bounds__(kThreads, 1) compress_tc_kernel(const __grid_c
 }
 
 // cache = (sum of partial blends) / (sum of partial row sums + eps)   (Eq. 7 after Eq. 4-5)
-__global__ void finalize_parts_kernel(TcCompressParams P) {
+// One block per 32 slots x 32 channels: the partials are channel-major (read along slots),
+// the cache is slot-major (written along channels); the tile is transposed in shared memory.
+__global__ void __launch_bounds__(256) finalize_parts_kernel(TcCompressParams P) {
     const CompressParams& p = P.base;
-    const int u = blockIdx.y, n = u / p.heads, h = u % p.heads;
-    const int x = blockIdx.x * blockDim.x + threadIdx.x;
-    if (x >= p.M * kD) return;
-    const int i = x / kD, ch = x % kD, sb = i / kSlots, il = i % kSlots;
+    __shared__ float tk[32][33], tv[32][33], inv_s[32];
+    const int u = blockIdx.z, n = u / p.heads, h = u % p.heads;
+    const int i0 = blockIdx.x * 32, c0 = blockIdx.y * 32;   // slot tile, channel tile
+    const int sb = i0 / kSlots, il0 = i0 % kSlots;
     const int64_t base = ((int64_t)u * P.slot_blocks + sb) * P.parts;
-    float s = 0.f, uk = 0.f, uv = 0.f;
-    for (int pt = 0; pt < P.parts; ++pt) {
-        s += P.part_s[(base + pt) * kSlots + il];
-        uk += P.part_U[((base + pt) * 2 + 0) * (kSlots * kD) + ch * kSlots + il];
-        uv += P.part_U[((base + pt) * 2 + 1) * (kSlots * kD) + ch * kSlots + il];
+    const int tx = threadIdx.x % 32, ty = threadIdx.x / 32;
+    if (ty == 0) {
+        float s = 0.f;
+        for (int pt = 0; pt < P.parts; ++pt) s += P.part_s[(base + pt) * kSlots + il0 + tx];
+        s += p.eps;
+        inv_s[tx] = 1.f / s;
+        if (c0 == 0) p.s[(int64_t)u * p.M + i0 + tx] = s;
     }
-    s += p.eps;
-    const float inv = 1.f / s;
-    unit_base_mut<__nv_bfloat16>(p.k_out, n, h)[(int64_t)i * p.k_out.st + ch] = __float2bfloat16_rn(uk * inv);
-    unit_base_mut<__nv_bfloat16>(p.v_out, n, h)[(int64_t)i * p.v_out.st + ch] = __float2bfloat16_rn(uv * inv);
-    if (ch == 0) p.s[(int64_t)u * p.M + i] = s;
+    for (int cc = ty; cc < 32; cc += 8) {      // tx runs along slots: 128-byte coalesced reads
+        float uk = 0.f, uv = 0.f;
+        for (int pt = 0; pt < P.parts; ++pt) {
+            uk += P.part_U[((base + pt) * 2 + 0) * (kSlots * kD) + (c0 + cc) * kSlots + il0 + tx];
+            uv += P.part_U[((base + pt) * 2 + 1) * (kSlots * kD) + (c0 + cc) * kSlots + il0 + tx];
+        }
+        tk[cc][tx] = uk;
+        tv[cc][tx] = uv;
+    }
+    __syncthreads();
+    for (int ii = ty; ii < 32; ii += 8) {      // tx runs along channels: coalesced writes
+        const float inv = inv_s[ii];
+        const int64_t row = (int64_t)(i0 + ii);
+        unit_base_mut<__nv_bfloat16>(p.k_out, n, h)[row * p.k_out.st + c0 + tx] = __float2bfloat16_rn(tk[tx][ii] * inv);
+        unit_base_mut<__nv_bfloat16>(p.v_out, n, h)[row * p.v_out.st + c0 + tx] = __float2bfloat16_rn(tv[tx][ii] * inv);
+    }
 }
+
 
 
 // ------------------------------------------------------------------ Eq. 1, chunk form
@@ -615,7 +631,7 @@ int tensor_compress(lococo_handle* h, const CompressParams& p, cudaStream_t st) 
     prof_end(p.prof, st);
     if (!ok) return -1;
     ++launches;
-    dim3 fgrid((p.M * kD + 255) / 256, p.units);
+    dim3 fgrid(p.M / 32, kD / 32, p.units);
     finalize_parts_kernel<<<fgrid, 256, 0, st>>>(P);
     if (cudaGetLastError() != cudaSuccess) return -1;
     ++launches;
