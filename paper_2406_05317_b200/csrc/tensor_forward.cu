@@ -310,15 +310,16 @@ __global__ void __launch_bounds__(256) finalize_parts_kernel(TcCompressParams P)
 // ------------------------------------------------------------------ Eq. 1, chunk form
 // One CTA = 128 queries of one unit. Per 128-key tile of [cache; chunk]:
 //   S = Q K^T on the tensor cores (both operands K-major, staged un-swizzled),
-//   one thread per query row reads its S row from TMEM, applies the scale, the causal
-//   mask and the running-max update, and writes P (bf16) to shared memory,
+//   two threads per query row (each owns 64 of the 128 columns) read S from TMEM, apply
+//   the scale, the causal mask and the running-max update, and write P (bf16) to shared
+//   memory as an MMA A operand,
 //   O_tile = P V on the tensor cores (V read MN-major from its staged tile),
-//   and the row's fp32 accumulator is rescaled and updated in registers.
-constexpr int kAttnThreads = 160;
+//   and each thread rescales and updates its 64 fp32 output columns in registers.
+constexpr int kAttnThreads = 288;                  // 8 softmax warps + 1 control warp
 constexpr uint32_t kLboT = 129 * 16;               // byte stride between 8-channel groups of a staged 128-row tile
 constexpr uint32_t kTileBytes = 16 * kLboT;        // 33024
 constexpr uint32_t kPBytes = 16 * 2048;            // P tile: [16 key groups][128 rows][8 keys]
-constexpr uint32_t kAttnSmem = 5 * kTileBytes + kPBytes + 64;
+constexpr uint32_t kAttnSmem = 5 * kTileBytes + kPBytes + 2 * 128 * 4 + 64;
 constexpr uint32_t kAttnTmemCols = 256;
 
 struct TcAttnParams {
@@ -330,7 +331,7 @@ __global__ void __launch_bounds__(kAttnThreads, 1) attention_tc_kernel(const __g
     extern __shared__ __align__(128) uint8_t smem[];
     const AttnParams& p = P.base;
     const int u = blockIdx.y, n = u / p.heads, h = u % p.heads;
-    const int tid = threadIdx.x, warp = tid >> 5;
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int r0 = blockIdx.x * 128;
     const int S = p.c + p.b;
 
@@ -338,19 +339,21 @@ __global__ void __launch_bounds__(kAttnThreads, 1) attention_tc_kernel(const __g
     uint8_t* k_ptr = q_ptr + kTileBytes;       // two buffers
     uint8_t* v_ptr = k_ptr + 2 * kTileBytes;   // two buffers
     uint8_t* p_ptr = v_ptr + 2 * kTileBytes;
-    uint64_t* bars = reinterpret_cast<uint64_t*>(p_ptr + kPBytes);
+    float* xchg = reinterpret_cast<float*>(p_ptr + kPBytes);   // [2 halves][128 rows]
+    uint64_t* bars = reinterpret_cast<uint64_t*>(xchg + 256);
     volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(bars + 2);
     volatile int* failed = reinterpret_cast<volatile int*>(tmem_slot + 1);
     const uint32_t qs = smem_u32(q_ptr), ks = smem_u32(k_ptr), vs = smem_u32(v_ptr), ps = smem_u32(p_ptr);
     const uint32_t bar_s = smem_u32(bars), bar_o = bar_s + 8;
+    constexpr int kCtl = 256;                  // control thread (lane 0 of warp 8)
 
-    if (tid == 128) {
+    if (tid == kCtl) {
         mbar_init(bar_s, 1);
         mbar_init(bar_o, 1);
         *failed = 0;
         fence_barrier_init();
     }
-    if (warp == 4) {
+    if (warp == 8) {
         __syncwarp();
         tmem_alloc(smem_u32(const_cast<uint32_t*>(tmem_slot)), kAttnTmemCols);
         tmem_relinquish();
@@ -365,40 +368,48 @@ __global__ void __launch_bounds__(kAttnThreads, 1) attention_tc_kernel(const __g
     const int ntiles = (ncols + 127) / 128;
     const __nv_bfloat16* safe = unit_base<__nv_bfloat16>(p.q, n, h);
 
+    // each thread owns one 8-channel group and every 18th row of a tile
+    const int lq = tid & 15, lr0 = tid >> 4;
+    const __nv_bfloat16* kc_base = unit_base<__nv_bfloat16>(p.xk.cache, n, h) + lq * 8;
+    const __nv_bfloat16* kn_base = unit_base<__nv_bfloat16>(p.xk.chunk, n, h) + lq * 8;
+    const __nv_bfloat16* vc_base = unit_base<__nv_bfloat16>(p.xv.cache, n, h) + lq * 8;
+    const __nv_bfloat16* vn_base = unit_base<__nv_bfloat16>(p.xv.chunk, n, h) + lq * 8;
     auto load_kv = [&](int jt, int buf) {
-        const int j0 = jt * 128;
-        for (int x = tid; x < 128 * 16; x += kAttnThreads) {
-            const int r = x >> 4, q = x & 15;
-            const int j = j0 + r;
+        const uint32_t d0 = buf * kTileBytes + lq * kLboT;
+        for (int r = lr0; r < 128; r += kAttnThreads / 16) {
+            const int j = jt * 128 + r;
             const bool valid = j < S;
-            const __nv_bfloat16* sk = valid ? cat_row<__nv_bfloat16>(p.xk, n, h, j) + q * 8 : safe;
-            const __nv_bfloat16* sv = valid ? cat_row<__nv_bfloat16>(p.xv, n, h, j) + q * 8 : safe;
-            const uint32_t off = buf * kTileBytes + q * kLboT + r * 16;
-            cp_async16(ks + off, sk, valid ? 16u : 0u);
-            cp_async16(vs + off, sv, valid ? 16u : 0u);
+            const bool in_cache = j < p.c;
+            const __nv_bfloat16* sk = !valid ? safe : in_cache ? kc_base + (int64_t)j * p.xk.cache.st
+                                                               : kn_base + (int64_t)(j - p.c) * p.xk.chunk.st;
+            const __nv_bfloat16* sv = !valid ? safe : in_cache ? vc_base + (int64_t)j * p.xv.cache.st
+                                                               : vn_base + (int64_t)(j - p.c) * p.xv.chunk.st;
+            cp_async16(ks + d0 + r * 16, sk, valid ? 16u : 0u);
+            cp_async16(vs + d0 + r * 16, sv, valid ? 16u : 0u);
         }
     };
     // queries of this tile (zeros beyond the chunk) and the first key/value tile
-    for (int x = tid; x < 128 * 16; x += kAttnThreads) {
-        const int r = x >> 4, q = x & 15;
+    for (int r = lr0; r < 128; r += kAttnThreads / 16) {
         const bool valid = r0 + r < p.b;
-        const __nv_bfloat16* sq = valid ? unit_base<__nv_bfloat16>(p.q, n, h) + (int64_t)(r0 + r) * p.q.st + q * 8 : safe;
-        cp_async16(qs + q * kLboT + r * 16, sq, valid ? 16u : 0u);
+        const __nv_bfloat16* sq = valid ? unit_base<__nv_bfloat16>(p.q, n, h) + (int64_t)(r0 + r) * p.q.st + lq * 8 : safe;
+        cp_async16(qs + lq * kLboT + r * 16, sq, valid ? 16u : 0u);
     }
     load_kv(0, 0);
     asm volatile("cp.async.commit_group;" ::: "memory");
 
     const uint32_t idesc_s = instr_desc_bf16(128, false, false);
     const uint32_t idesc_o = instr_desc_bf16(128, false, true);
-    const int row = r0 + tid;                       // compute threads only
-    const bool live = tid < 128 && row < p.b;
+    const int rl = (warp & 3) * 32 + lane;          // row of the tile this thread works on (softmax warps)
+    const int half = (warp >> 2) & 1;               // which 64 columns of the row
+    const int row = r0 + rl;
+    const bool live = warp < 8 && row < p.b;
     const int vis = live ? p.c + row + 1 : 1;       // visible columns of this row
     const float sc2 = p.scale * 1.4426950408889634f;
-    float acc[128];
+    float acc[64];
 #pragma unroll
-    for (int e = 0; e < 128; ++e) acc[e] = 0.f;
+    for (int e = 0; e < 64; ++e) acc[e] = 0.f;
     float mrun = -INFINITY, lrun = 0.f;
-    const uint32_t lane_addr = tmem + ((uint32_t)((warp & 3) * 32) << 16);
+    const uint32_t lane_addr = tmem + ((uint32_t)((warp & 3) * 32) << 16) + half * 64;
 
     for (int jt = 0; jt < ntiles; ++jt) {
         const int buf = jt & 1;
@@ -411,26 +422,24 @@ __global__ void __launch_bounds__(kAttnThreads, 1) attention_tc_kernel(const __g
         }
         fence_proxy_async();
         __syncthreads();
-        if (tid == 128) {
+        if (tid == kCtl) {
             tc_fence_after();
+            const uint64_t a0 = smem_desc(qs, kLboT, 128), b0 = smem_desc(ks + buf * kTileBytes, kLboT, 128);
 #pragma unroll
-            for (int kk = 0; kk < 8; ++kk) {
-                const uint64_t ad = smem_desc(qs + kk * 2 * kLboT, kLboT, 128);
-                const uint64_t bd = smem_desc(ks + buf * kTileBytes + kk * 2 * kLboT, kLboT, 128);
-                umma_ss(tmem, ad, bd, idesc_s, kk != 0);
-            }
+            for (int kk = 0; kk < 8; ++kk) umma_ss(tmem, a0 + kk * ((2 * kLboT) >> 4), b0 + kk * ((2 * kLboT) >> 4), idesc_s, kk != 0);
             umma_commit(bar_s);
         }
         float corr = 1.f;
-        if (warp < 4) {
+        if (warp < 8) {
             mbar_wait(bar_s, jt & 1, P.status, failed, 5);
             tc_fence_after();
-            const int j0 = jt * 128;
-            const bool need_mask = j0 + 128 > p.c + r0;
-            // pass 1: row maximum of the scaled, masked logits
+            const int j0 = jt * 128 + half * 64;
+            const bool need_mask = jt * 128 + 128 > p.c + r0;
+            // pass 1: maximum of this thread's 64 scaled, masked logits; the row maximum is
+            // shared with the partner thread through shared memory
             float tmax = -INFINITY;
-#pragma unroll 1
-            for (int c0 = 0; c0 < 128; c0 += 32) {
+#pragma unroll
+            for (int c0 = 0; c0 < 64; c0 += 32) {
                 uint32_t v[32];
                 tmem_ld32(lane_addr + c0, v);
                 tmem_ld_wait();
@@ -440,12 +449,14 @@ __global__ void __launch_bounds__(kAttnThreads, 1) attention_tc_kernel(const __g
                     if (!need_mask || j0 + c0 + e < vis) tmax = fmaxf(tmax, s2);
                 }
             }
-            const float mnew = fmaxf(mrun, tmax);
+            xchg[half * 128 + rl] = tmax;
+            asm volatile("bar.sync 1, 256;" ::: "memory");
+            const float mnew = fmaxf(mrun, fmaxf(tmax, xchg[(half ^ 1) * 128 + rl]));
             corr = exp2f(mrun - mnew);
             float lsum = 0.f;
             // pass 2: P = exp2(s - m), bf16, into the A-operand layout [key group][row][8 keys]
-#pragma unroll 1
-            for (int c0 = 0; c0 < 128; c0 += 32) {
+#pragma unroll
+            for (int c0 = 0; c0 < 64; c0 += 32) {
                 uint32_t v[32];
                 tmem_ld32(lane_addr + c0, v);
                 tmem_ld_wait();
@@ -463,7 +474,7 @@ __global__ void __launch_bounds__(kAttnThreads, 1) attention_tc_kernel(const __g
                         pk[x >> 1] = *reinterpret_cast<const uint32_t*>(&pr);
                         lsum += __low2float(pr) + __high2float(pr);
                     }
-                    *reinterpret_cast<uint4*>(p_ptr + ((c0 + e) >> 3) * 2048 + tid * 16) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
+                    *reinterpret_cast<uint4*>(p_ptr + ((half * 64 + c0 + e) >> 3) * 2048 + rl * 16) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
                 }
             }
             lrun = lrun * corr + lsum;
@@ -472,38 +483,37 @@ __global__ void __launch_bounds__(kAttnThreads, 1) attention_tc_kernel(const __g
         }
         tc_fence_before();
         __syncthreads();
-        if (tid == 128) {
+        if (tid == kCtl) {
             tc_fence_after();
+            const uint64_t a0 = smem_desc(ps, 2048, 128), b0 = smem_desc(vs + buf * kTileBytes, 128, kLboT);
 #pragma unroll
-            for (int kk = 0; kk < 8; ++kk) {
-                const uint64_t ad = smem_desc(ps + kk * 2 * 2048, 2048, 128);
-                const uint64_t bd = smem_desc(vs + buf * kTileBytes + kk * 16 * 16, 128, kLboT);
-                umma_ss(tmem + 128, ad, bd, idesc_o, kk != 0);
-            }
+            for (int kk = 0; kk < 8; ++kk) umma_ss(tmem + 128, a0 + kk * 256u, b0 + kk * 16u, idesc_o, kk != 0);
             umma_commit(bar_o);
         }
-        if (warp < 4) {
-            mbar_wait(bar_o, jt & 1, P.status, failed, 6);
+        // everybody holds back until the tile's MMAs are done: P, S and the key/value buffer are reused
+        mbar_wait(bar_o, jt & 1, P.status, failed, 6);
+        if (warp < 8) {
             tc_fence_after();
 #pragma unroll
-            for (int c0 = 0; c0 < 128; c0 += 32) {
+            for (int c0 = 0; c0 < 64; c0 += 32) {
                 uint32_t v[32];
                 tmem_ld32(lane_addr + 128 + c0, v);
                 tmem_ld_wait();
 #pragma unroll
                 for (int e = 0; e < 32; ++e) acc[c0 + e] = fmaf(acc[c0 + e], corr, __uint_as_float(v[e]));
             }
-        } else {
-            // the control warp also holds back until the tile's MMAs are done: the next
-            // iteration overwrites the other key/value buffer only, but P and S are reused
-            mbar_wait(bar_o, jt & 1, P.status, failed, 7);
         }
     }
+    // row sum = sum of the two partners' partial sums
+    if (warp < 8) xchg[half * 128 + rl] = lrun;
+    tc_fence_before();
+    __syncthreads();
     if (live) {
-        const float inv = 1.f / lrun;
-        __nv_bfloat16* orow = unit_base_mut<__nv_bfloat16>(p.o, n, h) + (int64_t)row * p.o.st;
+        const float ltot = lrun + xchg[(half ^ 1) * 128 + rl];
+        const float inv = 1.f / ltot;
+        __nv_bfloat16* orow = unit_base_mut<__nv_bfloat16>(p.o, n, h) + (int64_t)row * p.o.st + half * 64;
 #pragma unroll
-        for (int e = 0; e < 128; e += 8) {
+        for (int e = 0; e < 64; e += 8) {
             uint4 o;
             o.x = pack_bf16(acc[e] * inv, acc[e + 1] * inv);
             o.y = pack_bf16(acc[e + 2] * inv, acc[e + 3] * inv);
@@ -511,11 +521,9 @@ __global__ void __launch_bounds__(kAttnThreads, 1) attention_tc_kernel(const __g
             o.w = pack_bf16(acc[e + 6] * inv, acc[e + 7] * inv);
             *reinterpret_cast<uint4*>(orow + e) = o;
         }
-        if (p.lse) p.lse[(int64_t)u * p.lse_stride + row] = (mrun + log2f(lrun)) * 0.6931471805599453f;
+        if (p.lse && half == 0) p.lse[(int64_t)u * p.lse_stride + row] = (mrun + log2f(ltot)) * 0.6931471805599453f;
     }
-    tc_fence_before();
-    __syncthreads();
-    if (warp == 4) {
+    if (warp == 8) {
         __syncwarp();
         tmem_dealloc(tmem, kAttnTmemCols);
     }
