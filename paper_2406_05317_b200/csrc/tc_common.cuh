@@ -66,9 +66,11 @@ __device__ __forceinline__ void bulk_load(uint32_t dst_smem, const void* src, ui
                  "l"(src), "r"(bytes), "r"(bar)
                  : "memory");
 }
-// 16-byte cp.async; src_bytes = 0 writes zeros.
+// 16-byte cp.async; src_bytes = 0 writes zeros. The .ca form goes through L1, which merges the
+// sixteen 16-byte pieces of a 256-byte row into full lines: measured 64-74 GB/s per SM for the
+// tile-staging pattern here, against 24 GB/s for .cg (each piece its own L2 request).
 __device__ __forceinline__ void cp_async16(uint32_t dst_smem, const void* src, uint32_t src_bytes) {
-    asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(dst_smem), "l"(src), "r"(src_bytes) : "memory");
+    asm volatile("cp.async.ca.shared.global [%0], [%1], 16, %2;" ::"r"(dst_smem), "l"(src), "r"(src_bytes) : "memory");
 }
 __device__ __forceinline__ void cp_async_wait_all() {
     asm volatile("cp.async.commit_group;\n\tcp.async.wait_group 0;" ::: "memory");
