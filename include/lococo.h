@@ -219,7 +219,9 @@ lococo_status lococo_launch_count(const lococo_handle* handle, int64_t* out);
 /*
  * Optional timing of single kernel classes with CUDA events recorded on the launching
  * stream around each launch.  kind 0: the kernel that evaluates Eq. 6 (the conv
- * contraction, with whatever is fused into it); kind 1: the chunk-attention kernel (Eq. 1).
+ * contraction, with whatever is fused into it); kind 1: the chunk-attention kernel (Eq. 1);
+ * kind 2: the single launch lococo_process_sequence uses per chunk on the tensor-core path, which
+ * holds both of the above (Step 3 and Steps 4-5 of Algorithm 2 are independent of each other).
  * lococo_profile_enable(h, 1) starts a fresh recording, (h, 0) stops it;
  * lococo_profile_read waits for the recorded events and returns the summed duration in
  * milliseconds and the number of launches of that kind since the recording started.

@@ -63,21 +63,9 @@ lococo_status count(lococo_handle* h, int launched) {
     return LOCOCO_OK;
 }
 
-lococo_status compress_impl(lococo_handle* h, View kc, View vc, int c, View kn, View vn, int b, View ko, View vo,
-                            float* W_out, cudaStream_t st) {
+CompressParams make_compress_params(lococo_handle* h, View kc, View vc, int c, View kn, View vn, int b, View ko, View vo,
+                                    float* W_out) {
     const lococo_config& cfg = h->cfg;
-    if (c + b <= cfg.M) {
-        // fill branch of Algorithm 2; carry the old rows over when the output is another buffer
-        if (ko.ptr != kc.ptr || vo.ptr != vc.ptr) {
-            if (c > 0) {
-                FillParams f{kc, vc, ko, vo, cfg.heads, h->units, cfg.head_dim, 0, c};
-                lococo_status s = count(h, simt_fill(cfg.dtype, f, st));
-                if (s) return s;
-            }
-        }
-        FillParams f{kn, vn, ko, vo, cfg.heads, h->units, cfg.head_dim, c, b};
-        return count(h, simt_fill(cfg.dtype, f, st));
-    }
     CompressParams p{};
     p.xk = CatView{kc, kn, c, b};
     p.xv = CatView{vc, vn, c, b};
@@ -95,12 +83,11 @@ lococo_status compress_impl(lococo_handle* h, View kc, View vc, int c, View kn, 
     p.UV = reinterpret_cast<float*>(h->ws + h->off_UV);
     p.W_out = W_out;
     p.prof = h->prof.on ? &h->prof : nullptr;
-    if (h->use_tensor && tensor_compress_supported(h, p)) return count(h, tensor_compress(h, p, st));
-    return count(h, simt_compress(cfg.dtype, p, st));
+    return p;
 }
 
-lococo_status attention_impl(lococo_handle* h, View q, View kc, View vc, int c, View kn, View vn, int b, View o,
-                             float* lse, int64_t lse_stride, cudaStream_t st) {
+AttnParams make_attn_params(lococo_handle* h, View q, View kc, View vc, int c, View kn, View vn, int b, View o, float* lse,
+                            int64_t lse_stride) {
     const lococo_config& cfg = h->cfg;
     AttnParams p{};
     p.q = q; p.o = o;
@@ -110,8 +97,48 @@ lococo_status attention_impl(lococo_handle* h, View q, View kc, View vc, int c, 
     p.scale = h->scale;
     p.lse = lse; p.lse_stride = lse_stride;
     p.prof = h->prof.on ? &h->prof : nullptr;
+    return p;
+}
+
+lococo_status compress_impl(lococo_handle* h, View kc, View vc, int c, View kn, View vn, int b, View ko, View vo,
+                            float* W_out, cudaStream_t st) {
+    const lococo_config& cfg = h->cfg;
+    if (c + b <= cfg.M) {
+        // fill branch of Algorithm 2; carry the old rows over when the output is another buffer
+        if (ko.ptr != kc.ptr || vo.ptr != vc.ptr) {
+            if (c > 0) {
+                FillParams f{kc, vc, ko, vo, cfg.heads, h->units, cfg.head_dim, 0, c};
+                lococo_status s = count(h, simt_fill(cfg.dtype, f, st));
+                if (s) return s;
+            }
+        }
+        FillParams f{kn, vn, ko, vo, cfg.heads, h->units, cfg.head_dim, c, b};
+        return count(h, simt_fill(cfg.dtype, f, st));
+    }
+    const CompressParams p = make_compress_params(h, kc, vc, c, kn, vn, b, ko, vo, W_out);
+    if (h->use_tensor && tensor_compress_supported(h, p)) return count(h, tensor_compress(h, p, st));
+    return count(h, simt_compress(cfg.dtype, p, st));
+}
+
+lococo_status attention_impl(lococo_handle* h, View q, View kc, View vc, int c, View kn, View vn, int b, View o,
+                             float* lse, int64_t lse_stride, cudaStream_t st) {
+    const AttnParams p = make_attn_params(h, q, kc, vc, c, kn, vn, b, o, lse, lse_stride);
     if (h->use_tensor && tensor_attention_supported(h, p)) return count(h, tensor_attention(h, p, st));
-    return count(h, simt_attention(cfg.dtype, p, st));
+    return count(h, simt_attention(h->cfg.dtype, p, st));
+}
+
+// One step of Algorithm 2's loop with an in-place cache: Step 3 with the old cache, then the
+// update. On the tensor-core path both run as one launch (they are independent of each other).
+lococo_status step_impl(lococo_handle* h, View q, View kc, View vc, int c, View kn, View vn, int b, View o, float* lse,
+                        int64_t lse_stride, cudaStream_t st) {
+    if (h->use_tensor && c + b > h->cfg.M) {
+        const AttnParams a = make_attn_params(h, q, kc, vc, c, kn, vn, b, o, lse, lse_stride);
+        const CompressParams p = make_compress_params(h, kc, vc, c, kn, vn, b, kc, vc, nullptr);
+        if (tensor_attention_supported(h, a) && tensor_compress_supported(h, p)) return count(h, tensor_chunk_step(h, a, p, st));
+    }
+    lococo_status s = attention_impl(h, q, kc, vc, c, kn, vn, b, o, lse, lse_stride, st);
+    if (s) return s;
+    return compress_impl(h, kc, vc, c, kn, vn, b, kc, vc, nullptr, st);
 }
 
 bool chunk_args_ok(const lococo_handle* h, int c, int b) {
@@ -340,9 +367,7 @@ lococo_status lococo_process_sequence(lococo_handle* h, lococo_tensor Q, lococo_
         View qn = offset_tokens(Q, t0, e), kn = offset_tokens(K, t0, e), vn = offset_tokens(V, t0, e);
         View on = offset_tokens(O, t0, e);
         float* lse = sv ? reinterpret_cast<float*>(sv + 2 * snap_all) + t0 : nullptr;
-        s = attention_impl(h, qn, dev(K_cache), dev(V_cache), c, kn, vn, b, on, lse, L, st);
-        if (s) return s;
-        s = compress_impl(h, dev(K_cache), dev(V_cache), c, kn, vn, b, dev(K_cache), dev(V_cache), nullptr, st);
+        s = step_impl(h, qn, dev(K_cache), dev(V_cache), c, kn, vn, b, on, lse, L, st);
         if (s) return s;
         c = c + b <= cfg.M ? c + b : cfg.M;
     }

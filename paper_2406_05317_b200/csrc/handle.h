@@ -7,7 +7,7 @@
 
 namespace lococo {
 // Optional CUDA-event timing of individual kernel classes, on the launching stream.
-enum ProfKind { PROF_CONV = 0, PROF_ATTENTION = 1, PROF_KINDS = 2 };
+enum ProfKind { PROF_CONV = 0, PROF_ATTENTION = 1, PROF_STEP = 2, PROF_KINDS = 3 };
 struct Profiler {
     struct Rec { cudaEvent_t a, b; int kind; };
     bool on = false;
@@ -45,5 +45,6 @@ bool tensor_compress_supported(const lococo_handle* h, const CompressParams& p);
 int tensor_compress(lococo_handle* h, const CompressParams& p, cudaStream_t st);
 bool tensor_attention_supported(const lococo_handle* h, const AttnParams& p);
 int tensor_attention(lococo_handle* h, const AttnParams& p, cudaStream_t st);
+int tensor_chunk_step(lococo_handle* h, const AttnParams& a, const CompressParams& p, cudaStream_t st);
 
 }  // namespace lococo

@@ -61,10 +61,11 @@ __global__ void pack_image_kernel(const __nv_bfloat16* __restrict__ G, __nv_bflo
     }
 }
 
-__global__ void __launch_bounds__(kThreads, 1) compress_tc_kernel(const __grid_constant__ TcCompressParams P) {
-    extern __shared__ __align__(128) uint8_t smem[];
+// Work of one CTA: tiles [part*tiles_per_part, ...) of slot block sb of unit u. Runs with any
+// block size that is a multiple of 32 and at least 192 (warps beyond the sixth only help staging).
+__device__ __forceinline__ void compress_body(const TcCompressParams& P, uint8_t* smem, int part, int sb, int u) {
     const CompressParams& p = P.base;
-    const int part = blockIdx.x, sb = blockIdx.y, u = blockIdx.z;
+    const int nthr16 = blockDim.x / 16;
     const int n = u / p.heads, h = u % p.heads;
     const int tid = threadIdx.x, warp = tid >> 5;
     const int n_tile = P.n_tile, pad = (p.k - 1) / 2, rows = n_tile + p.k - 1;
@@ -146,10 +147,10 @@ __global__ void __launch_bounds__(kThreads, 1) compress_tc_kernel(const __grid_c
                 cp_async16(d0 + r * 16, src, valid ? 16u : 0u);
             }
         };
-        stage_tile(p.xk, zk, tid, kThreads / 16);
+        stage_tile(p.xk, zk, tid, nthr16);
         // the value tile is a conv input only when c_in = 2d; otherwise it is needed by the
         // blend only and is staged by the epilogue warps while the conv runs
-        if (P.halves == 2) stage_tile(p.xv, zv, tid, kThreads / 16);
+        if (P.halves == 2) stage_tile(p.xv, zv, tid, nthr16);
         cp_async_wait_all();
         fence_proxy_async();
         __syncthreads();
@@ -269,6 +270,11 @@ __global__ void __launch_bounds__(kThreads, 1) compress_tc_kernel(const __grid_c
     }
 }
 
+__global__ void __launch_bounds__(kThreads, 1) compress_tc_kernel(const __grid_constant__ TcCompressParams P) {
+    extern __shared__ __align__(128) uint8_t smem[];
+    compress_body(P, smem, blockIdx.x, blockIdx.y, blockIdx.z);
+}
+
 // cache = (sum of partial blends) / (sum of partial row sums + eps)   (Eq. 7 after Eq. 4-5)
 // One block per 32 slots x 32 channels: the partials are channel-major (read along slots),
 // the cache is slot-major (written along channels); the tile is transposed in shared memory.
@@ -327,12 +333,12 @@ struct TcAttnParams {
     int* status;
 };
 
-__global__ void __launch_bounds__(kAttnThreads, 1) attention_tc_kernel(const __grid_constant__ TcAttnParams P) {
-    extern __shared__ __align__(128) uint8_t smem[];
+// Work of one CTA (exactly kAttnThreads threads): query tile qtile of unit u.
+__device__ __forceinline__ void attention_body(const TcAttnParams& P, uint8_t* smem, int qtile, int u) {
     const AttnParams& p = P.base;
-    const int u = blockIdx.y, n = u / p.heads, h = u % p.heads;
+    const int n = u / p.heads, h = u % p.heads;
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-    const int r0 = blockIdx.x * 128;
+    const int r0 = qtile * 128;
     const int S = p.c + p.b;
 
     uint8_t* q_ptr = smem;
@@ -529,6 +535,40 @@ __global__ void __launch_bounds__(kAttnThreads, 1) attention_tc_kernel(const __g
     }
 }
 
+__global__ void __launch_bounds__(kAttnThreads, 1) attention_tc_kernel(const __grid_constant__ TcAttnParams P) {
+    extern __shared__ __align__(128) uint8_t smem[];
+    attention_body(P, smem, blockIdx.x, blockIdx.y);
+}
+
+// ------------------------------------------------------------------ one chunk step, one launch
+// Step 3 (attention with the OLD cache) and Steps 4-5 (the new cache) of Algorithm 2 read the same
+// inputs and do not depend on each other, so their CTAs share one grid: every CTA fills an SM by
+// itself, the attention CTAs differ in length (2..5 key tiles), and a mixed grid lets the block
+// scheduler pack all of them onto the 148 SMs instead of two launches of 128 CTAs each.
+// Block order: the long attention tiles first, then the compress CTAs, then the short attention tiles.
+struct TcStepParams {
+    TcAttnParams attn;
+    TcCompressParams comp;
+    int qtiles, n_attn_first, n_attn, comp_per_unit;   // comp_per_unit = parts * slot_blocks
+};
+
+__global__ void __launch_bounds__(kAttnThreads, 1) chunk_step_tc_kernel(const __grid_constant__ TcStepParams P) {
+    extern __shared__ __align__(128) uint8_t smem[];
+    const int units = P.attn.base.units;
+    int idx = blockIdx.x;
+    const int n_comp = units * P.comp_per_unit;
+    if (idx < P.n_attn_first) {
+        attention_body(P.attn, smem, P.qtiles - 1 - idx / units, idx % units);
+    } else if (idx < P.n_attn_first + n_comp) {
+        idx -= P.n_attn_first;
+        const int u = idx / P.comp_per_unit, rem = idx % P.comp_per_unit;
+        compress_body(P.comp, smem, rem % P.comp.parts, rem / P.comp.parts, u);
+    } else {
+        idx -= n_comp;
+        attention_body(P.attn, smem, P.qtiles - 1 - idx / units, idx % units);
+    }
+}
+
 struct Plan {
     int n_tile, tiles, parts, tiles_per_part, stages, rows_pad;
     size_t smem;
@@ -608,19 +648,13 @@ bool tensor_compress_supported(const lococo_handle* h, const CompressParams& p) 
     return h->use_tensor && p.S >= 1 && make_plan(p.S, p.k, p.units, p.M / kSlots, &pl);
 }
 
-int tensor_compress(lococo_handle* h, const CompressParams& p, cudaStream_t st) {
+static bool build_compress_params(lococo_handle* h, const CompressParams& p, TcCompressParams* out) {
     const int SB = p.M / kSlots;
     Plan pl;
-    if (!make_plan(p.S, p.k, p.units, SB, &pl)) return -1;
-    static bool attr_set = false;
-    if (!attr_set) {
-        if (cudaFuncSetAttribute(compress_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxSmem) != cudaSuccess)
-            return -1;
-        attr_set = true;
-    }
+    if (!make_plan(p.S, p.k, p.units, SB, &pl)) return false;
     const int Smax = h->cfg.M + h->cfg.max_chunk;
     const int max_parts = std::min(parts_cap(h->units, SB), (Smax + 63) / 64);
-    if (pl.parts > max_parts) return -1;
+    if (pl.parts > max_parts) return false;
     TcCompressParams P{};
     P.base = p;
     P.gimage = reinterpret_cast<const __nv_bfloat16*>(h->ws + h->off_gimage);
@@ -630,15 +664,14 @@ int tensor_compress(lococo_handle* h, const CompressParams& p, cudaStream_t st) 
     P.status = reinterpret_cast<int*>(h->ws + h->off_status);
     P.n_tile = pl.n_tile; P.tiles = pl.tiles; P.parts = pl.parts; P.tiles_per_part = pl.tiles_per_part;
     P.halves = p.c_in / 128; P.stages = pl.stages; P.rows_pad = pl.rows_pad; P.slot_blocks = SB;
+    *out = P;
+    return true;
+}
+
+// finalize (+ optional mixing-weight output) after the compress CTAs of either launch form
+static int finish_compress(const TcCompressParams& P, cudaStream_t st) {
+    const CompressParams& p = P.base;
     int launches = 0;
-    dim3 grid(pl.parts, SB, p.units);
-    prof_begin(p.prof, 0, st);
-    // the full 227 KB keeps one CTA per SM, so a CTA always finds its 512 TMEM columns free
-    compress_tc_kernel<<<grid, kThreads, kMaxSmem, st>>>(P);
-    const bool ok = cudaGetLastError() == cudaSuccess;
-    prof_end(p.prof, st);
-    if (!ok) return -1;
-    ++launches;
     dim3 fgrid(p.M / 32, kD / 32, p.units);
     finalize_parts_kernel<<<fgrid, 256, 0, st>>>(P);
     if (cudaGetLastError() != cudaSuccess) return -1;
@@ -649,6 +682,52 @@ int tensor_compress(lococo_handle* h, const CompressParams& p, cudaStream_t st) 
         launches += r;
     }
     return launches;
+}
+
+int tensor_compress(lococo_handle* h, const CompressParams& p, cudaStream_t st) {
+    TcCompressParams P;
+    if (!build_compress_params(h, p, &P)) return -1;
+    static bool attr_set = false;
+    if (!attr_set) {
+        if (cudaFuncSetAttribute(compress_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxSmem) != cudaSuccess)
+            return -1;
+        attr_set = true;
+    }
+    dim3 grid(P.parts, P.slot_blocks, p.units);
+    prof_begin(p.prof, 0, st);
+    // the full 227 KB keeps one CTA per SM, so a CTA always finds its 512 TMEM columns free
+    compress_tc_kernel<<<grid, kThreads, kMaxSmem, st>>>(P);
+    const bool ok = cudaGetLastError() == cudaSuccess;
+    prof_end(p.prof, st);
+    if (!ok) return -1;
+    const int r = finish_compress(P, st);
+    return r < 0 ? -1 : 1 + r;
+}
+
+// Attention with the old cache and the cache update of one chunk in a single launch.
+int tensor_chunk_step(lococo_handle* h, const AttnParams& a, const CompressParams& p, cudaStream_t st) {
+    TcStepParams P{};
+    if (!build_compress_params(h, p, &P.comp)) return -1;
+    P.attn.base = a;
+    P.attn.status = P.comp.status;
+    static bool attr_set = false;
+    if (!attr_set) {
+        if (cudaFuncSetAttribute(chunk_step_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxSmem) != cudaSuccess)
+            return -1;
+        attr_set = true;
+    }
+    P.qtiles = (a.b + 127) / 128;
+    P.n_attn = P.qtiles * a.units;
+    P.n_attn_first = ((P.qtiles + 1) / 2) * a.units;
+    P.comp_per_unit = P.comp.parts * P.comp.slot_blocks;
+    const int blocks = P.n_attn + a.units * P.comp_per_unit;
+    prof_begin(p.prof, 2, st);
+    chunk_step_tc_kernel<<<blocks, kAttnThreads, kMaxSmem, st>>>(P);
+    const bool ok = cudaGetLastError() == cudaSuccess;
+    prof_end(p.prof, st);
+    if (!ok) return -1;
+    const int r = finish_compress(P.comp, st);
+    return r < 0 ? -1 : 1 + r;
 }
 
 bool tensor_attention_supported(const lococo_handle* h, const AttnParams& p) {
