@@ -141,7 +141,7 @@ class Lococo:
 
     def __del__(self):
         h = getattr(self, "_h", None)
-        if h:
+        if h and _lib is not None:      # at interpreter shutdown the module globals may be gone already
             _lib.lococo_destroy(h)
             self._h = None
 

@@ -314,19 +314,27 @@ __global__ void __launch_bounds__(256) finalize_parts_kernel(TcCompressParams P)
 
 
 // ------------------------------------------------------------------ Eq. 1, chunk form
-// One CTA = 128 queries of one unit. Per 128-key tile of [cache; chunk]:
-//   S = Q K^T on the tensor cores (both operands K-major, staged un-swizzled),
-//   two threads per query row (each owns 64 of the 128 columns) read S from TMEM, apply
-//   the scale, the causal mask and the running-max update, and write P (bf16) to shared
-//   memory as an MMA A operand,
-//   O_tile = P V on the tensor cores (V read MN-major from its staged tile),
-//   and each thread rescales and updates its 64 fp32 output columns in registers.
-constexpr int kAttnThreads = 288;                  // 8 softmax warps + 1 control warp
-constexpr uint32_t kLboT = 129 * 16;               // byte stride between 8-channel groups of a staged 128-row tile
+// One CTA = 128 queries of one unit, pipelined over 128-key tiles of [cache; chunk] with three
+// kinds of warps that only meet at mbarriers:
+//   loaders (2 warps)   stage Q once and the K/V tiles, double-buffered, with cp.async;
+//   MMA issuer (1 lane) S_t = Q K_t^T into one of two TMEM buffers, then O += P_{t-1} V_{t-1},
+//                       so the next tile's logits are computed while this tile's softmax runs;
+//   softmax (8 warps)   two threads per query row (64 columns each): row maximum, P = exp2(s - m)
+//                       in bf16 to shared memory (double-buffered MMA A operand), running row sum.
+// O stays in TMEM for the whole CTA. The reference maximum m of a row is raised only when a
+// tile's maximum exceeds it by more than 8 (in log2 units): P then reaches at most 2^8, which
+// bf16 and the fp32 accumulator hold just as well, and the rescale of O (a TMEM round trip)
+// becomes rare; all sums use the same m, so the result is the exact softmax.
+constexpr int kAttnThreads = 384;                  // 8 softmax + 1 MMA-issue + 3 loader warps (384 x 168 registers fill the file)
+constexpr int kAttnLoaderWarps = 3;
+constexpr int kAttnLoaders = 32 * kAttnLoaderWarps;
+constexpr uint32_t kLboT = 129 * 16;               // Q/K/V tiles: [16 channel groups][129 x 16 B]: the odd row count
+                                                   // spreads the 16 groups of a row over the banks (cp.async writes)
 constexpr uint32_t kTileBytes = 16 * kLboT;        // 33024
-constexpr uint32_t kPBytes = 16 * 2048;            // P tile: [16 key groups][128 rows][8 keys]
-constexpr uint32_t kAttnSmem = 5 * kTileBytes + kPBytes + 2 * 128 * 4 + 64;
-constexpr uint32_t kAttnTmemCols = 256;
+constexpr uint32_t kPBytes = 32768;                // P tiles: [16 key groups][128 rows][8 keys]
+constexpr uint32_t kAttnSmem = 5 * kTileBytes + 2 * kPBytes + 256 * 4 + 128;   // Q, K x2, V x2, P x2, exchange, barriers
+constexpr uint32_t kAttnTmemCols = 512;            // S x2 (128 columns each), O (128)
+constexpr float kRescaleThreshold = 8.f;
 
 struct TcAttnParams {
     AttnParams base;
@@ -344,18 +352,31 @@ __device__ __forceinline__ void attention_body(const TcAttnParams& P, uint8_t* s
     uint8_t* q_ptr = smem;
     uint8_t* k_ptr = q_ptr + kTileBytes;       // two buffers
     uint8_t* v_ptr = k_ptr + 2 * kTileBytes;   // two buffers
-    uint8_t* p_ptr = v_ptr + 2 * kTileBytes;
-    float* xchg = reinterpret_cast<float*>(p_ptr + kPBytes);   // [2 halves][128 rows]
+    uint8_t* p_ptr = v_ptr + 2 * kTileBytes;   // two buffers
+    float* xchg = reinterpret_cast<float*>(p_ptr + 2 * kPBytes);      // [2 halves][128 rows]
     uint64_t* bars = reinterpret_cast<uint64_t*>(xchg + 256);
-    volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(bars + 2);
+    volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(bars + 12);
     volatile int* failed = reinterpret_cast<volatile int*>(tmem_slot + 1);
     const uint32_t qs = smem_u32(q_ptr), ks = smem_u32(k_ptr), vs = smem_u32(v_ptr), ps = smem_u32(p_ptr);
-    const uint32_t bar_s = smem_u32(bars), bar_o = bar_s + 8;
-    constexpr int kCtl = 256;                  // control thread (lane 0 of warp 8)
+    const uint32_t bar0 = smem_u32(bars);
+    // all indexed by b = tile & 1; the n-th use of a buffer completes phase n of its barriers
+    auto k_full = [&](int b) { return bar0 + 8 * b; };          // loaders -> MMA: K tile staged (first phase: Q too)
+    auto v_full = [&](int b) { return bar0 + 80 + 8 * b; };     // loaders -> MMA: V tile staged
+    auto s_full = [&](int b) { return bar0 + 16 + 8 * b; };     // MMA -> softmax: logits in TMEM
+    auto s_free = [&](int b) { return bar0 + 32 + 8 * b; };     // softmax -> MMA: logits consumed
+    auto p_full = [&](int b) { return bar0 + 48 + 8 * b; };     // softmax -> MMA: P written
+    auto pv_done = [&](int b) { return bar0 + 64 + 8 * b; };    // MMA -> loaders, softmax: K/V/P buffers free, O updated
+    constexpr int kMma = 256;                                   // lane 0 of warp 8
 
-    if (tid == kCtl) {
-        mbar_init(bar_s, 1);
-        mbar_init(bar_o, 1);
+    if (tid == kMma) {
+        for (int b = 0; b < 2; ++b) {
+            mbar_init(k_full(b), kAttnLoaders);
+            mbar_init(v_full(b), kAttnLoaders);
+            mbar_init(s_full(b), 1);
+            mbar_init(s_free(b), 256);
+            mbar_init(p_full(b), 256);
+            mbar_init(pv_done(b), 1);
+        }
         *failed = 0;
         fence_barrier_init();
     }
@@ -372,82 +393,138 @@ __device__ __forceinline__ void attention_body(const TcAttnParams& P, uint8_t* s
     const int last_row = min(r0 + 127, p.b - 1);
     const int ncols = p.c + last_row + 1;           // columns any query of this tile can see
     const int ntiles = (ncols + 127) / 128;
-    const __nv_bfloat16* safe = unit_base<__nv_bfloat16>(p.q, n, h);
 
-    // each thread owns one 8-channel group and every 18th row of a tile
-    const int lq = tid & 15, lr0 = tid >> 4;
-    const __nv_bfloat16* kc_base = unit_base<__nv_bfloat16>(p.xk.cache, n, h) + lq * 8;
-    const __nv_bfloat16* kn_base = unit_base<__nv_bfloat16>(p.xk.chunk, n, h) + lq * 8;
-    const __nv_bfloat16* vc_base = unit_base<__nv_bfloat16>(p.xv.cache, n, h) + lq * 8;
-    const __nv_bfloat16* vn_base = unit_base<__nv_bfloat16>(p.xv.chunk, n, h) + lq * 8;
-    auto load_kv = [&](int jt, int buf) {
-        const uint32_t d0 = buf * kTileBytes + lq * kLboT;
-        for (int r = lr0; r < 128; r += kAttnThreads / 16) {
-            const int j = jt * 128 + r;
-            const bool valid = j < S;
-            const bool in_cache = j < p.c;
-            const __nv_bfloat16* sk = !valid ? safe : in_cache ? kc_base + (int64_t)j * p.xk.cache.st
-                                                               : kn_base + (int64_t)(j - p.c) * p.xk.chunk.st;
-            const __nv_bfloat16* sv = !valid ? safe : in_cache ? vc_base + (int64_t)j * p.xv.cache.st
-                                                               : vn_base + (int64_t)(j - p.c) * p.xv.chunk.st;
-            cp_async16(ks + d0 + r * 16, sk, valid ? 16u : 0u);
-            cp_async16(vs + d0 + r * 16, sv, valid ? 16u : 0u);
+    // ---- staging of one 128-row tile by `nw` warps, this warp being number `lw` of them: 16 lanes
+    // per row (256 contiguous bytes in global memory), two rows per warp instruction. Rows at or
+    // beyond `nrows` are zero-filled.
+    const __nv_bfloat16* safe = unit_base<__nv_bfloat16>(p.q, n, h);
+    auto stage_rows = [&](uint32_t dst, const __nv_bfloat16* base, int64_t st, int nrows, int lw, int nw) {
+        const int q = lane & 15;
+        const uint32_t d0 = dst + q * kLboT;
+        const __nv_bfloat16* b0 = base + q * 8;
+        for (int r = 2 * lw + (lane >> 4); r < 128; r += 2 * nw) {
+            const bool valid = r < nrows;
+            cp_async16(d0 + r * 16, valid ? b0 + (int64_t)r * st : safe, valid ? 16u : 0u);
         }
     };
-    // queries of this tile (zeros beyond the chunk) and the first key/value tile
-    for (int r = lr0; r < 128; r += kAttnThreads / 16) {
-        const bool valid = r0 + r < p.b;
-        const __nv_bfloat16* sq = valid ? unit_base<__nv_bfloat16>(p.q, n, h) + (int64_t)(r0 + r) * p.q.st + lq * 8 : safe;
-        cp_async16(qs + lq * kLboT + r * 16, sq, valid ? 16u : 0u);
+    // keys (which = 0) or values (1) of key tile jt: the part inside the cache, then the part inside the chunk
+    auto load_tile = [&](int jt, int buf, int which, int lw, int nw) {
+        const CatView& x = which ? p.xv : p.xk;
+        const uint32_t dst = (which ? vs : ks) + buf * kTileBytes;
+        const int jb = jt * 128;
+        if (jb + 128 <= p.c) {
+            stage_rows(dst, unit_base<__nv_bfloat16>(x.cache, n, h) + (int64_t)jb * x.cache.st, x.cache.st, 128, lw, nw);
+        } else if (jb >= p.c) {
+            stage_rows(dst, unit_base<__nv_bfloat16>(x.chunk, n, h) + (int64_t)(jb - p.c) * x.chunk.st, x.chunk.st, S - jb, lw, nw);
+        } else {
+            // the tile straddles the end of the cache: row by row
+            const int q = lane & 15;
+            for (int r = 2 * lw + (lane >> 4); r < 128; r += 2 * nw) {
+                const int j = jb + r;
+                const bool valid = j < S;
+                const __nv_bfloat16* src = !valid ? safe
+                    : j < p.c ? unit_base<__nv_bfloat16>(x.cache, n, h) + (int64_t)j * x.cache.st + q * 8
+                              : unit_base<__nv_bfloat16>(x.chunk, n, h) + (int64_t)(j - p.c) * x.chunk.st + q * 8;
+                cp_async16(dst + q * kLboT + r * 16, src, valid ? 16u : 0u);
+            }
+        }
+    };
+    // ---- prologue, all warps: Q and the first two key/value tiles
+    {
+        constexpr int nw = kAttnThreads / 32;
+        stage_rows(qs, safe + (int64_t)r0 * p.q.st, p.q.st, p.b - r0, warp, nw);
+        load_tile(0, 0, 0, warp, nw);
+        load_tile(0, 0, 1, warp, nw);
+        if (ntiles > 1) {
+            load_tile(1, 1, 0, warp, nw);
+            load_tile(1, 1, 1, warp, nw);
+        }
+        cp_async_wait_all();
+        fence_proxy_async();
+        __syncthreads();
     }
-    load_kv(0, 0);
-    asm volatile("cp.async.commit_group;" ::: "memory");
 
-    const uint32_t idesc_s = instr_desc_bf16(128, false, false);
-    const uint32_t idesc_o = instr_desc_bf16(128, false, true);
+    if (warp >= 9) {
+        // ---------------- loaders
+        const int lw = warp - 9;
+        auto commit = [&]() { asm volatile("cp.async.commit_group;" ::: "memory"); };
+        // tiles 0 and 1 were staged by the prologue
+        mbar_arrive(k_full(0));
+        mbar_arrive(v_full(0));
+        if (ntiles > 1) {
+            mbar_arrive(k_full(1));
+            mbar_arrive(v_full(1));
+        }
+        // from here on, per-thread group order: [K(t+1)] [V(t+1)] ...; a tile is announced to the MMA
+        // issuer before this warp waits for any buffer that the issuer has to free
+        for (int jt = 1; jt + 1 < ntiles; ++jt) {
+            // tile jt is already announced; refill the buffers of tile jt-1 with tile jt+1. The key
+            // tile is announced as soon as it lands: the next S MMA needs it long before the value
+            // buffer is even free.
+            const int pb = (jt - 1) & 1, pph = ((jt - 1) >> 1) & 1;
+            mbar_wait(s_full(pb), pph, P.status, failed, 4);      // S(jt-1) has read the key buffer
+            load_tile(jt + 1, pb, 0, lw, kAttnLoaderWarps);
+            cp_async_wait_all();
+            fence_proxy_async();
+            mbar_arrive(k_full(pb));
+            mbar_wait(pv_done(pb), pph, P.status, failed, 5);     // PV(jt-1) has read the value buffer
+            load_tile(jt + 1, pb, 1, lw, kAttnLoaderWarps);
+            cp_async_wait_all();
+            fence_proxy_async();
+            mbar_arrive(v_full(pb));
+        }
+    } else if (tid == kMma) {
+        // ---------------- MMA issuer: S(0), then per tile S(t) followed by PV(t-1)
+        const uint32_t idesc_s = instr_desc_bf16(128, false, false);
+        const uint32_t idesc_o = instr_desc_bf16(128, false, true);
+        const uint64_t q0 = smem_desc(qs, kLboT, 128);
+        constexpr uint32_t kstep = (2 * kLboT) >> 4;   // two 8-channel groups per MMA
+        auto issue_pv = [&](int t) {
+            const int b = t & 1;
+            mbar_wait(v_full(b), (t >> 1) & 1, P.status, failed, 6);
+            mbar_wait(p_full(b), (t >> 1) & 1, P.status, failed, 6);
+            tc_fence_after();
+            const uint64_t a0 = smem_desc(ps + b * kPBytes, 2048, 128), b0 = smem_desc(vs + b * kTileBytes, 128, kLboT);
+#pragma unroll
+            for (int kk = 0; kk < 8; ++kk) umma_ss(tmem + 256, a0 + kk * 256u, b0 + kk * 16u, idesc_o, (t | kk) != 0);
+            umma_commit(pv_done(b));
+        };
+        for (int jt = 0; jt < ntiles; ++jt) {
+            const int b = jt & 1;
+            mbar_wait(k_full(b), (jt >> 1) & 1, P.status, failed, 7);
+            if (jt >= 2) mbar_wait(s_free(b), ((jt >> 1) - 1) & 1, P.status, failed, 8);
+            tc_fence_after();
+            const uint64_t k0 = smem_desc(ks + b * kTileBytes, kLboT, 128);
+#pragma unroll
+            for (int kk = 0; kk < 8; ++kk) umma_ss(tmem + b * 128, q0 + kk * kstep, k0 + kk * kstep, idesc_s, kk != 0);
+            umma_commit(s_full(b));
+            if (jt >= 1) issue_pv(jt - 1);
+        }
+        issue_pv(ntiles - 1);
+    }
     const int rl = (warp & 3) * 32 + lane;          // row of the tile this thread works on (softmax warps)
     const int half = (warp >> 2) & 1;               // which 64 columns of the row
     const int row = r0 + rl;
     const bool live = warp < 8 && row < p.b;
-    const int vis = live ? p.c + row + 1 : 1;       // visible columns of this row
-    const float sc2 = p.scale * 1.4426950408889634f;
-    float acc[64];
-#pragma unroll
-    for (int e = 0; e < 64; ++e) acc[e] = 0.f;
-    float mrun = -INFINITY, lrun = 0.f;
-    const uint32_t lane_addr = tmem + ((uint32_t)((warp & 3) * 32) << 16) + half * 64;
-
-    for (int jt = 0; jt < ntiles; ++jt) {
-        const int buf = jt & 1;
-        if (jt + 1 < ntiles) {
-            load_kv(jt + 1, buf ^ 1);
-            asm volatile("cp.async.commit_group;" ::: "memory");
-            asm volatile("cp.async.wait_group 1;" ::: "memory");
-        } else {
-            asm volatile("cp.async.wait_group 0;" ::: "memory");
-        }
-        fence_proxy_async();
-        __syncthreads();
-        if (tid == kCtl) {
+    const uint32_t lane_base = tmem + ((uint32_t)((warp & 3) * 32) << 16);
+    if (warp < 8) {
+        // ---------------- softmax
+        float m_used = 0.f, lrun = 0.f;
+        const int vis = live ? p.c + row + 1 : 1;   // visible columns of this row
+        const float sc2 = p.scale * 1.4426950408889634f;
+        for (int jt = 0; jt < ntiles; ++jt) {
+            const int b = jt & 1;
+            mbar_wait(s_full(b), (jt >> 1) & 1, P.status, failed, 9);
             tc_fence_after();
-            const uint64_t a0 = smem_desc(qs, kLboT, 128), b0 = smem_desc(ks + buf * kTileBytes, kLboT, 128);
-#pragma unroll
-            for (int kk = 0; kk < 8; ++kk) umma_ss(tmem, a0 + kk * ((2 * kLboT) >> 4), b0 + kk * ((2 * kLboT) >> 4), idesc_s, kk != 0);
-            umma_commit(bar_s);
-        }
-        float corr = 1.f;
-        if (warp < 8) {
-            mbar_wait(bar_s, jt & 1, P.status, failed, 5);
-            tc_fence_after();
+            const uint32_t s_addr = lane_base + b * 128 + half * 64;
             const int j0 = jt * 128 + half * 64;
             const bool need_mask = jt * 128 + 128 > p.c + r0;
-            // pass 1: maximum of this thread's 64 scaled, masked logits; the row maximum is
-            // shared with the partner thread through shared memory
+            // pass 1: maximum of this thread's 64 scaled, masked logits, shared with the partner
             float tmax = -INFINITY;
 #pragma unroll
             for (int c0 = 0; c0 < 64; c0 += 32) {
                 uint32_t v[32];
-                tmem_ld32(lane_addr + c0, v);
+                tmem_ld32(s_addr + c0, v);
                 tmem_ld_wait();
 #pragma unroll
                 for (int e = 0; e < 32; ++e) {
@@ -457,14 +534,39 @@ __device__ __forceinline__ void attention_body(const TcAttnParams& P, uint8_t* s
             }
             xchg[half * 128 + rl] = tmax;
             asm volatile("bar.sync 1, 256;" ::: "memory");
-            const float mnew = fmaxf(mrun, fmaxf(tmax, xchg[(half ^ 1) * 128 + rl]));
-            corr = exp2f(mrun - mnew);
-            float lsum = 0.f;
+            const float mt = fmaxf(tmax, xchg[(half ^ 1) * 128 + rl]);
+            asm volatile("bar.sync 1, 256;" ::: "memory");      // the slot is rewritten for the next tile
+            if (jt == 0) {
+                m_used = mt;        // finite: column 0 is visible to every row
+            } else {
+                // raise the reference maximum only for a large jump; O in TMEM is rescaled to match
+                const bool bump = mt > m_used + kRescaleThreshold;
+                if (__any_sync(0xffffffffu, bump)) {
+                    const float f = bump ? exp2f(m_used - mt) : 1.f;
+                    mbar_wait(pv_done((jt - 1) & 1), ((jt - 1) >> 1) & 1, P.status, failed, 10);
+                    tc_fence_after();
+#pragma unroll
+                    for (int c0 = 0; c0 < 64; c0 += 32) {
+                        uint32_t v[32];
+                        tmem_ld32(lane_base + 256 + half * 64 + c0, v);
+                        tmem_ld_wait();
+#pragma unroll
+                        for (int e = 0; e < 32; ++e) v[e] = __float_as_uint(__uint_as_float(v[e]) * f);
+                        tmem_st32(lane_base + 256 + half * 64 + c0, v);
+                    }
+                    tmem_st_wait();
+                    lrun *= f;
+                    if (bump) m_used = mt;
+                }
+            }
             // pass 2: P = exp2(s - m), bf16, into the A-operand layout [key group][row][8 keys]
+            if (jt >= 2) mbar_wait(pv_done(b), ((jt >> 1) - 1) & 1, P.status, failed, 11);
+            uint8_t* pdst = p_ptr + b * kPBytes + rl * 16;
+            float lsum = 0.f;
 #pragma unroll
             for (int c0 = 0; c0 < 64; c0 += 32) {
                 uint32_t v[32];
-                tmem_ld32(lane_addr + c0, v);
+                tmem_ld32(s_addr + c0, v);
                 tmem_ld_wait();
 #pragma unroll
                 for (int e = 0; e < 32; e += 8) {
@@ -472,63 +574,52 @@ __device__ __forceinline__ void attention_body(const TcAttnParams& P, uint8_t* s
 #pragma unroll
                     for (int x = 0; x < 8; x += 2) {
                         const int ja = j0 + c0 + e + x;
-                        float pa = exp2f(__uint_as_float(v[e + x]) * sc2 - mnew);
-                        float pb = exp2f(__uint_as_float(v[e + x + 1]) * sc2 - mnew);
+                        float pa = exp2f(__uint_as_float(v[e + x]) * sc2 - m_used);
+                        float pb = exp2f(__uint_as_float(v[e + x + 1]) * sc2 - m_used);
                         if (need_mask && ja >= vis) pa = 0.f;
                         if (need_mask && ja + 1 >= vis) pb = 0.f;
                         const __nv_bfloat162 pr = __floats2bfloat162_rn(pa, pb);
                         pk[x >> 1] = *reinterpret_cast<const uint32_t*>(&pr);
                         lsum += __low2float(pr) + __high2float(pr);
                     }
-                    *reinterpret_cast<uint4*>(p_ptr + ((half * 64 + c0 + e) >> 3) * 2048 + rl * 16) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
+                    *reinterpret_cast<uint4*>(pdst + ((half * 64 + c0 + e) >> 3) * 2048) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
                 }
             }
-            lrun = lrun * corr + lsum;
-            mrun = mnew;
+            lrun += lsum;
+            tc_fence_before();
+            mbar_arrive(s_free(b));      // this thread's reads of S[b] are complete (wait::ld above)
             fence_proxy_async();
+            mbar_arrive(p_full(b));
         }
-        tc_fence_before();
-        __syncthreads();
-        if (tid == kCtl) {
-            tc_fence_after();
-            const uint64_t a0 = smem_desc(ps, 2048, 128), b0 = smem_desc(vs + buf * kTileBytes, 128, kLboT);
-#pragma unroll
-            for (int kk = 0; kk < 8; ++kk) umma_ss(tmem + 128, a0 + kk * 256u, b0 + kk * 16u, idesc_o, kk != 0);
-            umma_commit(bar_o);
-        }
-        // everybody holds back until the tile's MMAs are done: P, S and the key/value buffer are reused
-        mbar_wait(bar_o, jt & 1, P.status, failed, 6);
-        if (warp < 8) {
-            tc_fence_after();
-#pragma unroll
-            for (int c0 = 0; c0 < 64; c0 += 32) {
-                uint32_t v[32];
-                tmem_ld32(lane_addr + 128 + c0, v);
-                tmem_ld_wait();
-#pragma unroll
-                for (int e = 0; e < 32; ++e) acc[c0 + e] = fmaf(acc[c0 + e], corr, __uint_as_float(v[e]));
-            }
-        }
-    }
-    // row sum = sum of the two partners' partial sums
-    if (warp < 8) xchg[half * 128 + rl] = lrun;
-    tc_fence_before();
-    __syncthreads();
-    if (live) {
+        // the last PV has updated O
+        mbar_wait(pv_done((ntiles - 1) & 1), ((ntiles - 1) >> 1) & 1, P.status, failed, 12);
+        tc_fence_after();
+        xchg[half * 128 + rl] = lrun;
+        asm volatile("bar.sync 1, 256;" ::: "memory");
         const float ltot = lrun + xchg[(half ^ 1) * 128 + rl];
         const float inv = 1.f / ltot;
-        __nv_bfloat16* orow = unit_base_mut<__nv_bfloat16>(p.o, n, h) + (int64_t)row * p.o.st + half * 64;
+        __nv_bfloat16* orow = unit_base_mut<__nv_bfloat16>(p.o, n, h) + (int64_t)(live ? row : 0) * p.o.st + half * 64;
 #pragma unroll
-        for (int e = 0; e < 64; e += 8) {
-            uint4 o;
-            o.x = pack_bf16(acc[e] * inv, acc[e + 1] * inv);
-            o.y = pack_bf16(acc[e + 2] * inv, acc[e + 3] * inv);
-            o.z = pack_bf16(acc[e + 4] * inv, acc[e + 5] * inv);
-            o.w = pack_bf16(acc[e + 6] * inv, acc[e + 7] * inv);
-            *reinterpret_cast<uint4*>(orow + e) = o;
+        for (int c0 = 0; c0 < 64; c0 += 32) {
+            uint32_t v[32];
+            tmem_ld32(lane_base + 256 + half * 64 + c0, v);
+            tmem_ld_wait();
+            if (live) {
+#pragma unroll
+                for (int e = 0; e < 32; e += 8) {
+                    uint4 o;
+                    o.x = pack_bf16(__uint_as_float(v[e]) * inv, __uint_as_float(v[e + 1]) * inv);
+                    o.y = pack_bf16(__uint_as_float(v[e + 2]) * inv, __uint_as_float(v[e + 3]) * inv);
+                    o.z = pack_bf16(__uint_as_float(v[e + 4]) * inv, __uint_as_float(v[e + 5]) * inv);
+                    o.w = pack_bf16(__uint_as_float(v[e + 6]) * inv, __uint_as_float(v[e + 7]) * inv);
+                    *reinterpret_cast<uint4*>(orow + c0 + e) = o;
+                }
+            }
         }
-        if (p.lse && half == 0) p.lse[(int64_t)u * p.lse_stride + row] = (mrun + log2f(ltot)) * 0.6931471805599453f;
+        if (live && p.lse && half == 0) p.lse[(int64_t)u * p.lse_stride + row] = (m_used + log2f(ltot)) * 0.6931471805599453f;
     }
+    tc_fence_before();
+    __syncthreads();
     if (warp == 8) {
         __syncwarp();
         tmem_dealloc(tmem, kAttnTmemCols);
