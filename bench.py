@@ -201,6 +201,11 @@ def run_ours(args):
     staging = torch.empty(ctx.host_staging_bytes(w.L), dtype=torch.uint8, device="cuda")
     flush = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")   # larger than the 126 MB L2
 
+    # a side stream: the library replays the chunk loop from a CUDA graph on capturable streams only
+    side = torch.cuda.Stream()
+    torch.cuda.synchronize()
+    torch.cuda.set_stream(side)
+
     def barrier():
         if world > 1:
             dist.barrier()

@@ -171,6 +171,9 @@ lococo_status lococo_saved_bytes(const lococo_handle* handle, int32_t L, int32_t
  * Q, K, V, O hold L tokens; K_cache/V_cache (M rows per unit) and *cache_len_inout
  * (host) carry the cache state in and out, so a sequence can be suspended and resumed
  * between calls.  saved (device, optional) is laid out as lococo_saved_bytes describes.
+ * Calls that repeat the previous call's arguments exactly (same views, L, B, cache length) on a
+ * capturable stream (not the legacy default stream) are replayed from a cached CUDA graph from the
+ * third such call on; buffer contents may change freely between calls.
  */
 lococo_status lococo_process_sequence(lococo_handle* handle, lococo_tensor Q, lococo_tensor K, lococo_tensor V,
                                       int32_t L, int32_t B, lococo_tensor O, lococo_tensor K_cache,

@@ -57,6 +57,14 @@ lococo_status ready(const lococo_handle* h) {
     return LOCOCO_OK;
 }
 
+// The cached loop graph holds workspace pointers and the bias choice: drop it when they change.
+void drop_loop_graph(lococo_handle* h) {
+    if (h->loop_graph.exec) cudaGraphExecDestroy(h->loop_graph.exec);
+    h->loop_graph.exec = nullptr;
+    h->loop_graph.key_len = 0;
+    h->loop_graph.seen = 0;
+}
+
 lococo_status count(lococo_handle* h, int launched) {
     if (launched < 0) return LOCOCO_ERR_CUDA;
     h->launches += launched;
@@ -249,6 +257,7 @@ lococo_status lococo_create(const lococo_config* c, lococo_handle** out) {
 lococo_status lococo_destroy(lococo_handle* h) {
     if (!h) return LOCOCO_ERR_INVALID_ARG;
     h->prof.release();
+    if (h->loop_graph.exec) cudaGraphExecDestroy(h->loop_graph.exec);
     delete h;
     return LOCOCO_OK;
 }
@@ -263,6 +272,7 @@ lococo_status lococo_set_workspace(lococo_handle* h, void* ptr, size_t bytes, vo
     if (!h || !ptr) return LOCOCO_ERR_INVALID_ARG;
     if (reinterpret_cast<uintptr_t>(ptr) & 255u) return LOCOCO_ERR_INVALID_ARG;
     if (bytes < h->ws_need) return LOCOCO_ERR_WORKSPACE;
+    drop_loop_graph(h);
     h->ws = static_cast<char*>(ptr);
     h->weights_set = false;
     if (cudaMemsetAsync(h->ws + h->off_status, 0, 256, static_cast<cudaStream_t>(stream)) != cudaSuccess)
@@ -278,6 +288,7 @@ lococo_status lococo_set_weights(lococo_handle* h, const void* G, const void* bi
     const int sets = c.weights_per_head ? c.heads : 1;
     lococo_status s = count(h, simt_pack_weights(c.dtype, G, h->ws + h->off_gpack, sets, c.M, c.c_in, c.k, st));
     if (s) return s;
+    drop_loop_graph(h);
     h->has_bias = bias != nullptr;
     if (bias) {
         s = count(h, simt_convert_bias(c.dtype, bias, reinterpret_cast<float*>(h->ws + h->off_bias), sets * c.M, st));
@@ -335,6 +346,43 @@ lococo_status lococo_saved_bytes(const lococo_handle* h, int32_t L, int32_t B, s
     return LOCOCO_OK;
 }
 
+}  // extern "C"
+
+namespace {
+// Algorithm 2's loop as stream-ordered launches.
+lococo_status run_chunk_loop(lococo_handle* h, lococo_tensor Q, lococo_tensor K, lococo_tensor V, int32_t L, int32_t B,
+                             lococo_tensor O, lococo_tensor K_cache, lococo_tensor V_cache, int* c_inout, void* saved,
+                             cudaStream_t st) {
+    const lococo_config& cfg = h->cfg;
+    const size_t e = h->elt;
+    int c = *c_inout;
+    const int n_chunks = (L + B - 1) / B;
+    const size_t snap_step = (size_t)h->units * cfg.M * cfg.head_dim * e;
+    const size_t snap_all = align_up((size_t)n_chunks * snap_step, 256);
+    char* sv = static_cast<char*>(saved);
+    for (int n = 0; n < n_chunks; ++n) {
+        const int t0 = n * B;
+        const int b = L - t0 < B ? L - t0 : B;
+        if (sv) {
+            lococo_tensor sk = contiguous(sv + (size_t)n * snap_step, cfg.heads, cfg.M, cfg.head_dim);
+            lococo_tensor svv = contiguous(sv + snap_all + (size_t)n * snap_step, cfg.heads, cfg.M, cfg.head_dim);
+            FillParams f{dev(K_cache), dev(V_cache), dev(sk), dev(svv), cfg.heads, h->units, cfg.head_dim, 0, cfg.M};
+            lococo_status s = count(h, simt_fill(cfg.dtype, f, st));
+            if (s) return s;
+        }
+        View qn = offset_tokens(Q, t0, e), kn = offset_tokens(K, t0, e), vn = offset_tokens(V, t0, e);
+        View on = offset_tokens(O, t0, e);
+        float* lse = sv ? reinterpret_cast<float*>(sv + 2 * snap_all) + t0 : nullptr;
+        lococo_status s = step_impl(h, qn, dev(K_cache), dev(V_cache), c, kn, vn, b, on, lse, L, st);
+        if (s) return s;
+        c = c + b <= cfg.M ? c + b : cfg.M;
+    }
+    *c_inout = c;
+    return LOCOCO_OK;
+}
+}  // namespace
+
+extern "C" {
 lococo_status lococo_process_sequence(lococo_handle* h, lococo_tensor Q, lococo_tensor K, lococo_tensor V, int32_t L,
                                       int32_t B, lococo_tensor O, lococo_tensor K_cache, lococo_tensor V_cache,
                                       int32_t* cache_len_inout, void* saved, void* stream) {
@@ -349,28 +397,68 @@ lococo_status lococo_process_sequence(lococo_handle* h, lococo_tensor Q, lococo_
     if (O.ptr == Q.ptr || O.ptr == K.ptr || O.ptr == V.ptr || K_cache.ptr == V_cache.ptr) return LOCOCO_ERR_INVALID_ARG;
     if (saved && (reinterpret_cast<uintptr_t>(saved) & 255u)) return LOCOCO_ERR_INVALID_ARG;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
-    const lococo_config& cfg = h->cfg;
-    const int n_chunks = (L + B - 1) / B;
-    const size_t snap_step = (size_t)h->units * cfg.M * cfg.head_dim * e;
-    const size_t snap_all = align_up((size_t)n_chunks * snap_step, 256);
-    char* sv = static_cast<char*>(saved);
-    for (int n = 0; n < n_chunks; ++n) {
-        const int t0 = n * B;
-        const int b = L - t0 < B ? L - t0 : B;
-        if (sv) {
-            lococo_tensor sk = contiguous(sv + (size_t)n * snap_step, cfg.heads, cfg.M, cfg.head_dim);
-            lococo_tensor svv = contiguous(sv + snap_all + (size_t)n * snap_step, cfg.heads, cfg.M, cfg.head_dim);
-            FillParams f{dev(K_cache), dev(V_cache), dev(sk), dev(svv), cfg.heads, h->units, cfg.head_dim, 0, cfg.M};
-            s = count(h, simt_fill(cfg.dtype, f, st));
-            if (s) return s;
+    const int c_in = c;
+
+    // The loop is a fixed sequence of launches for a given argument set, so repeated calls with the
+    // same arguments (a serving loop over one set of buffers) replay it as a CUDA graph: kernel-to-
+    // kernel hand-over inside a graph is shorter than between stream launches. First call: eager.
+    // Second identical call: captured, instantiated, launched. Later calls: graph launch only.
+    lococo_handle::LoopGraph& lg = h->loop_graph;
+    struct Key { lococo_tensor Q, K, V, O, Kc, Vc; void* saved; int32_t L, B, c, pad; } key;
+    std::memset(&key, 0, sizeof(key));   // padding bytes take part in the comparison
+    key.Q = Q; key.K = K; key.V = V; key.O = O; key.Kc = K_cache; key.Vc = V_cache;
+    key.saved = saved; key.L = L; key.B = B; key.c = c_in;
+    static_assert(sizeof(key) <= sizeof(lg.key), "key buffer too small");
+    cudaStreamCaptureStatus cap = cudaStreamCaptureStatusNone;
+    // (the legacy default stream cannot be captured: callers on it always get the eager loop)
+    const bool graph_ok = !lg.disabled && !h->prof.on && h->use_tensor && st != nullptr && st != cudaStreamLegacy &&
+                          st != cudaStreamPerThread && cudaStreamIsCapturing(st, &cap) == cudaSuccess && cap == cudaStreamCaptureStatusNone;
+    const bool same = graph_ok && lg.key_len == sizeof(key) && std::memcmp(lg.key, &key, sizeof(key)) == 0;
+    if (same && lg.exec) {
+        if (cudaGraphLaunch(lg.exec, st) == cudaSuccess) {
+            h->launches += lg.launches;
+            *cache_len_inout = lg.c_out;
+            return LOCOCO_OK;
         }
-        View qn = offset_tokens(Q, t0, e), kn = offset_tokens(K, t0, e), vn = offset_tokens(V, t0, e);
-        View on = offset_tokens(O, t0, e);
-        float* lse = sv ? reinterpret_cast<float*>(sv + 2 * snap_all) + t0 : nullptr;
-        s = step_impl(h, qn, dev(K_cache), dev(V_cache), c, kn, vn, b, on, lse, L, st);
-        if (s) return s;
-        c = c + b <= cfg.M ? c + b : cfg.M;
+        lg.disabled = true;
     }
+    if (graph_ok && !same) {
+        if (lg.exec) { cudaGraphExecDestroy(lg.exec); lg.exec = nullptr; }
+        std::memset(lg.key, 0, sizeof(lg.key));
+        std::memcpy(lg.key, &key, sizeof(key));
+        lg.key_len = sizeof(key);
+        lg.seen = 0;
+    }
+    const bool capture = graph_ok && same && !lg.disabled && lg.seen >= 1 && !lg.exec;
+    if (graph_ok) ++lg.seen;
+    if (capture && cudaStreamBeginCapture(st, cudaStreamCaptureModeThreadLocal) != cudaSuccess) {
+        lg.disabled = true;
+        cudaGetLastError();   // clear the refusal so that it is not mistaken for a launch failure
+        return lococo_process_sequence(h, Q, K, V, L, B, O, K_cache, V_cache, cache_len_inout, saved, stream);
+    }
+    const int64_t launches_before = h->launches;
+    s = run_chunk_loop(h, Q, K, V, L, B, O, K_cache, V_cache, &c, saved, st);
+    if (capture) {
+        cudaGraph_t graph = nullptr;
+        const bool ended = cudaStreamEndCapture(st, &graph) == cudaSuccess && graph != nullptr;
+        bool launched = false;
+        if (ended && s == LOCOCO_OK && cudaGraphInstantiate(&lg.exec, graph, 0) == cudaSuccess) {
+            lg.launches = h->launches - launches_before;
+            lg.c_out = c;
+            launched = cudaGraphLaunch(lg.exec, st) == cudaSuccess;
+        }
+        if (graph) cudaGraphDestroy(graph);
+        if (!launched) {
+            // nothing has run yet (the launches were only recorded): fall back to the eager loop
+            if (lg.exec) { cudaGraphExecDestroy(lg.exec); lg.exec = nullptr; }
+            lg.disabled = true;
+            cudaGetLastError();
+            h->launches = launches_before;
+            c = c_in;
+            s = run_chunk_loop(h, Q, K, V, L, B, O, K_cache, V_cache, &c, saved, st);
+        }
+    }
+    if (s) return s;
     *cache_len_inout = c;
     return LOCOCO_OK;
 }

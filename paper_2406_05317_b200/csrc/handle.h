@@ -32,6 +32,16 @@ struct lococo_handle {
     size_t off_status = 0, off_gpack = 0, off_bias = 0, off_s = 0, off_UK = 0, off_UV = 0, off_R = 0;
     size_t off_gimage = 0, off_part = 0, off_counter = 0;  // tensor-core path
     int64_t launches = 0;
+    // CUDA graph of the chunk loop for the most recent argument set of lococo_process_sequence
+    struct LoopGraph {
+        unsigned char key[256] = {};   // the call's arguments, byte for byte
+        size_t key_len = 0;
+        int seen = 0;                  // identical calls so far (the graph is captured on the second)
+        cudaGraphExec_t exec = nullptr;
+        int64_t launches = 0;          // kernels inside the graph
+        int c_out = 0;                 // cache length after the loop
+        bool disabled = false;         // a graph call failed once: stay eager
+    } loop_graph;
     lococo::Profiler prof;
 };
 
