@@ -676,7 +676,12 @@ size_t smem_bytes(int n_tile, int k, int stages) {
 }
 
 // Tile width and CTA count: fewest waves of 148 SMs, then least padded work.
-bool make_plan(int S, int k, int units, int slot_blocks, Plan* out) {
+// Cost model from measured CTA timelines (microseconds): a fixed part (set-up, key staging, partial
+// stores), and per position tile one ring stage per (tap, channel half) that takes the longer of the
+// weight copy (0.37) and its eight MMAs (N/2 cycles each), plus epilogue and blends. A stand-alone
+// launch is charged by waves of 148 SMs; CTAs that share a grid with attention CTAs (`fused`) are
+// charged by their total SM time, which favours wider tiles (fewer CTAs, overheads paid less often).
+bool make_plan(int S, int k, int halves, int units, int slot_blocks, bool fused, Plan* out) {
     double best = 1e30;
     const int cap = parts_cap(units, slot_blocks);
     for (int n_tile = 224; n_tile >= 64; n_tile -= 32) {
@@ -689,7 +694,9 @@ bool make_plan(int S, int k, int units, int slot_blocks, Plan* out) {
             const int parts_eff = (tiles + tpp - 1) / tpp;
             const long ctas = (long)units * slot_blocks * parts_eff;
             const long waves = (ctas + 147) / 148;
-            const double cost = (double)waves * tpp * (n_tile + 24) + (stages < 4 ? 1.0 : 0.0);
+            const double stage_us = std::max(0.37, n_tile * 0.5 * 8.0 / 1965.0);
+            const double cta_us = 4.0 + tpp * (k * halves * stage_us + 3.5);
+            const double cost = (fused ? ctas * cta_us / 148.0 + 0.5 * cta_us : waves * cta_us) + (stages < 4 ? 0.05 : 0.0);
             if (cost < best) {
                 best = cost;
                 *out = Plan{n_tile, tiles, parts_eff, tpp, stages, (n_tile + k - 1) | 1, smem_bytes(n_tile, k, stages)};
@@ -707,7 +714,7 @@ bool tensor_config_supported(const lococo_config* c) {
     if (c->dtype != LOCOCO_BF16 || c->head_dim != kD) return false;
     if (c->M % kSlots != 0) return false;
     Plan pl;
-    return make_plan(c->M + c->max_chunk, c->k, c->batch * c->heads, c->M / kSlots, &pl);
+    return make_plan(c->M + c->max_chunk, c->k, c->c_in / 128, c->batch * c->heads, c->M / kSlots, false, &pl);
 }
 
 void tensor_layout_workspace(lococo_handle* h, size_t* off) {
@@ -736,13 +743,13 @@ int tensor_pack_weights(lococo_handle* h, const void* G, cudaStream_t st) {
 
 bool tensor_compress_supported(const lococo_handle* h, const CompressParams& p) {
     Plan pl;
-    return h->use_tensor && p.S >= 1 && make_plan(p.S, p.k, p.units, p.M / kSlots, &pl);
+    return h->use_tensor && p.S >= 1 && make_plan(p.S, p.k, p.c_in / 128, p.units, p.M / kSlots, false, &pl);
 }
 
-static bool build_compress_params(lococo_handle* h, const CompressParams& p, TcCompressParams* out) {
+static bool build_compress_params(lococo_handle* h, const CompressParams& p, bool fused, TcCompressParams* out) {
     const int SB = p.M / kSlots;
     Plan pl;
-    if (!make_plan(p.S, p.k, p.units, SB, &pl)) return false;
+    if (!make_plan(p.S, p.k, p.c_in / 128, p.units, SB, fused, &pl)) return false;
     const int Smax = h->cfg.M + h->cfg.max_chunk;
     const int max_parts = std::min(parts_cap(h->units, SB), (Smax + 63) / 64);
     if (pl.parts > max_parts) return false;
@@ -777,7 +784,7 @@ static int finish_compress(const TcCompressParams& P, cudaStream_t st) {
 
 int tensor_compress(lococo_handle* h, const CompressParams& p, cudaStream_t st) {
     TcCompressParams P;
-    if (!build_compress_params(h, p, &P)) return -1;
+    if (!build_compress_params(h, p, false, &P)) return -1;
     static bool attr_set = false;
     if (!attr_set) {
         if (cudaFuncSetAttribute(compress_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxSmem) != cudaSuccess)
@@ -798,7 +805,7 @@ int tensor_compress(lococo_handle* h, const CompressParams& p, cudaStream_t st) 
 // Attention with the old cache and the cache update of one chunk in a single launch.
 int tensor_chunk_step(lococo_handle* h, const AttnParams& a, const CompressParams& p, cudaStream_t st) {
     TcStepParams P{};
-    if (!build_compress_params(h, p, &P.comp)) return -1;
+    if (!build_compress_params(h, p, true, &P.comp)) return -1;
     P.attn.base = a;
     P.attn.status = P.comp.status;
     static bool attr_set = false;
