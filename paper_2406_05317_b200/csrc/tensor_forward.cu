@@ -663,6 +663,7 @@ __global__ void __launch_bounds__(kAttnThreads, 1) chunk_step_tc_kernel(const __
 struct Plan {
     int n_tile, tiles, parts, tiles_per_part, stages, rows_pad;
     size_t smem;
+    double cta_us;   // estimated duration of one compress CTA
 };
 
 int parts_cap(int units, int slot_blocks) {
@@ -699,7 +700,7 @@ bool make_plan(int S, int k, int halves, int units, int slot_blocks, bool fused,
             const double cost = (fused ? ctas * cta_us / 148.0 + 0.5 * cta_us : waves * cta_us) + (stages < 4 ? 0.05 : 0.0);
             if (cost < best) {
                 best = cost;
-                *out = Plan{n_tile, tiles, parts_eff, tpp, stages, (n_tile + k - 1) | 1, smem_bytes(n_tile, k, stages)};
+                *out = Plan{n_tile, tiles, parts_eff, tpp, stages, (n_tile + k - 1) | 1, smem_bytes(n_tile, k, stages), cta_us};
             }
         }
     }
@@ -746,7 +747,8 @@ bool tensor_compress_supported(const lococo_handle* h, const CompressParams& p) 
     return h->use_tensor && p.S >= 1 && make_plan(p.S, p.k, p.c_in / 128, p.units, p.M / kSlots, false, &pl);
 }
 
-static bool build_compress_params(lococo_handle* h, const CompressParams& p, bool fused, TcCompressParams* out) {
+static bool build_compress_params(lococo_handle* h, const CompressParams& p, bool fused, TcCompressParams* out,
+                                  double* cta_us = nullptr) {
     const int SB = p.M / kSlots;
     Plan pl;
     if (!make_plan(p.S, p.k, p.c_in / 128, p.units, SB, fused, &pl)) return false;
@@ -763,6 +765,7 @@ static bool build_compress_params(lococo_handle* h, const CompressParams& p, boo
     P.n_tile = pl.n_tile; P.tiles = pl.tiles; P.parts = pl.parts; P.tiles_per_part = pl.tiles_per_part;
     P.halves = p.c_in / 128; P.stages = pl.stages; P.rows_pad = pl.rows_pad; P.slot_blocks = SB;
     *out = P;
+    if (cta_us) *cta_us = pl.cta_us;
     return true;
 }
 
@@ -805,7 +808,8 @@ int tensor_compress(lococo_handle* h, const CompressParams& p, cudaStream_t st) 
 // Attention with the old cache and the cache update of one chunk in a single launch.
 int tensor_chunk_step(lococo_handle* h, const AttnParams& a, const CompressParams& p, cudaStream_t st) {
     TcStepParams P{};
-    if (!build_compress_params(h, p, true, &P.comp)) return -1;
+    double comp_us = 0.0;
+    if (!build_compress_params(h, p, true, &P.comp, &comp_us)) return -1;
     P.attn.base = a;
     P.attn.status = P.comp.status;
     static bool attr_set = false;
@@ -816,7 +820,14 @@ int tensor_chunk_step(lococo_handle* h, const AttnParams& a, const CompressParam
     }
     P.qtiles = (a.b + 127) / 128;
     P.n_attn = P.qtiles * a.units;
-    P.n_attn_first = ((P.qtiles + 1) / 2) * a.units;
+    // longest first: the attention tiles estimated to outlast a compress CTA (7 us fixed + 2.4 us per
+    // key tile, from measured timelines), then the compress CTAs, then the remaining attention tiles
+    int longer = 0;
+    for (int t = P.qtiles - 1; t >= 0; --t) {
+        const int cols = a.c + std::min(a.b, (t + 1) * 128);
+        if (7.0 + 2.4 * ((cols + 127) / 128) > comp_us) ++longer; else break;
+    }
+    P.n_attn_first = longer * a.units;
     P.comp_per_unit = P.comp.parts * P.comp.slot_blocks;
     const int blocks = P.n_attn + a.units * P.comp_per_unit;
     prof_begin(p.prof, 2, st);
