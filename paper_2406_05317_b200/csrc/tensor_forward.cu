@@ -457,21 +457,26 @@ __device__ __forceinline__ void attention_body(const TcAttnParams& P, uint8_t* s
         }
         // from here on, per-thread group order: [K(t+1)] [V(t+1)] ...; a tile is announced to the MMA
         // issuer before this warp waits for any buffer that the issuer has to free
-        for (int jt = 1; jt + 1 < ntiles; ++jt) {
-            // tile jt is already announced; refill the buffers of tile jt-1 with tile jt+1. The key
-            // tile is announced as soon as it lands: the next S MMA needs it long before the value
-            // buffer is even free.
-            const int pb = (jt - 1) & 1, pph = ((jt - 1) >> 1) & 1;
-            mbar_wait(s_full(pb), pph, P.status, failed, 4);      // S(jt-1) has read the key buffer
-            load_tile(jt + 1, pb, 0, lw, kAttnLoaderWarps);
+        // Tile t (>= 2) goes into the buffers of tile t-2. Its keys are needed first (by S(t), while
+        // softmax(t-1) still runs), its values only by PV(t): the key copy is awaited and announced at
+        // once, the value copy is left in flight and announced in the next round, so one round costs one
+        // copy latency, not two. Every wait below is on MMAs whose inputs were announced in earlier rounds.
+        for (int t = 2; t < ntiles; ++t) {
+            const int b = t & 1, ph = ((t - 2) >> 1) & 1;
+            mbar_wait(s_full(b), ph, P.status, failed, 4);        // S(t-2) has read the key buffer
+            load_tile(t, b, 0, lw, kAttnLoaderWarps);
+            cp_async_wait_all();                                  // V(t-1) and K(t) have landed
+            fence_proxy_async();
+            if (t > 2) mbar_arrive(v_full((t - 1) & 1));
+            mbar_arrive(k_full(b));
+            mbar_wait(pv_done(b), ph, P.status, failed, 5);       // PV(t-2) has read the value buffer
+            load_tile(t, b, 1, lw, kAttnLoaderWarps);
+            commit();
+        }
+        if (ntiles > 2) {
             cp_async_wait_all();
             fence_proxy_async();
-            mbar_arrive(k_full(pb));
-            mbar_wait(pv_done(pb), pph, P.status, failed, 5);     // PV(jt-1) has read the value buffer
-            load_tile(jt + 1, pb, 1, lw, kAttnLoaderWarps);
-            cp_async_wait_all();
-            fence_proxy_async();
-            mbar_arrive(v_full(pb));
+            mbar_arrive(v_full((ntiles - 1) & 1));
         }
     } else if (tid == kMma) {
         // ---------------- MMA issuer: S(0), then per tile S(t) followed by PV(t-1)
