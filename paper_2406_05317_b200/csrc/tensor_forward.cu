@@ -27,7 +27,7 @@ constexpr int kSlots = 128;              // slots per CTA (MMA M)
 constexpr int kD = 128;                  // head dimension
 constexpr int kStageBytes = 32768;       // one tap x 128 channels x 128 slots, bf16
 constexpr int kThreads = 192;            // 4 loader/epilogue warps + MMA-issue warp + weight-producer warp
-constexpr int kMaxSmem = 232448;         // 227 KB
+constexpr int kMaxSmem = 232448 - 128;   // dynamic shared memory per CTA: 227 KB less the kernels' few static words
 constexpr uint32_t kTmemCols = 512;
 constexpr uint32_t kColUK = 256, kColUV = 384;
 
@@ -63,7 +63,10 @@ __global__ void pack_image_kernel(const __nv_bfloat16* __restrict__ G, __nv_bflo
 
 // Work of one CTA: tiles [part*tiles_per_part, ...) of slot block sb of unit u. Runs with any
 // block size that is a multiple of 32 and at least 192 (warps beyond the sixth only help staging).
-__device__ __forceinline__ void compress_body(const TcCompressParams& P, uint8_t* smem, int part, int sb, int u) {
+// `tmem`: base of 512 TMEM columns the CTA owns. `cache_cg`: read cache rows around L1 (set when the
+// cache was rewritten by other SMs earlier in the SAME kernel; L1 is coherent only across launches).
+__device__ __forceinline__ void compress_body(const TcCompressParams& P, uint8_t* smem, uint32_t tmem, bool cache_cg, int part,
+                                              int sb, int u) {
     const CompressParams& p = P.base;
     const int nthr16 = blockDim.x / 16;
     const int n = u / p.heads, h = u % p.heads;
@@ -92,15 +95,9 @@ __device__ __forceinline__ void compress_body(const TcCompressParams& P, uint8_t
         *failed = 0;
         fence_barrier_init();
     }
-    if (warp == 4) {
-        __syncwarp();
-        tmem_alloc(smem_u32(const_cast<uint32_t*>(tmem_slot)), kTmemCols);
-        tmem_relinquish();
-    }
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
-    const uint32_t tmem = *tmem_slot;
 
     const int set = p.weights_per_head ? h : 0;
     const __nv_bfloat16* gimg =
@@ -142,9 +139,11 @@ __device__ __forceinline__ void compress_body(const TcCompressParams& P, uint8_t
             for (int r = first >> 4; r < rows; r += step) {
                 const int j = j0 - pad + r;
                 const bool valid = j >= 0 && j < p.S;
-                const __nv_bfloat16* src = !valid ? safe : (j < xv_.c ? cbase + (int64_t)j * xv_.cache.st
-                                                                       : kbase + (int64_t)(j - xv_.c) * xv_.chunk.st);
-                cp_async16(d0 + r * 16, src, valid ? 16u : 0u);
+                const bool in_cache = valid && j < xv_.c;
+                const __nv_bfloat16* src = !valid ? safe : (in_cache ? cbase + (int64_t)j * xv_.cache.st
+                                                                     : kbase + (int64_t)(j - xv_.c) * xv_.chunk.st);
+                if (in_cache && cache_cg) cp_async16_cg(d0 + r * 16, src, 16u);
+                else cp_async16(d0 + r * 16, src, valid ? 16u : 0u);
             }
         };
         stage_tile(p.xk, zk, tid, nthr16);
@@ -264,15 +263,34 @@ __device__ __forceinline__ void compress_body(const TcCompressParams& P, uint8_t
     }
     tc_fence_before();
     __syncthreads();
-    if (warp == 4) {
-        __syncwarp();
-        tmem_dealloc(tmem, kTmemCols);
+    if (tid == 128) {
+        for (int s = 0; s < 2 * NS + 2; ++s) mbar_inval(bar_full + 8 * s);
     }
+}
+
+// The CTA's TMEM (all 512 columns; one CTA per SM) is allocated around the work, not inside it.
+__device__ __forceinline__ uint32_t cta_tmem_acquire(uint32_t* slot) {
+    if (threadIdx.x < 32) {
+        tmem_alloc(smem_u32(slot), kTmemCols);
+        tmem_relinquish();
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    return *reinterpret_cast<volatile uint32_t*>(slot);
+}
+__device__ __forceinline__ void cta_tmem_release(uint32_t tmem) {
+    tc_fence_before();
+    __syncthreads();
+    if (threadIdx.x < 32) tmem_dealloc(tmem, kTmemCols);
 }
 
 __global__ void __launch_bounds__(kThreads, 1) compress_tc_kernel(const __grid_constant__ TcCompressParams P) {
     extern __shared__ __align__(128) uint8_t smem[];
-    compress_body(P, smem, blockIdx.x, blockIdx.y, blockIdx.z);
+    __shared__ uint32_t tmem_slot;
+    const uint32_t tmem = cta_tmem_acquire(&tmem_slot);
+    compress_body(P, smem, tmem, false, blockIdx.x, blockIdx.y, blockIdx.z);
+    cta_tmem_release(tmem);
 }
 
 // cache = (sum of partial blends) / (sum of partial row sums + eps)   (Eq. 7 after Eq. 4-5)
@@ -342,7 +360,8 @@ struct TcAttnParams {
 };
 
 // Work of one CTA (exactly kAttnThreads threads): query tile qtile of unit u.
-__device__ __forceinline__ void attention_body(const TcAttnParams& P, uint8_t* smem, int qtile, int u) {
+// `tmem`, `cache_cg`: as for compress_body.
+__device__ __forceinline__ void attention_body(const TcAttnParams& P, uint8_t* smem, uint32_t tmem, bool cache_cg, int qtile, int u) {
     const AttnParams& p = P.base;
     const int n = u / p.heads, h = u % p.heads;
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -380,15 +399,9 @@ __device__ __forceinline__ void attention_body(const TcAttnParams& P, uint8_t* s
         *failed = 0;
         fence_barrier_init();
     }
-    if (warp == 8) {
-        __syncwarp();
-        tmem_alloc(smem_u32(const_cast<uint32_t*>(tmem_slot)), kAttnTmemCols);
-        tmem_relinquish();
-    }
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
-    const uint32_t tmem = *tmem_slot;
 
     const int last_row = min(r0 + 127, p.b - 1);
     const int ncols = p.c + last_row + 1;           // columns any query of this tile can see
@@ -398,13 +411,14 @@ __device__ __forceinline__ void attention_body(const TcAttnParams& P, uint8_t* s
     // per row (256 contiguous bytes in global memory), two rows per warp instruction. Rows at or
     // beyond `nrows` are zero-filled.
     const __nv_bfloat16* safe = unit_base<__nv_bfloat16>(p.q, n, h);
-    auto stage_rows = [&](uint32_t dst, const __nv_bfloat16* base, int64_t st, int nrows, int lw, int nw) {
+    auto stage_rows = [&](uint32_t dst, const __nv_bfloat16* base, int64_t st, int nrows, int lw, int nw, bool cg) {
         const int q = lane & 15;
         const uint32_t d0 = dst + q * kLboT;
         const __nv_bfloat16* b0 = base + q * 8;
         for (int r = 2 * lw + (lane >> 4); r < 128; r += 2 * nw) {
             const bool valid = r < nrows;
-            cp_async16(d0 + r * 16, valid ? b0 + (int64_t)r * st : safe, valid ? 16u : 0u);
+            if (cg) cp_async16_cg(d0 + r * 16, valid ? b0 + (int64_t)r * st : safe, valid ? 16u : 0u);
+            else cp_async16(d0 + r * 16, valid ? b0 + (int64_t)r * st : safe, valid ? 16u : 0u);
         }
     };
     // keys (which = 0) or values (1) of key tile jt: the part inside the cache, then the part inside the chunk
@@ -413,9 +427,9 @@ __device__ __forceinline__ void attention_body(const TcAttnParams& P, uint8_t* s
         const uint32_t dst = (which ? vs : ks) + buf * kTileBytes;
         const int jb = jt * 128;
         if (jb + 128 <= p.c) {
-            stage_rows(dst, unit_base<__nv_bfloat16>(x.cache, n, h) + (int64_t)jb * x.cache.st, x.cache.st, 128, lw, nw);
+            stage_rows(dst, unit_base<__nv_bfloat16>(x.cache, n, h) + (int64_t)jb * x.cache.st, x.cache.st, 128, lw, nw, cache_cg);
         } else if (jb >= p.c) {
-            stage_rows(dst, unit_base<__nv_bfloat16>(x.chunk, n, h) + (int64_t)(jb - p.c) * x.chunk.st, x.chunk.st, S - jb, lw, nw);
+            stage_rows(dst, unit_base<__nv_bfloat16>(x.chunk, n, h) + (int64_t)(jb - p.c) * x.chunk.st, x.chunk.st, S - jb, lw, nw, false);
         } else {
             // the tile straddles the end of the cache: row by row
             const int q = lane & 15;
@@ -425,14 +439,15 @@ __device__ __forceinline__ void attention_body(const TcAttnParams& P, uint8_t* s
                 const __nv_bfloat16* src = !valid ? safe
                     : j < p.c ? unit_base<__nv_bfloat16>(x.cache, n, h) + (int64_t)j * x.cache.st + q * 8
                               : unit_base<__nv_bfloat16>(x.chunk, n, h) + (int64_t)(j - p.c) * x.chunk.st + q * 8;
-                cp_async16(dst + q * kLboT + r * 16, src, valid ? 16u : 0u);
+                if (cache_cg && valid && j < p.c) cp_async16_cg(dst + q * kLboT + r * 16, src, 16u);
+                else cp_async16(dst + q * kLboT + r * 16, src, valid ? 16u : 0u);
             }
         }
     };
     // ---- prologue, all warps: Q and the first two key/value tiles
     {
         constexpr int nw = kAttnThreads / 32;
-        stage_rows(qs, safe + (int64_t)r0 * p.q.st, p.q.st, p.b - r0, warp, nw);
+        stage_rows(qs, safe + (int64_t)r0 * p.q.st, p.q.st, p.b - r0, warp, nw, false);
         load_tile(0, 0, 0, warp, nw);
         load_tile(0, 0, 1, warp, nw);
         if (ntiles > 1) {
@@ -625,15 +640,17 @@ __device__ __forceinline__ void attention_body(const TcAttnParams& P, uint8_t* s
     }
     tc_fence_before();
     __syncthreads();
-    if (warp == 8) {
-        __syncwarp();
-        tmem_dealloc(tmem, kAttnTmemCols);
+    if (tid == kMma) {
+        for (int s = 0; s < 12; ++s) mbar_inval(bar0 + 8 * s);
     }
 }
 
 __global__ void __launch_bounds__(kAttnThreads, 1) attention_tc_kernel(const __grid_constant__ TcAttnParams P) {
     extern __shared__ __align__(128) uint8_t smem[];
-    attention_body(P, smem, blockIdx.x, blockIdx.y);
+    __shared__ uint32_t tmem_slot;
+    const uint32_t tmem = cta_tmem_acquire(&tmem_slot);
+    attention_body(P, smem, tmem, false, blockIdx.x, blockIdx.y);
+    cta_tmem_release(tmem);
 }
 
 // ------------------------------------------------------------------ one chunk step, one launch
@@ -648,21 +665,28 @@ struct TcStepParams {
     int qtiles, n_attn_first, n_attn, comp_per_unit;   // comp_per_unit = parts * slot_blocks
 };
 
-__global__ void __launch_bounds__(kAttnThreads, 1) chunk_step_tc_kernel(const __grid_constant__ TcStepParams P) {
-    extern __shared__ __align__(128) uint8_t smem[];
+// Work item `idx` of one chunk step, in the order above.
+__device__ __forceinline__ void step_item(const TcStepParams& P, uint8_t* smem, uint32_t tmem, bool cache_cg, int idx) {
     const int units = P.attn.base.units;
-    int idx = blockIdx.x;
     const int n_comp = units * P.comp_per_unit;
     if (idx < P.n_attn_first) {
-        attention_body(P.attn, smem, P.qtiles - 1 - idx / units, idx % units);
+        attention_body(P.attn, smem, tmem, cache_cg, P.qtiles - 1 - idx / units, idx % units);
     } else if (idx < P.n_attn_first + n_comp) {
         idx -= P.n_attn_first;
         const int u = idx / P.comp_per_unit, rem = idx % P.comp_per_unit;
-        compress_body(P.comp, smem, rem % P.comp.parts, rem / P.comp.parts, u);
+        compress_body(P.comp, smem, tmem, cache_cg, rem % P.comp.parts, rem / P.comp.parts, u);
     } else {
         idx -= n_comp;
-        attention_body(P.attn, smem, P.qtiles - 1 - idx / units, idx % units);
+        attention_body(P.attn, smem, tmem, cache_cg, P.qtiles - 1 - idx / units, idx % units);
     }
+}
+
+__global__ void __launch_bounds__(kAttnThreads, 1) chunk_step_tc_kernel(const __grid_constant__ TcStepParams P) {
+    extern __shared__ __align__(128) uint8_t smem[];
+    __shared__ uint32_t tmem_slot;
+    const uint32_t tmem = cta_tmem_acquire(&tmem_slot);
+    step_item(P, smem, tmem, false, blockIdx.x);
+    cta_tmem_release(tmem);
 }
 
 struct Plan {
