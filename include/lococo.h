@@ -50,8 +50,16 @@ typedef enum {
 typedef enum { LOCOCO_F32 = 0, LOCOCO_BF16 = 1 } lococo_dtype;
 
 /* Which kernels serve a call. AUTO: tensor-core (tcgen05) kernels where the shape and
- * dtype allow, CUDA-core kernels otherwise. */
-typedef enum { LOCOCO_PATH_AUTO = 0, LOCOCO_PATH_SIMT = 1, LOCOCO_PATH_TENSOR = 2 } lococo_path;
+ * dtype allow, CUDA-core kernels otherwise. TENSOR_PERSISTENT: the tensor-core kernels, with
+ * the compress steps of lococo_process_sequence (Algorithm 2, loop) run by ONE cooperative
+ * launch whose CTAs stay resident and meet at a device-wide barrier between the steps,
+ * instead of one launch per chunk; results are identical bit for bit. */
+typedef enum {
+    LOCOCO_PATH_AUTO = 0,
+    LOCOCO_PATH_SIMT = 1,
+    LOCOCO_PATH_TENSOR = 2,
+    LOCOCO_PATH_TENSOR_PERSISTENT = 3
+} lococo_path;
 
 typedef struct {
     int32_t batch;            /* sequences processed together */
@@ -224,7 +232,8 @@ lococo_status lococo_launch_count(const lococo_handle* handle, int64_t* out);
  * stream around each launch.  kind 0: the kernel that evaluates Eq. 6 (the conv
  * contraction, with whatever is fused into it); kind 1: the chunk-attention kernel (Eq. 1);
  * kind 2: the single launch lococo_process_sequence uses per chunk on the tensor-core path, which
- * holds both of the above (Step 3 and Steps 4-5 of Algorithm 2 are independent of each other).
+ * holds both of the above (Step 3 and Steps 4-5 of Algorithm 2 are independent of each other);
+ * kind 3: the persistent launch that runs all consecutive compress steps of a lococo_process_sequence call.
  * lococo_profile_enable(h, 1) starts a fresh recording, (h, 0) stops it;
  * lococo_profile_read waits for the recorded events and returns the summed duration in
  * milliseconds and the number of launches of that kind since the recording started.

@@ -19,7 +19,7 @@ _lib = ctypes.CDLL(str(_LIB_PATH))
 
 OK, ERR_INVALID_ARG, ERR_UNSUPPORTED_SHAPE, ERR_WORKSPACE, ERR_CUDA, ERR_TIMEOUT = range(6)
 F32, BF16 = 0, 1
-PATH_AUTO, PATH_SIMT, PATH_TENSOR = 0, 1, 2
+PATH_AUTO, PATH_SIMT, PATH_TENSOR, PATH_TENSOR_PERSISTENT = 0, 1, 2, 3
 
 
 class Config(ctypes.Structure):

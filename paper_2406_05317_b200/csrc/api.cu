@@ -231,7 +231,7 @@ lococo_status lococo_create(const lococo_config* c, lococo_handle** out) {
     if (c->dtype != LOCOCO_F32 && c->dtype != LOCOCO_BF16) return LOCOCO_ERR_INVALID_ARG;
     if (c->c_in != c->head_dim && c->c_in != 2 * c->head_dim) return LOCOCO_ERR_INVALID_ARG;
     if (c->weights_per_head != 0 && c->weights_per_head != 1) return LOCOCO_ERR_INVALID_ARG;
-    if (c->path < LOCOCO_PATH_AUTO || c->path > LOCOCO_PATH_TENSOR) return LOCOCO_ERR_INVALID_ARG;
+    if (c->path < LOCOCO_PATH_AUTO || c->path > LOCOCO_PATH_TENSOR_PERSISTENT) return LOCOCO_ERR_INVALID_ARG;
     if (!(c->norm_eps >= 0.f) || !(c->softmax_scale >= 0.f)) return LOCOCO_ERR_INVALID_ARG;
     if (c->head_dim != 64 && c->head_dim != 128) return LOCOCO_ERR_UNSUPPORTED_SHAPE;
     if (c->k > 63) return LOCOCO_ERR_UNSUPPORTED_SHAPE;
@@ -244,11 +244,12 @@ lococo_status lococo_create(const lococo_config* c, lococo_handle** out) {
     h->elt = c->dtype == LOCOCO_F32 ? 4 : 2;
     h->scale = c->softmax_scale > 0.f ? c->softmax_scale : 1.0f / std::sqrt((float)c->head_dim);
     const bool tensor_ok = tensor_config_supported(c);
-    if (c->path == LOCOCO_PATH_TENSOR && !tensor_ok) {
+    if (c->path >= LOCOCO_PATH_TENSOR && !tensor_ok) {
         delete h;
         return LOCOCO_ERR_UNSUPPORTED_SHAPE;
     }
     h->use_tensor = tensor_ok && c->path != LOCOCO_PATH_SIMT;
+    h->persistent_loop = c->path == LOCOCO_PATH_TENSOR_PERSISTENT;
     layout_workspace(h);
     *out = h;
     return LOCOCO_OK;
@@ -258,6 +259,7 @@ lococo_status lococo_destroy(lococo_handle* h) {
     if (!h) return LOCOCO_ERR_INVALID_ARG;
     h->prof.release();
     if (h->loop_graph.exec) cudaGraphExecDestroy(h->loop_graph.exec);
+    tensor_sequence_release(h);
     delete h;
     return LOCOCO_OK;
 }
@@ -356,6 +358,7 @@ lococo_status run_chunk_loop(lococo_handle* h, lococo_tensor Q, lococo_tensor K,
     const lococo_config& cfg = h->cfg;
     const size_t e = h->elt;
     int c = *c_inout;
+    h->seq_count = 0;   // nothing is left queued from a call that failed half-way
     const int n_chunks = (L + B - 1) / B;
     const size_t snap_step = (size_t)h->units * cfg.M * cfg.head_dim * e;
     const size_t snap_all = align_up((size_t)n_chunks * snap_step, 256);
@@ -373,10 +376,24 @@ lococo_status run_chunk_loop(lococo_handle* h, lococo_tensor Q, lococo_tensor K,
         View qn = offset_tokens(Q, t0, e), kn = offset_tokens(K, t0, e), vn = offset_tokens(V, t0, e);
         View on = offset_tokens(O, t0, e);
         float* lse = sv ? reinterpret_cast<float*>(sv + 2 * snap_all) + t0 : nullptr;
-        lococo_status s = step_impl(h, qn, dev(K_cache), dev(V_cache), c, kn, vn, b, on, lse, L, st);
-        if (s) return s;
+        // on request, consecutive compress steps are queued for ONE persistent launch
+        // (not while snapshots for a backward pass are wanted: they are taken between the steps)
+        bool queued = false;
+        if (h->persistent_loop && !sv && c + b > cfg.M) {
+            const AttnParams a = make_attn_params(h, qn, dev(K_cache), dev(V_cache), c, kn, vn, b, on, nullptr, L);
+            const CompressParams p = make_compress_params(h, dev(K_cache), dev(V_cache), c, kn, vn, b, dev(K_cache), dev(V_cache), nullptr);
+            queued = tensor_attention_supported(h, a) && tensor_compress_supported(h, p) && tensor_sequence_add(h, a, p, st);
+        }
+        if (!queued) {
+            lococo_status s = count(h, tensor_sequence_launch(h, st, h->prof.on ? &h->prof : nullptr));   // flush what is queued, in order
+            if (s) return s;
+            s = step_impl(h, qn, dev(K_cache), dev(V_cache), c, kn, vn, b, on, lse, L, st);
+            if (s) return s;
+        }
         c = c + b <= cfg.M ? c + b : cfg.M;
     }
+    lococo_status s = count(h, tensor_sequence_launch(h, st, h->prof.on ? &h->prof : nullptr));
+    if (s) return s;
     *c_inout = c;
     return LOCOCO_OK;
 }

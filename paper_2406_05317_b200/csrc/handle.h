@@ -7,7 +7,7 @@
 
 namespace lococo {
 // Optional CUDA-event timing of individual kernel classes, on the launching stream.
-enum ProfKind { PROF_CONV = 0, PROF_ATTENTION = 1, PROF_STEP = 2, PROF_KINDS = 3 };
+enum ProfKind { PROF_CONV = 0, PROF_ATTENTION = 1, PROF_STEP = 2, PROF_SEQUENCE = 3, PROF_KINDS = 4 };
 struct Profiler {
     struct Rec { cudaEvent_t a, b; int kind; };
     bool on = false;
@@ -25,12 +25,19 @@ struct lococo_handle {
     size_t elt = 0;         // bytes per stored element
     float scale = 0.f;      // softmax scale in effect
     bool use_tensor = false;
+    bool persistent_loop = false;   // chunk loop as one cooperative launch (LOCOCO_PATH_TENSOR_PERSISTENT)
     bool weights_set = false;
     bool has_bias = false;
     char* ws = nullptr;     // caller-owned device workspace
     size_t ws_need = 0;
     size_t off_status = 0, off_gpack = 0, off_bias = 0, off_s = 0, off_UK = 0, off_UV = 0, off_R = 0;
-    size_t off_gimage = 0, off_part = 0, off_counter = 0;  // tensor-core path
+    size_t off_gimage = 0, off_part = 0, off_steps = 0, off_sync = 0;  // tensor-core path
+    // persistent chunk loop: step descriptors staged in pinned host memory (a small ring, one slot per call)
+    static constexpr int kSeqSlots = 4;
+    unsigned char* seq_host = nullptr;
+    cudaEvent_t seq_event[kSeqSlots] = {};
+    int seq_slot = 0, seq_count = 0;
+    int coop_grid = 0;      // 0: not probed yet, -1: persistent kernel unavailable, > 0: its grid size
     int64_t launches = 0;
     // CUDA graph of the chunk loop for the most recent argument set of lococo_process_sequence
     struct LoopGraph {
@@ -56,5 +63,9 @@ int tensor_compress(lococo_handle* h, const CompressParams& p, cudaStream_t st);
 bool tensor_attention_supported(const lococo_handle* h, const AttnParams& p);
 int tensor_attention(lococo_handle* h, const AttnParams& p, cudaStream_t st);
 int tensor_chunk_step(lococo_handle* h, const AttnParams& a, const CompressParams& p, cudaStream_t st);
+// Persistent chunk loop: queue consecutive compress steps, then run them all in one cooperative launch.
+bool tensor_sequence_add(lococo_handle* h, const AttnParams& a, const CompressParams& p, cudaStream_t st);
+int tensor_sequence_launch(lococo_handle* h, cudaStream_t st, void* prof);
+void tensor_sequence_release(lococo_handle* h);
 
 }  // namespace lococo

@@ -296,40 +296,50 @@ __global__ void __launch_bounds__(kThreads, 1) compress_tc_kernel(const __grid_c
 // cache = (sum of partial blends) / (sum of partial row sums + eps)   (Eq. 7 after Eq. 4-5)
 // One block per 32 slots x 32 channels: the partials are channel-major (read along slots),
 // the cache is slot-major (written along channels); the tile is transposed in shared memory.
-__global__ void __launch_bounds__(256) finalize_parts_kernel(TcCompressParams P) {
+// Runs with at least 256 threads; threads beyond the first 256 only take part in the barriers.
+// Partials are read around L1 (__ldcg): in the persistent kernel other SMs wrote them moments ago.
+__device__ __forceinline__ void finalize_tile(const TcCompressParams& P, float (*tk)[33], float (*tv)[33], float* inv_s,
+                                              int bx, int by, int u) {
     const CompressParams& p = P.base;
-    __shared__ float tk[32][33], tv[32][33], inv_s[32];
-    const int u = blockIdx.z, n = u / p.heads, h = u % p.heads;
-    const int i0 = blockIdx.x * 32, c0 = blockIdx.y * 32;   // slot tile, channel tile
+    const int n = u / p.heads, h = u % p.heads;
+    const int i0 = bx * 32, c0 = by * 32;   // slot tile, channel tile
     const int sb = i0 / kSlots, il0 = i0 % kSlots;
     const int64_t base = ((int64_t)u * P.slot_blocks + sb) * P.parts;
     const int tx = threadIdx.x % 32, ty = threadIdx.x / 32;
+    __syncthreads();                            // the tile buffers may still be read by the previous tile
     if (ty == 0) {
         float s = 0.f;
-        for (int pt = 0; pt < P.parts; ++pt) s += P.part_s[(base + pt) * kSlots + il0 + tx];
+        for (int pt = 0; pt < P.parts; ++pt) s += __ldcg(P.part_s + (base + pt) * kSlots + il0 + tx);
         s += p.eps;
         inv_s[tx] = 1.f / s;
         if (c0 == 0) p.s[(int64_t)u * p.M + i0 + tx] = s;
     }
-    for (int cc = ty; cc < 32; cc += 8) {      // tx runs along slots: 128-byte coalesced reads
-        float uk = 0.f, uv = 0.f;
-        for (int pt = 0; pt < P.parts; ++pt) {
-            uk += P.part_U[((base + pt) * 2 + 0) * (kSlots * kD) + (c0 + cc) * kSlots + il0 + tx];
-            uv += P.part_U[((base + pt) * 2 + 1) * (kSlots * kD) + (c0 + cc) * kSlots + il0 + tx];
+    if (ty < 8) {
+        for (int cc = ty; cc < 32; cc += 8) {      // tx runs along slots: 128-byte coalesced reads
+            float uk = 0.f, uv = 0.f;
+            for (int pt = 0; pt < P.parts; ++pt) {
+                uk += __ldcg(P.part_U + ((base + pt) * 2 + 0) * (kSlots * kD) + (c0 + cc) * kSlots + il0 + tx);
+                uv += __ldcg(P.part_U + ((base + pt) * 2 + 1) * (kSlots * kD) + (c0 + cc) * kSlots + il0 + tx);
+            }
+            tk[cc][tx] = uk;
+            tv[cc][tx] = uv;
         }
-        tk[cc][tx] = uk;
-        tv[cc][tx] = uv;
     }
     __syncthreads();
-    for (int ii = ty; ii < 32; ii += 8) {      // tx runs along channels: coalesced writes
-        const float inv = inv_s[ii];
-        const int64_t row = (int64_t)(i0 + ii);
-        unit_base_mut<__nv_bfloat16>(p.k_out, n, h)[row * p.k_out.st + c0 + tx] = __float2bfloat16_rn(tk[tx][ii] * inv);
-        unit_base_mut<__nv_bfloat16>(p.v_out, n, h)[row * p.v_out.st + c0 + tx] = __float2bfloat16_rn(tv[tx][ii] * inv);
+    if (ty < 8) {
+        for (int ii = ty; ii < 32; ii += 8) {      // tx runs along channels: coalesced writes
+            const float inv = inv_s[ii];
+            const int64_t row = (int64_t)(i0 + ii);
+            unit_base_mut<__nv_bfloat16>(p.k_out, n, h)[row * p.k_out.st + c0 + tx] = __float2bfloat16_rn(tk[tx][ii] * inv);
+            unit_base_mut<__nv_bfloat16>(p.v_out, n, h)[row * p.v_out.st + c0 + tx] = __float2bfloat16_rn(tv[tx][ii] * inv);
+        }
     }
 }
 
-
+__global__ void __launch_bounds__(256) finalize_parts_kernel(TcCompressParams P) {
+    __shared__ float tk[32][33], tv[32][33], inv_s[32];
+    finalize_tile(P, tk, tv, inv_s, blockIdx.x, blockIdx.y, blockIdx.z);
+}
 
 // ------------------------------------------------------------------ Eq. 1, chunk form
 // One CTA = 128 queries of one unit, pipelined over 128-key tiles of [cache; chunk] with three
@@ -689,6 +699,78 @@ __global__ void __launch_bounds__(kAttnThreads, 1) chunk_step_tc_kernel(const __
     cta_tmem_release(tmem);
 }
 
+// ------------------------------------------------------------------ the whole chunk loop, one launch
+// A persistent cooperative grid (one CTA per SM) walks the steps of Algorithm 2. Per step the CTAs pull
+// the attention and compress work items of chunk_step_tc_kernel from a counter, meet at a grid barrier,
+// share the finalize tiles (new cache = partial blends / row sums), meet again, and go on to the next
+// chunk: no launch and no TMEM/set-up cost between chunks. The cache stays where it is (2 MB, L2); the
+// only care it needs is that reads of it go around L1 from the second step on, because another SM
+// rewrote it inside this same kernel.
+struct TcSeqParams {
+    const TcStepParams* steps;   // device
+    int n_steps;
+    int* work;                   // [n_steps] work-item counters, zeroed before the launch
+    int* barrier;                // one arrival counter, zeroed before the launch
+    int* status;
+};
+
+// Bounded: a CTA that waits too long records code 20 and goes on, so the kernel still terminates.
+__device__ __forceinline__ void grid_barrier(int* counter, int target, int* status) {
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        __threadfence();
+        atomicAdd(counter, 1);
+        bool ok = false;
+        for (uint32_t i = 0; i < (1u << 22); ++i) {
+            int seen;
+            asm volatile("ld.acquire.gpu.global.s32 %0, [%1];" : "=r"(seen) : "l"(counter) : "memory");
+            if (seen >= target) { ok = true; break; }
+            __nanosleep(64);
+        }
+        if (!ok) atomicCAS(status, 0, 20);
+        __threadfence();
+    }
+    __syncthreads();
+}
+
+__global__ void __launch_bounds__(kAttnThreads, 1) sequence_tc_kernel(const __grid_constant__ TcSeqParams Q) {
+    extern __shared__ __align__(128) uint8_t smem[];
+    __shared__ uint32_t tmem_slot;
+    __shared__ int item_s;
+    const uint32_t tmem = cta_tmem_acquire(&tmem_slot);
+    int arrivals = 0;
+    for (int n = 0; n < Q.n_steps; ++n) {
+        // a thread-private copy: parameters read through a global pointer cannot be kept in registers
+        // across the bodies' stores, and the bodies read them inside their hot loops
+        const TcStepParams P = Q.steps[n];
+        const CompressParams& cp = P.comp.base;
+        const bool cache_cg = n > 0;
+        const int total = P.n_attn + cp.units * P.comp_per_unit;
+        while (true) {
+            if (threadIdx.x == 0) item_s = atomicAdd(Q.work + n, 1);
+            __syncthreads();
+            const int item = item_s;
+            __syncthreads();
+            if (item >= total) break;
+            step_item(P, smem, tmem, cache_cg, item);
+        }
+        arrivals += gridDim.x;
+        grid_barrier(Q.barrier, arrivals, Q.status);
+        // finalize tiles (32 slots x 32 channels), shared statically; the staging memory is free now
+        float (*tk)[33] = reinterpret_cast<float (*)[33]>(smem);
+        float (*tv)[33] = tk + 32;
+        float* inv_s = reinterpret_cast<float*>(tv + 32);
+        const int tx_n = cp.M / 32, ty_n = kD / 32, per_unit = tx_n * ty_n;
+        for (int t = blockIdx.x; t < per_unit * cp.units; t += gridDim.x)
+            finalize_tile(P.comp, tk, tv, inv_s, (t % per_unit) % tx_n, (t % per_unit) / tx_n, t / per_unit);
+        arrivals += gridDim.x;
+        grid_barrier(Q.barrier, arrivals, Q.status);
+    }
+    cta_tmem_release(tmem);
+}
+
+constexpr int kMaxSeqSteps = 256;   // steps one persistent launch can hold
+
 struct Plan {
     int n_tile, tiles, parts, tiles_per_part, stages, rows_pad;
     size_t smem;
@@ -759,6 +841,10 @@ void tensor_layout_workspace(lococo_handle* h, size_t* off) {
     *off = align(*off + sets * (size_t)c.M * c.c_in * c.k * 2);
     h->off_part = *off;
     *off = align(*off + (size_t)h->units * SB * max_parts * (2 * kSlots * kD + kSlots) * sizeof(float));
+    h->off_steps = *off;
+    *off = align(*off + (size_t)kMaxSeqSteps * sizeof(TcStepParams));
+    h->off_sync = *off;
+    *off = align(*off + (size_t)(kMaxSeqSteps + 64) * sizeof(int));
 }
 
 int tensor_pack_weights(lococo_handle* h, const void* G, cudaStream_t st) {
@@ -834,19 +920,12 @@ int tensor_compress(lococo_handle* h, const CompressParams& p, cudaStream_t st) 
     return r < 0 ? -1 : 1 + r;
 }
 
-// Attention with the old cache and the cache update of one chunk in a single launch.
-int tensor_chunk_step(lococo_handle* h, const AttnParams& a, const CompressParams& p, cudaStream_t st) {
+static bool build_step_params(lococo_handle* h, const AttnParams& a, const CompressParams& p, TcStepParams* out) {
     TcStepParams P{};
     double comp_us = 0.0;
-    if (!build_compress_params(h, p, true, &P.comp, &comp_us)) return -1;
+    if (!build_compress_params(h, p, true, &P.comp, &comp_us)) return false;
     P.attn.base = a;
     P.attn.status = P.comp.status;
-    static bool attr_set = false;
-    if (!attr_set) {
-        if (cudaFuncSetAttribute(chunk_step_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxSmem) != cudaSuccess)
-            return -1;
-        attr_set = true;
-    }
     P.qtiles = (a.b + 127) / 128;
     P.n_attn = P.qtiles * a.units;
     // longest first: the attention tiles estimated to outlast a compress CTA (7 us fixed + 2.4 us per
@@ -858,6 +937,20 @@ int tensor_chunk_step(lococo_handle* h, const AttnParams& a, const CompressParam
     }
     P.n_attn_first = longer * a.units;
     P.comp_per_unit = P.comp.parts * P.comp.slot_blocks;
+    *out = P;
+    return true;
+}
+
+// Attention with the old cache and the cache update of one chunk in a single launch.
+int tensor_chunk_step(lococo_handle* h, const AttnParams& a, const CompressParams& p, cudaStream_t st) {
+    TcStepParams P;
+    if (!build_step_params(h, a, p, &P)) return -1;
+    static bool attr_set = false;
+    if (!attr_set) {
+        if (cudaFuncSetAttribute(chunk_step_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxSmem) != cudaSuccess)
+            return -1;
+        attr_set = true;
+    }
     const int blocks = P.n_attn + a.units * P.comp_per_unit;
     prof_begin(p.prof, 2, st);
     chunk_step_tc_kernel<<<blocks, kAttnThreads, kMaxSmem, st>>>(P);
@@ -866,6 +959,90 @@ int tensor_chunk_step(lococo_handle* h, const AttnParams& a, const CompressParam
     if (!ok) return -1;
     const int r = finish_compress(P.comp, st);
     return r < 0 ? -1 : 1 + r;
+}
+
+// ---- persistent chunk loop
+static bool sequence_available(lococo_handle* h) {
+    if (h->coop_grid == 0) {
+        h->coop_grid = -1;
+        int dev = 0, coop = 0, sms = 0, per_sm = 0;
+        if (cudaGetDevice(&dev) != cudaSuccess) return false;
+        cudaDeviceGetAttribute(&coop, cudaDevAttrCooperativeLaunch, dev);
+        cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+        if (!coop || sms < 1) return false;
+        if (cudaFuncSetAttribute(sequence_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxSmem) != cudaSuccess ||
+            cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, sequence_tc_kernel, kAttnThreads, kMaxSmem) != cudaSuccess ||
+            per_sm < 1) {
+            cudaGetLastError();
+            return false;
+        }
+        if (cudaHostAlloc(reinterpret_cast<void**>(&h->seq_host),
+                          (size_t)lococo_handle::kSeqSlots * kMaxSeqSteps * sizeof(TcStepParams), cudaHostAllocDefault) != cudaSuccess) {
+            cudaGetLastError();
+            h->seq_host = nullptr;
+            return false;
+        }
+        h->coop_grid = sms * per_sm;
+    }
+    return h->coop_grid > 0;
+}
+
+bool tensor_sequence_add(lococo_handle* h, const AttnParams& a, const CompressParams& p, cudaStream_t st) {
+    if (!sequence_available(h) || h->seq_count >= kMaxSeqSteps) return false;
+    TcStepParams P;
+    if (!build_step_params(h, a, p, &P)) return false;
+    if (h->seq_count == 0) {
+        // take the next host slot; make sure the copy that last read it has been carried out
+        h->seq_slot = (h->seq_slot + 1) % lococo_handle::kSeqSlots;
+        cudaStreamCaptureStatus cap = cudaStreamCaptureStatusNone;
+        cudaStreamIsCapturing(st, &cap);
+        if (cap == cudaStreamCaptureStatusNone && h->seq_event[h->seq_slot]) cudaEventSynchronize(h->seq_event[h->seq_slot]);
+    }
+    TcStepParams* slot = reinterpret_cast<TcStepParams*>(h->seq_host) + (size_t)h->seq_slot * kMaxSeqSteps;
+    slot[h->seq_count++] = P;
+    return true;
+}
+
+int tensor_sequence_launch(lococo_handle* h, cudaStream_t st, void* prof) {
+    const int n = h->seq_count;
+    h->seq_count = 0;
+    if (n == 0) return 0;
+    const TcStepParams* slot = reinterpret_cast<const TcStepParams*>(h->seq_host) + (size_t)h->seq_slot * kMaxSeqSteps;
+    TcSeqParams Q{};
+    Q.steps = reinterpret_cast<const TcStepParams*>(h->ws + h->off_steps);
+    Q.n_steps = n;
+    Q.work = reinterpret_cast<int*>(h->ws + h->off_sync);
+    Q.barrier = Q.work + kMaxSeqSteps;
+    Q.status = reinterpret_cast<int*>(h->ws + h->off_status);
+    if (cudaMemcpyAsync(h->ws + h->off_steps, slot, (size_t)n * sizeof(TcStepParams), cudaMemcpyHostToDevice, st) != cudaSuccess ||
+        cudaMemsetAsync(h->ws + h->off_sync, 0, (size_t)(kMaxSeqSteps + 64) * sizeof(int), st) != cudaSuccess)
+        return -1;
+    cudaStreamCaptureStatus cap = cudaStreamCaptureStatusNone;
+    cudaStreamIsCapturing(st, &cap);
+    if (cap == cudaStreamCaptureStatusNone) {
+        if (!h->seq_event[h->seq_slot] && cudaEventCreateWithFlags(&h->seq_event[h->seq_slot], cudaEventDisableTiming) != cudaSuccess)
+            return -1;
+        cudaEventRecord(h->seq_event[h->seq_slot], st);
+    }
+    void* args[] = {&Q};
+    prof_begin(prof, 3, st);
+    const cudaError_t e = cudaLaunchCooperativeKernel(reinterpret_cast<void*>(sequence_tc_kernel), dim3(h->coop_grid),
+                                                      dim3(kAttnThreads), args, kMaxSmem, st);
+    prof_end(prof, st);
+    if (e != cudaSuccess) {
+        cudaGetLastError();
+        return -1;
+    }
+    return 1;
+}
+
+void tensor_sequence_release(lococo_handle* h) {
+    if (h->seq_host) cudaFreeHost(h->seq_host);
+    h->seq_host = nullptr;
+    for (auto& e : h->seq_event) {
+        if (e) cudaEventDestroy(e);
+        e = nullptr;
+    }
 }
 
 bool tensor_attention_supported(const lococo_handle* h, const AttnParams& p) {

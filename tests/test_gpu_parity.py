@@ -302,3 +302,24 @@ def test_repeated_identical_calls_replay_the_same_loop(api):
     torch.cuda.synchronize()
     assert torch.equal(O, O2) and torch.equal(Kc, Kc2) and torch.equal(Vc, Vc2)
     assert ctx.device_status() == api.OK
+
+
+def test_persistent_loop_equals_stepwise_launches(api):
+    # PATH_TENSOR_PERSISTENT runs the compress steps of a call inside one cooperative kernel; the
+    # default tensor-core path launches every step: same CTA bodies, same bits, fewer launches
+    w = wl.CONFIGS["cfg3"].slice(batch=2, heads=4, L=1024)     # 2 fill steps, then 14 compress steps
+    Q, K, V = (to_device(x, w.dtype) for x in wl.make_qkv(w))
+    res = []
+    for path in (api.PATH_TENSOR_PERSISTENT, api.PATH_TENSOR):
+        ctx, G, _ = make_ctx(api, w, path=path)
+        O = torch.empty_like(Q)
+        Kc = torch.zeros(w.batch, w.heads, w.M, w.d, dtype=Q.dtype, device="cuda")
+        Vc = torch.zeros_like(Kc)
+        before = ctx.launch_count()
+        c = ctx.process_sequence(Q, K, V, w.B, O, Kc, Vc, 0)
+        torch.cuda.synchronize()
+        assert ctx.device_status() == api.OK
+        res.append((O, Kc, Vc, c, ctx.launch_count() - before))
+    assert res[0][3] == res[1][3] == w.M
+    assert torch.equal(res[0][0], res[1][0]) and torch.equal(res[0][1], res[1][1]) and torch.equal(res[0][2], res[1][2])
+    assert res[0][4] < res[1][4]        # one persistent launch instead of two per step
