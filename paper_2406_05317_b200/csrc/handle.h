@@ -37,7 +37,8 @@ struct lococo_handle {
     unsigned char* seq_host = nullptr;
     cudaEvent_t seq_event[kSeqSlots] = {};
     int seq_slot = 0, seq_count = 0;
-    int coop_grid = 0;      // 0: not probed yet, -1: persistent kernel unavailable, > 0: its grid size
+    int seq_items = 0, seq_per_unit = 0;   // items queued so far: all units, one unit
+    int coop_grid = 0;      // 0: not probed yet, -1: persistent kernel unavailable, > 0: CTAs that fit the device
     int64_t launches = 0;
     // CUDA graph of the chunk loop for the most recent argument set of lococo_process_sequence
     struct LoopGraph {

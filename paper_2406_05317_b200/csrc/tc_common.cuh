@@ -70,6 +70,20 @@ __device__ __forceinline__ void bulk_load(uint32_t dst_smem, const void* src, ui
                  "l"(src), "r"(bytes), "r"(bar)
                  : "memory");
 }
+// Tiled copy global -> shared through the tensor copy engine, rank 4, one box of the tensor map at
+// coordinates (x, y, z, w); x times the element size must be a multiple of 16 bytes. Elements outside
+// the tensor arrive as zeros. Completion is signalled on the mbarrier as transaction bytes.
+__device__ __forceinline__ void tma_load_4d(uint32_t dst_smem, const void* tensor_map, int x, int y, int z, int w, uint32_t bar) {
+    asm volatile(
+        "cp.async.bulk.tensor.4d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4, %5}], [%6];" ::"r"(dst_smem),
+        "l"(tensor_map), "r"(x), "r"(y), "r"(z), "r"(w), "r"(bar)
+        : "memory");
+}
+// Makes a tensor map that was written to global memory before this kernel started (by a copy on the
+// same stream) the one the copy engine uses, whatever an earlier kernel read from that address.
+__device__ __forceinline__ void tensormap_acquire(const void* tensor_map) {
+    asm volatile("fence.proxy.tensormap::generic.acquire.gpu [%0], 128;" ::"l"(tensor_map) : "memory");
+}
 // 16-byte cp.async; src_bytes = 0 writes zeros. The .ca form goes through L1, which merges the
 // sixteen 16-byte pieces of a 256-byte row into full lines: measured 64-74 GB/s per SM for the
 // tile-staging pattern here, against 24 GB/s for .cg (each piece its own L2 request).
@@ -112,6 +126,23 @@ __device__ __forceinline__ uint64_t smem_desc(uint32_t addr, uint32_t lbo, uint3
     d |= (uint64_t)((sbo >> 4) & 0x3FFF) << 32;
     d |= (uint64_t)1 << 46;  // descriptor version of sm_100
     return d;                // base offset 0, layout type 0 (no swizzle)
+}
+// Shared-memory matrix descriptor for the 128-byte swizzle (the layout the tensor copy engine writes
+// for a box whose inner extent is 128 bytes): rows of 128 bytes, the 16-byte chunk index XORed with
+// (row mod 8); tiles start on 1024-byte boundaries.
+//   K-major  : a row holds 64 consecutive K elements; sbo = byte stride between 8-row groups (1024
+//              when rows are dense), lbo is not used (one 16-byte unit); the k-th MMA of a row
+//              (16 elements) starts 32*k bytes into the tile.
+//   MN-major : a row holds 64 consecutive M/N elements of one K index; lbo = byte stride between
+//              64-element blocks along M/N, sbo = byte stride between 8-row groups along K.
+__device__ __forceinline__ uint64_t smem_desc_sw128(uint32_t addr, uint32_t lbo, uint32_t sbo) {
+    uint64_t d = 0;
+    d |= (uint64_t)((addr >> 4) & 0x3FFF);
+    d |= (uint64_t)((lbo >> 4) & 0x3FFF) << 16;
+    d |= (uint64_t)((sbo >> 4) & 0x3FFF) << 32;
+    d |= (uint64_t)1 << 46;  // descriptor version of sm_100
+    d |= (uint64_t)2 << 61;  // layout type: 128-byte swizzle
+    return d;
 }
 // Instruction descriptor: bf16 x bf16 -> fp32, M = 128, N multiple of 16.
 __device__ __forceinline__ uint32_t instr_desc_bf16(int n, bool a_mn_major, bool b_mn_major) {

@@ -13,6 +13,8 @@
 //      now contracted over positions (MN-major B operand);
 // and the division by the row sum is applied after all tiles are summed (it commutes
 // with the blend), by finalize_parts_kernel.
+#include <cuda.h>   // tensor map types only: the encoder is looked up at run time
+
 #include <algorithm>
 
 #include "handle.h"
@@ -26,7 +28,7 @@ using namespace tc;
 constexpr int kSlots = 128;              // slots per CTA (MMA M)
 constexpr int kD = 128;                  // head dimension
 constexpr int kStageBytes = 32768;       // one tap x 128 channels x 128 slots, bf16
-constexpr int kThreads = 192;            // 4 loader/epilogue warps + MMA-issue warp + weight-producer warp
+constexpr int kThreads = 384;            // twelve warps: see compress_body
 constexpr int kMaxSmem = 232448 - 128;   // dynamic shared memory per CTA: 227 KB less the kernels' few static words
 constexpr uint32_t kTmemCols = 512;
 constexpr uint32_t kColUK = 256, kColUV = 384;
@@ -36,6 +38,7 @@ struct TcCompressParams {
     const __nv_bfloat16* gimage;  // [sets][slot blocks][k][halves][16][128][8]
     float* part_U;                // [units][slot blocks][parts][2][128 channels][128 slots]
     float* part_s;                // [units][slot blocks][parts][128]
+    int part_stride;              // partial sets reserved per (unit, slot block): >= parts
     float* R_store;               // optional [units][M][S]
     int* status;
     int n_tile, tiles, parts, tiles_per_part, halves, stages, rows_pad, slot_blocks;
@@ -61,8 +64,10 @@ __global__ void pack_image_kernel(const __nv_bfloat16* __restrict__ G, __nv_bflo
     }
 }
 
-// Work of one CTA: tiles [part*tiles_per_part, ...) of slot block sb of unit u. Runs with any
-// block size that is a multiple of 32 and at least 192 (warps beyond the sixth only help staging).
+// Work of one CTA of exactly 384 threads: tiles [part*tiles_per_part, ...) of slot block sb of unit u.
+// Thread 128 issues the MMAs, thread 160 feeds the weight ring, every thread stages rows, and all
+// twelve warps share the two epilogues: warp w owns accumulator rows (TMEM lanes) 32*(w%4)..+31
+// and every third 32-column chunk, starting with chunk w/4.
 // `tmem`: base of 512 TMEM columns the CTA owns. `cache_cg`: read cache rows around L1 (set when the
 // cache was rewritten by other SMs earlier in the SAME kernel; L1 is coherent only across launches).
 __device__ __forceinline__ void compress_body(const TcCompressParams& P, uint8_t* smem, uint32_t tmem, bool cache_cg, int part,
@@ -71,6 +76,8 @@ __device__ __forceinline__ void compress_body(const TcCompressParams& P, uint8_t
     const int nthr16 = blockDim.x / 16;
     const int n = u / p.heads, h = u % p.heads;
     const int tid = threadIdx.x, warp = tid >> 5;
+    const int eg = warp >> 2;                          // epilogue group: which column chunks
+    const int rl = (warp & 3) * 32 + (tid & 31);       // accumulator row = slot within the block
     const int n_tile = P.n_tile, pad = (p.k - 1) / 2, rows = n_tile + p.k - 1;
     const int NS = P.stages;
     const uint32_t lbo_z = (uint32_t)P.rows_pad * 16u;
@@ -104,9 +111,9 @@ __device__ __forceinline__ void compress_body(const TcCompressParams& P, uint8_t
         P.gimage + ((int64_t)set * P.slot_blocks + sb) * (int64_t)p.k * P.halves * (kStageBytes / 2);
     const uint32_t idesc_conv = instr_desc_bf16(n_tile, false, false);
     const uint32_t idesc_blend = instr_desc_bf16(kD, false, true);
-    const int slot = sb * kSlots + tid;  // meaningful for tid < 128
+    const int slot = sb * kSlots + rl;
     float bias_i = 0.f;
-    if (tid < kSlots && p.bias) bias_i = p.bias[(p.weights_per_head ? h * p.M : 0) + slot];
+    if (p.bias) bias_i = p.bias[(p.weights_per_head ? h * p.M : 0) + slot];
     const __nv_bfloat16* safe = unit_base<__nv_bfloat16>(p.xk.chunk, n, h);
 
     float ssum = 0.f;
@@ -181,19 +188,21 @@ __device__ __forceinline__ void compress_body(const TcCompressParams& P, uint8_t
         g += total;
 
         // ---- 3. accumulator -> bias, ReLU, row sum (Eq. 7), bf16 -> A operand of the blends
-        if (warp < 4) {
-            if (P.halves == 1) {
-                stage_tile(p.xv, zv, tid, kSlots / 16);
-                cp_async_wait_all();
-            }
-            mbar_wait(bar_acc, tile_it & 1, P.status, failed, 3);
-            tc_fence_after();
-            const uint32_t lane_addr = tmem + ((uint32_t)(warp * 32) << 16);
+        if (P.halves == 1 && (warp < 4 || warp >= 8)) {
+            stage_tile(p.xv, zv, warp < 4 ? tid : tid - 128, 16);
+            cp_async_wait_all();
+        }
+        __syncwarp();
+        mbar_wait(bar_acc, tile_it & 1, P.status, failed, 3);
+        tc_fence_after();
+        {
+            const uint32_t lane_addr = tmem + ((uint32_t)((warp & 3) * 32) << 16);
             float* rstore = P.R_store ? P.R_store + ((int64_t)u * p.M + slot) * p.S : nullptr;
-            for (int c0 = 0; c0 < n_tile; c0 += 32) {
+            for (int c0 = eg * 32; c0 < n_tile; c0 += 96) {
                 uint32_t v[32];
                 tmem_ld32(lane_addr + c0, v);
                 tmem_ld_wait();
+                const bool ragged = j0 + c0 + 32 > p.S;
 #pragma unroll
                 for (int e = 0; e < 32; e += 8) {
                     uint32_t pk[4];
@@ -202,8 +211,8 @@ __device__ __forceinline__ void compress_body(const TcCompressParams& P, uint8_t
                         const int ja = j0 + c0 + e + x;
                         float ra = fmaxf(__uint_as_float(v[e + x]) + bias_i, 0.f);
                         float rb = fmaxf(__uint_as_float(v[e + x + 1]) + bias_i, 0.f);
-                        if (ja >= p.S) ra = 0.f;
-                        if (ja + 1 >= p.S) rb = 0.f;
+                        if (ragged && ja >= p.S) ra = 0.f;
+                        if (ragged && ja + 1 >= p.S) rb = 0.f;
                         const __nv_bfloat162 pr = __floats2bfloat162_rn(ra, rb);
                         pk[x >> 1] = *reinterpret_cast<const uint32_t*>(&pr);
                         const float fa = __low2float(pr), fb = __high2float(pr);
@@ -213,7 +222,7 @@ __device__ __forceinline__ void compress_body(const TcCompressParams& P, uint8_t
                             if (ja + 1 < p.S) rstore[ja + 1] = fb;
                         }
                     }
-                    *reinterpret_cast<uint4*>(ring_ptr + ((c0 + e) >> 3) * 2048 + tid * 16) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
+                    *reinterpret_cast<uint4*>(ring_ptr + ((c0 + e) >> 3) * 2048 + rl * 16) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
                 }
             }
             fence_proxy_async();
@@ -240,26 +249,26 @@ __device__ __forceinline__ void compress_body(const TcCompressParams& P, uint8_t
     }
 
     // ---- partial blends and row sums of this CTA's tiles
-    if (warp < 4 && tile_it > 0) {
+    if (tile_it > 0) {
         tc_fence_after();
-        const uint32_t lane_addr = tmem + ((uint32_t)(warp * 32) << 16);
-        const int64_t pidx = ((int64_t)u * P.slot_blocks + sb) * P.parts + part;
-        // stored channel-major ([channel][slot]) so that a warp's 32 lanes write 128 contiguous bytes
-        float* outK = P.part_U + (pidx * 2 + 0) * (kSlots * kD) + tid;
-        float* outV = P.part_U + (pidx * 2 + 1) * (kSlots * kD) + tid;
+        float* sums = reinterpret_cast<float*>(ring_ptr);      // [3 groups][128 rows]; the ring is idle now
+        sums[eg * kSlots + rl] = ssum;
+        const uint32_t lane_addr = tmem + ((uint32_t)((warp & 3) * 32) << 16);
+        const int64_t pidx = ((int64_t)u * P.slot_blocks + sb) * P.part_stride + part;
+        // stored channel-major ([channel][slot]) so that a warp's 32 lanes write 128 contiguous bytes;
+        // the eight (matrix, 32-channel chunk) pieces go round the three groups
 #pragma unroll 1
-        for (int c0 = 0; c0 < kD; c0 += 32) {
-            uint32_t a[32], b[32];
-            tmem_ld32(lane_addr + kColUK + c0, a);
-            tmem_ld32(lane_addr + kColUV + c0, b);
+        for (int piece = eg; piece < 2 * (kD / 32); piece += 3) {
+            const int mat = piece & 1, c0 = (piece >> 1) * 32;
+            float* out = P.part_U + (pidx * 2 + mat) * (kSlots * kD) + rl;
+            uint32_t a[32];
+            tmem_ld32(lane_addr + (mat ? kColUV : kColUK) + c0, a);
             tmem_ld_wait();
 #pragma unroll
-            for (int e = 0; e < 32; ++e) {
-                outK[(c0 + e) * kSlots] = __uint_as_float(a[e]);
-                outV[(c0 + e) * kSlots] = __uint_as_float(b[e]);
-            }
+            for (int e = 0; e < 32; ++e) out[(c0 + e) * kSlots] = __uint_as_float(a[e]);
         }
-        P.part_s[pidx * kSlots + tid] = ssum;
+        __syncthreads();
+        if (tid < kSlots) P.part_s[pidx * kSlots + tid] = sums[tid] + sums[kSlots + tid] + sums[2 * kSlots + tid];
     }
     tc_fence_before();
     __syncthreads();
@@ -304,7 +313,7 @@ __device__ __forceinline__ void finalize_tile(const TcCompressParams& P, float (
     const int n = u / p.heads, h = u % p.heads;
     const int i0 = bx * 32, c0 = by * 32;   // slot tile, channel tile
     const int sb = i0 / kSlots, il0 = i0 % kSlots;
-    const int64_t base = ((int64_t)u * P.slot_blocks + sb) * P.parts;
+    const int64_t base = ((int64_t)u * P.slot_blocks + sb) * P.part_stride;
     const int tx = threadIdx.x % 32, ty = threadIdx.x / 32;
     __syncthreads();                            // the tile buffers may still be read by the previous tile
     if (ty == 0) {
@@ -356,56 +365,67 @@ __global__ void __launch_bounds__(256) finalize_parts_kernel(TcCompressParams P)
 constexpr int kAttnThreads = 384;                  // 8 softmax + 1 MMA-issue + 3 loader warps (384 x 168 registers fill the file)
 constexpr int kAttnLoaderWarps = 3;
 constexpr int kAttnLoaders = 32 * kAttnLoaderWarps;
-constexpr uint32_t kLboT = 129 * 16;               // Q/K/V tiles: [16 channel groups][129 x 16 B]: the odd row count
-                                                   // spreads the 16 groups of a row over the banks (cp.async writes)
-constexpr uint32_t kTileBytes = 16 * kLboT;        // 33024
-constexpr uint32_t kPBytes = 32768;                // P tiles: [16 key groups][128 rows][8 keys]
-constexpr uint32_t kAttnSmem = 5 * kTileBytes + 2 * kPBytes + 256 * 4 + 128;   // Q, K x2, V x2, P x2, exchange, barriers
+constexpr uint32_t kHalfBytes = 16384;             // 128 rows x 64 channels: rows of 128 bytes, 128-byte swizzle
+constexpr uint32_t kTileBytes = 2 * kHalfBytes;    // Q/K/V tiles: channels 0-63, then channels 64-127
+constexpr uint32_t kPBytes = 32768;                // P tiles: [16 key groups][128 rows][8 keys], no swizzle
+constexpr uint32_t kAttnSmem = 5 * kTileBytes + 2 * kPBytes + 256 * 4 + 128 + 1024;   // Q, K x2, V x2, P x2, exchange, barriers, alignment
 constexpr uint32_t kAttnTmemCols = 512;            // S x2 (128 columns each), O (128)
 constexpr float kRescaleThreshold = 8.f;
 
-struct TcAttnParams {
+// Tensor maps of the five operands: [batch, heads, tokens, 128] bf16 views cut into boxes of 128 tokens x
+// 64 channels. A map the driver would not encode (its bit in tma_mask clear) leaves that operand to the
+// loader warps' 16-byte copies, which write the same swizzled tile.
+enum { kMapQ = 0, kMapKChunk = 1, kMapVChunk = 2, kMapKCache = 3, kMapVCache = 4, kMaps = 5 };
+struct alignas(64) TcAttnParams {
+    CUtensorMap maps[kMaps];
     AttnParams base;
     int* status;
+    unsigned tma_mask;
 };
 
-// Work of one CTA (exactly kAttnThreads threads): query tile qtile of unit u.
-// `tmem`, `cache_cg`: as for compress_body.
-__device__ __forceinline__ void attention_body(const TcAttnParams& P, uint8_t* smem, uint32_t tmem, bool cache_cg, int qtile, int u) {
+// Work of one CTA (exactly kAttnThreads threads): query tile qtile of unit u. `tmem`: as for
+// compress_body. `maps`: P.maps where the copy engine can read them (kernel parameter space or global
+// memory); `maps_fresh`: they were written to global memory after an earlier kernel used that address.
+__device__ __forceinline__ void attention_body(const TcAttnParams& P, const CUtensorMap* maps, bool maps_fresh, uint8_t* smem_raw,
+                                               uint32_t tmem, int qtile, int u) {
     const AttnParams& p = P.base;
     const int n = u / p.heads, h = u % p.heads;
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int r0 = qtile * 128;
     const int S = p.c + p.b;
 
+    // the swizzle is a function of the shared-memory address: tiles start on 1024-byte boundaries
+    uint8_t* smem = smem_raw + ((1024u - (smem_u32(smem_raw) & 1023u)) & 1023u);
     uint8_t* q_ptr = smem;
     uint8_t* k_ptr = q_ptr + kTileBytes;       // two buffers
     uint8_t* v_ptr = k_ptr + 2 * kTileBytes;   // two buffers
     uint8_t* p_ptr = v_ptr + 2 * kTileBytes;   // two buffers
     float* xchg = reinterpret_cast<float*>(p_ptr + 2 * kPBytes);      // [2 halves][128 rows]
     uint64_t* bars = reinterpret_cast<uint64_t*>(xchg + 256);
-    volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(bars + 12);
-    volatile int* failed = reinterpret_cast<volatile int*>(tmem_slot + 1);
+    volatile int* failed = reinterpret_cast<volatile int*>(bars + 13);
     const uint32_t qs = smem_u32(q_ptr), ks = smem_u32(k_ptr), vs = smem_u32(v_ptr), ps = smem_u32(p_ptr);
     const uint32_t bar0 = smem_u32(bars);
     // all indexed by b = tile & 1; the n-th use of a buffer completes phase n of its barriers
-    auto k_full = [&](int b) { return bar0 + 8 * b; };          // loaders -> MMA: K tile staged (first phase: Q too)
-    auto v_full = [&](int b) { return bar0 + 80 + 8 * b; };     // loaders -> MMA: V tile staged
+    auto k_full = [&](int b) { return bar0 + 8 * b; };          // loader -> MMA: K tile staged
+    auto v_full = [&](int b) { return bar0 + 80 + 8 * b; };     // loader -> MMA: V tile staged
     auto s_full = [&](int b) { return bar0 + 16 + 8 * b; };     // MMA -> softmax: logits in TMEM
     auto s_free = [&](int b) { return bar0 + 32 + 8 * b; };     // softmax -> MMA: logits consumed
     auto p_full = [&](int b) { return bar0 + 48 + 8 * b; };     // softmax -> MMA: P written
-    auto pv_done = [&](int b) { return bar0 + 64 + 8 * b; };    // MMA -> loaders, softmax: K/V/P buffers free, O updated
+    auto pv_done = [&](int b) { return bar0 + 64 + 8 * b; };    // MMA -> loader, softmax: K/V/P buffers free, O updated
+    const uint32_t q_full = bar0 + 96;                          // loader -> MMA: Q tile staged
     constexpr int kMma = 256;                                   // lane 0 of warp 8
+    constexpr int kLoad = 288;                                  // lane 0 of warp 9: issues the tensor copies
 
     if (tid == kMma) {
         for (int b = 0; b < 2; ++b) {
-            mbar_init(k_full(b), kAttnLoaders);
-            mbar_init(v_full(b), kAttnLoaders);
+            mbar_init(k_full(b), 1);
+            mbar_init(v_full(b), 1);
             mbar_init(s_full(b), 1);
             mbar_init(s_free(b), 256);
             mbar_init(p_full(b), 256);
             mbar_init(pv_done(b), 1);
         }
+        mbar_init(q_full, 1);
         *failed = 0;
         fence_barrier_init();
     }
@@ -417,116 +437,127 @@ __device__ __forceinline__ void attention_body(const TcAttnParams& P, uint8_t* s
     const int ncols = p.c + last_row + 1;           // columns any query of this tile can see
     const int ntiles = (ncols + 127) / 128;
 
-    // ---- staging of one 128-row tile by `nw` warps, this warp being number `lw` of them: 16 lanes
-    // per row (256 contiguous bytes in global memory), two rows per warp instruction. Rows at or
-    // beyond `nrows` are zero-filled.
-    const __nv_bfloat16* safe = unit_base<__nv_bfloat16>(p.q, n, h);
-    auto stage_rows = [&](uint32_t dst, const __nv_bfloat16* base, int64_t st, int nrows, int lw, int nw, bool cg) {
-        const int q = lane & 15;
-        const uint32_t d0 = dst + q * kLboT;
-        const __nv_bfloat16* b0 = base + q * 8;
-        for (int r = 2 * lw + (lane >> 4); r < 128; r += 2 * nw) {
-            const bool valid = r < nrows;
-            if (cg) cp_async16_cg(d0 + r * 16, valid ? b0 + (int64_t)r * st : safe, valid ? 16u : 0u);
-            else cp_async16(d0 + r * 16, valid ? b0 + (int64_t)r * st : safe, valid ? 16u : 0u);
-        }
-    };
-    // keys (which = 0) or values (1) of key tile jt: the part inside the cache, then the part inside the chunk
-    auto load_tile = [&](int jt, int buf, int which, int lw, int nw) {
-        const CatView& x = which ? p.xv : p.xk;
-        const uint32_t dst = (which ? vs : ks) + buf * kTileBytes;
-        const int jb = jt * 128;
-        if (jb + 128 <= p.c) {
-            stage_rows(dst, unit_base<__nv_bfloat16>(x.cache, n, h) + (int64_t)jb * x.cache.st, x.cache.st, 128, lw, nw, cache_cg);
-        } else if (jb >= p.c) {
-            stage_rows(dst, unit_base<__nv_bfloat16>(x.chunk, n, h) + (int64_t)(jb - p.c) * x.chunk.st, x.chunk.st, S - jb, lw, nw, false);
-        } else {
-            // the tile straddles the end of the cache: row by row
-            const int q = lane & 15;
-            for (int r = 2 * lw + (lane >> 4); r < 128; r += 2 * nw) {
-                const int j = jb + r;
-                const bool valid = j < S;
-                const __nv_bfloat16* src = !valid ? safe
-                    : j < p.c ? unit_base<__nv_bfloat16>(x.cache, n, h) + (int64_t)j * x.cache.st + q * 8
-                              : unit_base<__nv_bfloat16>(x.chunk, n, h) + (int64_t)(j - p.c) * x.chunk.st + q * 8;
-                if (cache_cg && valid && j < p.c) cp_async16_cg(dst + q * kLboT + r * 16, src, 16u);
-                else cp_async16(dst + q * kLboT + r * 16, src, valid ? 16u : 0u);
-            }
-        }
-    };
-    // ---- prologue, all warps: Q and the first two key/value tiles
-    {
-        constexpr int nw = kAttnThreads / 32;
-        stage_rows(qs, safe + (int64_t)r0 * p.q.st, p.q.st, p.b - r0, warp, nw, false);
-        load_tile(0, 0, 0, warp, nw);
-        load_tile(0, 0, 1, warp, nw);
-        if (ntiles > 1) {
-            load_tile(1, 1, 0, warp, nw);
-            load_tile(1, 1, 1, warp, nw);
-        }
-        cp_async_wait_all();
-        fence_proxy_async();
-        __syncthreads();
-    }
-
     if (warp >= 9) {
-        // ---------------- loaders
+        // ---------------- loader: one lane drives the copy engine; the three warps together stage what
+        // the engine cannot (an operand without a tensor map, the tile that straddles the end of the cache)
         const int lw = warp - 9;
-        auto commit = [&]() { asm volatile("cp.async.commit_group;" ::: "memory"); };
-        // tiles 0 and 1 were staged by the prologue
-        mbar_arrive(k_full(0));
-        mbar_arrive(v_full(0));
-        if (ntiles > 1) {
-            mbar_arrive(k_full(1));
-            mbar_arrive(v_full(1));
+        const bool elected = tid == kLoad;
+        const unsigned mask = P.tma_mask;
+        const __nv_bfloat16* safe = unit_base<__nv_bfloat16>(p.q, n, h);
+        if (elected && maps_fresh) {
+            for (int i = 0; i < kMaps; ++i)
+                if ((mask >> i) & 1) tensormap_acquire(maps + i);
         }
-        // from here on, per-thread group order: [K(t+1)] [V(t+1)] ...; a tile is announced to the MMA
-        // issuer before this warp waits for any buffer that the issuer has to free
-        // Tile t (>= 2) goes into the buffers of tile t-2. Its keys are needed first (by S(t), while
-        // softmax(t-1) still runs), its values only by PV(t): the key copy is awaited and announced at
-        // once, the value copy is left in flight and announced in the next round, so one round costs one
-        // copy latency, not two. Every wait below is on MMAs whose inputs were announced in earlier rounds.
-        for (int t = 2; t < ntiles; ++t) {
-            const int b = t & 1, ph = ((t - 2) >> 1) & 1;
-            mbar_wait(s_full(b), ph, P.status, failed, 4);        // S(t-2) has read the key buffer
-            load_tile(t, b, 0, lw, kAttnLoaderWarps);
-            cp_async_wait_all();                                  // V(t-1) and K(t) have landed
-            fence_proxy_async();
-            if (t > 2) mbar_arrive(v_full((t - 1) & 1));
-            mbar_arrive(k_full(b));
-            mbar_wait(pv_done(b), ph, P.status, failed, 5);       // PV(t-2) has read the value buffer
-            load_tile(t, b, 1, lw, kAttnLoaderWarps);
-            commit();
-        }
-        if (ntiles > 2) {
+        // one 128-row tile through the engine: both 64-channel halves, signalled on `bar` as bytes
+        auto engine_tile = [&](uint32_t dst, uint32_t bar, int mi, int token) {
+            if (elected) {
+                mbar_expect_tx(bar, kTileBytes);
+                tma_load_4d(dst, maps + mi, 0, token, h, n, bar);
+                tma_load_4d(dst + kHalfBytes, maps + mi, 64, token, h, n, bar);
+            }
+        };
+        // swizzled address of the 16-byte piece q (8 channels) of row r
+        auto piece = [&](uint32_t dst, int r, int q) { return dst + (uint32_t)(q >> 3) * kHalfBytes + (uint32_t)r * 128u + (uint32_t)(((q & 7) ^ (r & 7)) << 4); };
+        // 16 lanes per row (256 contiguous bytes in global memory), two rows per warp instruction; rows at
+        // or beyond `nrows` are zero-filled
+        auto copy_rows = [&](uint32_t dst, const __nv_bfloat16* base, int64_t st, int nrows) {
+            const int q = lane & 15;
+            for (int r = 2 * lw + (lane >> 4); r < 128; r += 2 * kAttnLoaderWarps) {
+                const bool valid = r < nrows;
+                cp_async16(piece(dst, r, q), valid ? base + (int64_t)r * st + q * 8 : safe, valid ? 16u : 0u);
+            }
+        };
+        auto announce_copied = [&](uint32_t bar) {
             cp_async_wait_all();
             fence_proxy_async();
-            mbar_arrive(v_full((ntiles - 1) & 1));
+            asm volatile("bar.sync 2, 96;" ::: "memory");
+            if (elected) mbar_arrive(bar);
+        };
+        // keys (which = 0) or values (1) of key tile jt into buffer buf
+        auto load_kv = [&](int jt, int buf, int which) {
+            const CatView& x = which ? p.xv : p.xk;
+            const uint32_t dst = (which ? vs : ks) + buf * kTileBytes;
+            const uint32_t bar = which ? v_full(buf) : k_full(buf);
+            const int jb = jt * 128;
+            if (jb + 128 <= p.c) {
+                const int mi = kMapKCache + which;
+                if ((mask >> mi) & 1) {
+                    engine_tile(dst, bar, mi, jb);
+                } else {
+                    copy_rows(dst, unit_base<__nv_bfloat16>(x.cache, n, h) + (int64_t)jb * x.cache.st, x.cache.st, 128);
+                    announce_copied(bar);
+                }
+            } else if (jb >= p.c) {
+                const int mi = kMapKChunk + which;
+                if ((mask >> mi) & 1) {
+                    engine_tile(dst, bar, mi, jb - p.c);
+                } else {
+                    copy_rows(dst, unit_base<__nv_bfloat16>(x.chunk, n, h) + (int64_t)(jb - p.c) * x.chunk.st, x.chunk.st, S - jb);
+                    announce_copied(bar);
+                }
+            } else {
+                // the tile straddles the end of the cache: row by row
+                const int q = lane & 15;
+                for (int r = 2 * lw + (lane >> 4); r < 128; r += 2 * kAttnLoaderWarps) {
+                    const int j = jb + r;
+                    const bool valid = j < S;
+                    const __nv_bfloat16* src = !valid ? safe
+                        : j < p.c ? unit_base<__nv_bfloat16>(x.cache, n, h) + (int64_t)j * x.cache.st + q * 8
+                                  : unit_base<__nv_bfloat16>(x.chunk, n, h) + (int64_t)(j - p.c) * x.chunk.st + q * 8;
+                    cp_async16(piece(dst, r, q), src, valid ? 16u : 0u);
+                }
+                announce_copied(bar);
+            }
+        };
+        if (mask & 1u) {
+            engine_tile(qs, q_full, kMapQ, r0);
+        } else {
+            copy_rows(qs, safe + (int64_t)r0 * p.q.st, p.q.st, p.b - r0);
+            announce_copied(q_full);
+        }
+        load_kv(0, 0, 0);
+        load_kv(0, 0, 1);
+        if (ntiles > 1) {
+            load_kv(1, 1, 0);
+            load_kv(1, 1, 1);
+        }
+        // Tile t (>= 2) goes into the buffers of tile t-2: its keys as soon as S(t-2) has read the key
+        // buffer, its values as soon as PV(t-2) has read the value buffer. A tile is announced (or left
+        // to the engine to announce) before this warp waits for the next buffer.
+        for (int t = 2; t < ntiles; ++t) {
+            const int b = t & 1, ph = ((t - 2) >> 1) & 1;
+            mbar_wait(s_full(b), ph, P.status, failed, 4);
+            load_kv(t, b, 0);
+            mbar_wait(pv_done(b), ph, P.status, failed, 5);
+            load_kv(t, b, 1);
         }
     } else if (tid == kMma) {
         // ---------------- MMA issuer: S(0), then per tile S(t) followed by PV(t-1)
         const uint32_t idesc_s = instr_desc_bf16(128, false, false);
         const uint32_t idesc_o = instr_desc_bf16(128, false, true);
-        const uint64_t q0 = smem_desc(qs, kLboT, 128);
-        constexpr uint32_t kstep = (2 * kLboT) >> 4;   // two 8-channel groups per MMA
+        const uint64_t q0 = smem_desc_sw128(qs, 16, 1024);
+        // the kk-th 16-channel step of a K-major tile: which half, then 32 bytes per step inside the row
+        auto kstep = [](int kk) { return (uint64_t)(((kk >> 2) * kHalfBytes + (kk & 3) * 32u) >> 4); };
         auto issue_pv = [&](int t) {
             const int b = t & 1;
             mbar_wait(v_full(b), (t >> 1) & 1, P.status, failed, 6);
             mbar_wait(p_full(b), (t >> 1) & 1, P.status, failed, 6);
             tc_fence_after();
-            const uint64_t a0 = smem_desc(ps + b * kPBytes, 2048, 128), b0 = smem_desc(vs + b * kTileBytes, 128, kLboT);
+            // V is the MN-major operand: 64-channel blocks kHalfBytes apart, 16 keys (two 8-row groups) per step
+            const uint64_t a0 = smem_desc(ps + b * kPBytes, 2048, 128), b0 = smem_desc_sw128(vs + b * kTileBytes, kHalfBytes, 1024);
 #pragma unroll
-            for (int kk = 0; kk < 8; ++kk) umma_ss(tmem + 256, a0 + kk * 256u, b0 + kk * 16u, idesc_o, (t | kk) != 0);
+            for (int kk = 0; kk < 8; ++kk) umma_ss(tmem + 256, a0 + kk * 256u, b0 + kk * 128u, idesc_o, (t | kk) != 0);
             umma_commit(pv_done(b));
         };
+        mbar_wait(q_full, 0, P.status, failed, 7);
         for (int jt = 0; jt < ntiles; ++jt) {
             const int b = jt & 1;
             mbar_wait(k_full(b), (jt >> 1) & 1, P.status, failed, 7);
             if (jt >= 2) mbar_wait(s_free(b), ((jt >> 1) - 1) & 1, P.status, failed, 8);
             tc_fence_after();
-            const uint64_t k0 = smem_desc(ks + b * kTileBytes, kLboT, 128);
+            const uint64_t k0 = smem_desc_sw128(ks + b * kTileBytes, 16, 1024);
 #pragma unroll
-            for (int kk = 0; kk < 8; ++kk) umma_ss(tmem + b * 128, q0 + kk * kstep, k0 + kk * kstep, idesc_s, kk != 0);
+            for (int kk = 0; kk < 8; ++kk) umma_ss(tmem + b * 128, q0 + kstep(kk), k0 + kstep(kk), idesc_s, kk != 0);
             umma_commit(s_full(b));
             if (jt >= 1) issue_pv(jt - 1);
         }
@@ -651,7 +682,7 @@ __device__ __forceinline__ void attention_body(const TcAttnParams& P, uint8_t* s
     tc_fence_before();
     __syncthreads();
     if (tid == kMma) {
-        for (int s = 0; s < 12; ++s) mbar_inval(bar0 + 8 * s);
+        for (int s = 0; s < 13; ++s) mbar_inval(bar0 + 8 * s);
     }
 }
 
@@ -659,7 +690,7 @@ __global__ void __launch_bounds__(kAttnThreads, 1) attention_tc_kernel(const __g
     extern __shared__ __align__(128) uint8_t smem[];
     __shared__ uint32_t tmem_slot;
     const uint32_t tmem = cta_tmem_acquire(&tmem_slot);
-    attention_body(P, smem, tmem, false, blockIdx.x, blockIdx.y);
+    attention_body(P, P.maps, false, smem, tmem, blockIdx.x, blockIdx.y);
     cta_tmem_release(tmem);
 }
 
@@ -673,6 +704,8 @@ struct TcStepParams {
     TcAttnParams attn;
     TcCompressParams comp;
     int qtiles, n_attn_first, n_attn, comp_per_unit;   // comp_per_unit = parts * slot_blocks
+    // position in the item list of a persistent launch (sequence_tc_kernel)
+    int items_per_unit, item_end, finished_target;     // finished_target: items of a unit up to and including this step
 };
 
 // Work item `idx` of one chunk step, in the order above.
@@ -680,14 +713,14 @@ __device__ __forceinline__ void step_item(const TcStepParams& P, uint8_t* smem, 
     const int units = P.attn.base.units;
     const int n_comp = units * P.comp_per_unit;
     if (idx < P.n_attn_first) {
-        attention_body(P.attn, smem, tmem, cache_cg, P.qtiles - 1 - idx / units, idx % units);
+        attention_body(P.attn, P.attn.maps, false, smem, tmem, P.qtiles - 1 - idx / units, idx % units);
     } else if (idx < P.n_attn_first + n_comp) {
         idx -= P.n_attn_first;
         const int u = idx / P.comp_per_unit, rem = idx % P.comp_per_unit;
         compress_body(P.comp, smem, tmem, cache_cg, rem % P.comp.parts, rem / P.comp.parts, u);
     } else {
         idx -= n_comp;
-        attention_body(P.attn, smem, tmem, cache_cg, P.qtiles - 1 - idx / units, idx % units);
+        attention_body(P.attn, P.attn.maps, false, smem, tmem, P.qtiles - 1 - idx / units, idx % units);
     }
 }
 
@@ -700,71 +733,169 @@ __global__ void __launch_bounds__(kAttnThreads, 1) chunk_step_tc_kernel(const __
 }
 
 // ------------------------------------------------------------------ the whole chunk loop, one launch
-// A persistent cooperative grid (one CTA per SM) walks the steps of Algorithm 2. Per step the CTAs pull
-// the attention and compress work items of chunk_step_tc_kernel from a counter, meet at a grid barrier,
-// share the finalize tiles (new cache = partial blends / row sums), meet again, and go on to the next
-// chunk: no launch and no TMEM/set-up cost between chunks. The cache stays where it is (2 MB, L2); the
-// only care it needs is that reads of it go around L1 from the second step on, because another SM
-// rewrote it inside this same kernel.
+// A persistent grid (one CTA per SM) works through the steps of Algorithm 2 as ONE list of work items,
+// step after step and unit after unit inside a step, pulled from a counter. Steps of different units
+// are independent, so there is no device-wide barrier: an item of step n waits only until ITS unit's
+// cache holds the result of step n-1 (a per-unit step counter), and the CTA that completes the last
+// item of a (step, unit) pair rebuilds that unit's cache from the partial blends and publishes the
+// counter. While the slowest unit of a step is still busy, the other SMs already run the next step of
+// the units that are done; launch gaps, TMEM set-up and the per-step tail of the block scheduler go.
+// Items are handed out in list order and only ever wait for items earlier in the list, which a
+// running CTA has already taken: every wait ends whether or not all CTAs are resident at once.
 struct TcSeqParams {
     const TcStepParams* steps;   // device
-    int n_steps;
-    int* work;                   // [n_steps] work-item counters, zeroed before the launch
-    int* barrier;                // one arrival counter, zeroed before the launch
+    int n_steps, total_items;
+    int* work;                   // next item of the list; zeroed before the launch
+    int* finished;               // [units] items completed so far; zeroed before the launch
+    int* version;                // [units] steps whose cache update is complete; zeroed before the launch
     int* status;
 };
 
-// Bounded: a CTA that waits too long records code 20 and goes on, so the kernel still terminates.
-__device__ __forceinline__ void grid_barrier(int* counter, int target, int* status) {
-    __syncthreads();
-    if (threadIdx.x == 0) {
-        __threadfence();
-        atomicAdd(counter, 1);
-        bool ok = false;
-        for (uint32_t i = 0; i < (1u << 22); ++i) {
-            int seen;
-            asm volatile("ld.acquire.gpu.global.s32 %0, [%1];" : "=r"(seen) : "l"(counter) : "memory");
-            if (seen >= target) { ok = true; break; }
-            __nanosleep(64);
-        }
-        if (!ok) atomicCAS(status, 0, 20);
-        __threadfence();
+// New cache of unit u from the partial blends and row sums (Eq. 7 after Eq. 4-5), by one CTA of 384
+// threads. The partial sets (64 KB each, channel-major) come in through the copy engine, up to three at
+// a time; with more than three the earlier ones are folded into the first buffer. Sums run over the
+// sets in order, as in finalize_tile. A thread then owns one slot and eight channels: it reads along
+// channels (stride = one row of slots, its lane's bank), scales by 1/(s + eps) and stores 16 bytes.
+__device__ __forceinline__ void finalize_unit(const TcCompressParams& P, uint8_t* smem, int u) {
+    const CompressParams& p = P.base;
+    const int n = u / p.heads, h = u % p.heads;
+    constexpr int kSet = kSlots * kD;                             // floats per partial set
+    float* bufs = reinterpret_cast<float*>(smem);                 // [3][128 channels][128 slots]
+    float* inv_s = bufs + 3 * kSet;
+    uint64_t* bar = reinterpret_cast<uint64_t*>(inv_s + kSlots);
+    volatile int* failed = reinterpret_cast<volatile int*>(bar + 1);
+    const uint32_t bar_a = smem_u32(bar), bufs_a = smem_u32(bufs);
+    const int tid = threadIdx.x;
+    if (tid == 0) {
+        mbar_init(bar_a, 1);
+        *failed = 0;
+        fence_barrier_init();
     }
     __syncthreads();
+    uint32_t phase = 0;
+    for (int sb = 0; sb < P.slot_blocks; ++sb) {
+        const int64_t base = ((int64_t)u * P.slot_blocks + sb) * P.part_stride;
+        if (tid < kSlots) {
+            float sum = 0.f;
+            for (int pt = 0; pt < P.parts; ++pt) sum += __ldcg(P.part_s + (base + pt) * kSlots + tid);
+            sum += p.eps;
+            inv_s[tid] = 1.f / sum;
+            p.s[(int64_t)u * p.M + sb * kSlots + tid] = sum;
+        }
+        __syncthreads();
+        for (int mat = 0; mat < 2; ++mat) {
+            int live = 0;                                         // buffers to add up at the end
+            for (int pt = 0; pt < P.parts;) {
+                const int first_buf = pt == 0 ? 0 : 1;
+                const int cnt = min(P.parts - pt, 3 - first_buf);
+                if (tid == 0) {
+                    // the buffers' earlier accesses and the partials' arrival, before the copy engine's
+                    asm volatile("fence.proxy.async;" ::: "memory");
+                    mbar_expect_tx(bar_a, (uint32_t)cnt * kSet * 4u);
+                    for (int i = 0; i < cnt; ++i) {
+                        const float* src = P.part_U + ((base + pt + i) * 2 + mat) * kSet;
+                        for (uint32_t piece = 0; piece < kSet * 4u; piece += kStageBytes)
+                            bulk_load(bufs_a + (first_buf + i) * kSet * 4u + piece, reinterpret_cast<const uint8_t*>(src) + piece,
+                                      kStageBytes, bar_a);
+                    }
+                }
+                mbar_wait(bar_a, phase, P.status, failed, 21);
+                phase ^= 1;
+                pt += cnt;
+                live = first_buf + cnt;
+                if (pt < P.parts) {                               // more sets than buffers: fold into the first
+                    for (int i4 = tid; i4 < kSet / 4; i4 += kAttnThreads) {
+                        float4 acc = reinterpret_cast<float4*>(bufs)[i4];
+                        for (int b = 1; b < live; ++b) {
+                            const float4 v = reinterpret_cast<const float4*>(bufs + b * kSet)[i4];
+                            acc.x += v.x; acc.y += v.y; acc.z += v.z; acc.w += v.w;
+                        }
+                        reinterpret_cast<float4*>(bufs)[i4] = acc;
+                    }
+                    __syncthreads();
+                }
+            }
+            const View& out = mat ? p.v_out : p.k_out;
+            for (int idx = tid; idx < (kD / 8) * kSlots; idx += kAttnThreads) {
+                const int g = idx / kSlots, sl = idx % kSlots;
+                const float* src = bufs + (g * 8) * kSlots + sl;
+                float v[8];
+#pragma unroll
+                for (int e = 0; e < 8; ++e) v[e] = 0.f;
+                for (int b = 0; b < live; ++b) {
+#pragma unroll
+                    for (int e = 0; e < 8; ++e) v[e] += src[b * kSet + e * kSlots];
+                }
+                const float inv = inv_s[sl];
+                uint4 o;
+                o.x = pack_bf16(v[0] * inv, v[1] * inv);
+                o.y = pack_bf16(v[2] * inv, v[3] * inv);
+                o.z = pack_bf16(v[4] * inv, v[5] * inv);
+                o.w = pack_bf16(v[6] * inv, v[7] * inv);
+                *reinterpret_cast<uint4*>(unit_base_mut<__nv_bfloat16>(out, n, h) + (int64_t)(sb * kSlots + sl) * out.st + g * 8) = o;
+            }
+            __syncthreads();
+        }
+    }
+    if (tid == 0) mbar_inval(bar_a);
 }
 
 __global__ void __launch_bounds__(kAttnThreads, 1) sequence_tc_kernel(const __grid_constant__ TcSeqParams Q) {
     extern __shared__ __align__(128) uint8_t smem[];
     __shared__ uint32_t tmem_slot;
-    __shared__ int item_s;
+    __shared__ int item_s, last_s;
     const uint32_t tmem = cta_tmem_acquire(&tmem_slot);
-    int arrivals = 0;
-    for (int n = 0; n < Q.n_steps; ++n) {
-        // a thread-private copy: parameters read through a global pointer cannot be kept in registers
-        // across the bodies' stores, and the bodies read them inside their hot loops
-        const TcStepParams P = Q.steps[n];
-        const CompressParams& cp = P.comp.base;
-        const bool cache_cg = n > 0;
-        const int total = P.n_attn + cp.units * P.comp_per_unit;
-        while (true) {
-            if (threadIdx.x == 0) item_s = atomicAdd(Q.work + n, 1);
-            __syncthreads();
-            const int item = item_s;
-            __syncthreads();
-            if (item >= total) break;
-            step_item(P, smem, tmem, cache_cg, item);
+    int n = 0;
+    // a thread-private copy: parameters read through a global pointer cannot be kept in registers
+    // across the bodies' stores, and the bodies read them inside their hot loops
+    TcStepParams P = Q.steps[0];
+    while (true) {
+        if (threadIdx.x == 0) {
+            // after a wait has run out anywhere the results are void: stop handing out work
+            item_s = *reinterpret_cast<volatile int*>(Q.status) == 0 ? atomicAdd(Q.work, 1) : Q.total_items;
         }
-        arrivals += gridDim.x;
-        grid_barrier(Q.barrier, arrivals, Q.status);
-        // finalize tiles (32 slots x 32 channels), shared statically; the staging memory is free now
-        float (*tk)[33] = reinterpret_cast<float (*)[33]>(smem);
-        float (*tv)[33] = tk + 32;
-        float* inv_s = reinterpret_cast<float*>(tv + 32);
-        const int tx_n = cp.M / 32, ty_n = kD / 32, per_unit = tx_n * ty_n;
-        for (int t = blockIdx.x; t < per_unit * cp.units; t += gridDim.x)
-            finalize_tile(P.comp, tk, tv, inv_s, (t % per_unit) % tx_n, (t % per_unit) / tx_n, t / per_unit);
-        arrivals += gridDim.x;
-        grid_barrier(Q.barrier, arrivals, Q.status);
+        __syncthreads();
+        const int item = item_s;
+        __syncthreads();
+        if (item >= Q.total_items) break;
+        while (n + 1 < Q.n_steps && item >= P.item_end) P = Q.steps[++n];
+        const int local = item - (P.item_end - P.items_per_unit * P.attn.base.units);
+        const int u = local / P.items_per_unit;
+        int r = local % P.items_per_unit;
+        if (n > 0) {
+            // unit u's cache must hold the result of step n-1 (bounded wait; acquire, then the CTA barrier,
+            // orders every thread's reads of the cache and of nothing older after the publication)
+            if (threadIdx.x == 0) {
+                bool ok = false;
+                for (uint32_t i = 0; i < (1u << 22); ++i) {
+                    int seen;
+                    asm volatile("ld.acquire.gpu.global.s32 %0, [%1];" : "=r"(seen) : "l"(Q.version + u) : "memory");
+                    if (seen >= n) { ok = true; break; }
+                    __nanosleep(32);
+                }
+                if (!ok) atomicCAS(Q.status, 0, 20);
+                __threadfence();
+            }
+            __syncthreads();
+        }
+        // within a unit: compress CTAs first (the longest), then the attention tiles, longest first
+        if (r < P.comp_per_unit) compress_body(P.comp, smem, tmem, false, r % P.comp.parts, r / P.comp.parts, u);
+        else attention_body(P.attn, Q.steps[n].attn.maps, true, smem, tmem, P.qtiles - 1 - (r - P.comp_per_unit), u);
+        __syncthreads();
+        if (threadIdx.x == 0) {
+            __threadfence();                                        // this item's stores, then the count
+            const int done = atomicAdd(Q.finished + u, 1) + 1;
+            last_s = done == P.finished_target;
+            if (last_s) __threadfence();
+        }
+        __syncthreads();
+        if (last_s) {
+            finalize_unit(P.comp, smem, u);
+            if (threadIdx.x == 0) {
+                __threadfence();
+                asm volatile("st.release.gpu.global.s32 [%0], %1;" ::"l"(Q.version + u), "r"(n + 1) : "memory");
+            }
+        }
     }
     cta_tmem_release(tmem);
 }
@@ -844,7 +975,7 @@ void tensor_layout_workspace(lococo_handle* h, size_t* off) {
     h->off_steps = *off;
     *off = align(*off + (size_t)kMaxSeqSteps * sizeof(TcStepParams));
     h->off_sync = *off;
-    *off = align(*off + (size_t)(kMaxSeqSteps + 64) * sizeof(int));
+    *off = align(*off + (size_t)(64 + 2 * h->units) * sizeof(int));   // item counter, then per unit: finished, version
 }
 
 int tensor_pack_weights(lococo_handle* h, const void* G, cudaStream_t st) {
@@ -878,6 +1009,7 @@ static bool build_compress_params(lococo_handle* h, const CompressParams& p, boo
     P.R_store = p.W_out ? p.R : nullptr;
     P.status = reinterpret_cast<int*>(h->ws + h->off_status);
     P.n_tile = pl.n_tile; P.tiles = pl.tiles; P.parts = pl.parts; P.tiles_per_part = pl.tiles_per_part;
+    P.part_stride = fused ? max_parts : pl.parts;   // fixed regions where steps with different plans share a launch
     P.halves = p.c_in / 128; P.stages = pl.stages; P.rows_pad = pl.rows_pad; P.slot_blocks = SB;
     *out = P;
     if (cta_us) *cta_us = pl.cta_us;
@@ -920,12 +1052,63 @@ int tensor_compress(lococo_handle* h, const CompressParams& p, cudaStream_t st) 
     return r < 0 ? -1 : 1 + r;
 }
 
+// ---- tensor maps of the attention operands
+using EncodeTiledFn = CUresult (*)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
+                                   const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                   CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+static EncodeTiledFn encode_tiled() {
+    static EncodeTiledFn fn = [] {
+        void* sym = nullptr;
+        cudaDriverEntryPointQueryResult res;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &sym, cudaEnableDefault, &res) != cudaSuccess ||
+            res != cudaDriverEntryPointSuccess) {
+            cudaGetLastError();
+            sym = nullptr;
+        }
+        return reinterpret_cast<EncodeTiledFn>(sym);
+    }();
+    return fn;
+}
+
+// View [batch, heads, tokens, 128] of bf16, `tokens` rows valid (rows beyond read as zeros): boxes of
+// 128 tokens x 64 channels in the 128-byte swizzle.
+static bool make_tile_map(CUtensorMap* map, const View& v, int tokens, int heads, int batch) {
+    EncodeTiledFn fn = encode_tiled();
+    if (!fn || tokens < 1) return false;
+    const cuuint64_t dims[4] = {(cuuint64_t)kD, (cuuint64_t)tokens, (cuuint64_t)heads, (cuuint64_t)batch};
+    cuuint64_t strides[3] = {(cuuint64_t)v.st * 2, (cuuint64_t)v.sh * 2, (cuuint64_t)v.sb * 2};
+    // a dimension of extent 1 never uses its stride: give it a harmless one
+    if (heads == 1) strides[1] = strides[0] * (cuuint64_t)tokens;
+    if (batch == 1) strides[2] = strides[1] * (cuuint64_t)heads;
+    for (cuuint64_t st : strides)
+        if (st == 0 || st % 16 != 0 || st >= ((cuuint64_t)1 << 40)) return false;
+    if (v.st < 0 || v.sh < 0 || v.sb < 0 || reinterpret_cast<uintptr_t>(v.ptr) % 16 != 0) return false;
+    const cuuint32_t box[4] = {64, 128, 1, 1};
+    const cuuint32_t estr[4] = {1, 1, 1, 1};
+    return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, v.ptr, dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+              CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+static void fill_attention_maps(TcAttnParams* P) {
+    const AttnParams& a = P->base;
+    const int batch = a.units / a.heads;
+    P->tma_mask = 0;
+    if (make_tile_map(&P->maps[kMapQ], a.q, a.b, a.heads, batch)) P->tma_mask |= 1u << kMapQ;
+    if (make_tile_map(&P->maps[kMapKChunk], a.xk.chunk, a.b, a.heads, batch)) P->tma_mask |= 1u << kMapKChunk;
+    if (make_tile_map(&P->maps[kMapVChunk], a.xv.chunk, a.b, a.heads, batch)) P->tma_mask |= 1u << kMapVChunk;
+    if (a.c >= 128) {
+        if (make_tile_map(&P->maps[kMapKCache], a.xk.cache, a.c, a.heads, batch)) P->tma_mask |= 1u << kMapKCache;
+        if (make_tile_map(&P->maps[kMapVCache], a.xv.cache, a.c, a.heads, batch)) P->tma_mask |= 1u << kMapVCache;
+    }
+}
+
 static bool build_step_params(lococo_handle* h, const AttnParams& a, const CompressParams& p, TcStepParams* out) {
     TcStepParams P{};
     double comp_us = 0.0;
     if (!build_compress_params(h, p, true, &P.comp, &comp_us)) return false;
     P.attn.base = a;
     P.attn.status = P.comp.status;
+    fill_attention_maps(&P.attn);
     P.qtiles = (a.b + 127) / 128;
     P.n_attn = P.qtiles * a.units;
     // longest first: the attention tiles estimated to outlast a compress CTA (7 us fixed + 2.4 us per
@@ -965,11 +1148,10 @@ int tensor_chunk_step(lococo_handle* h, const AttnParams& a, const CompressParam
 static bool sequence_available(lococo_handle* h) {
     if (h->coop_grid == 0) {
         h->coop_grid = -1;
-        int dev = 0, coop = 0, sms = 0, per_sm = 0;
+        int dev = 0, sms = 0, per_sm = 0;
         if (cudaGetDevice(&dev) != cudaSuccess) return false;
-        cudaDeviceGetAttribute(&coop, cudaDevAttrCooperativeLaunch, dev);
         cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
-        if (!coop || sms < 1) return false;
+        if (sms < 1) return false;
         if (cudaFuncSetAttribute(sequence_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxSmem) != cudaSuccess ||
             cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, sequence_tc_kernel, kAttnThreads, kMaxSmem) != cudaSuccess ||
             per_sm < 1) {
@@ -991,13 +1173,21 @@ bool tensor_sequence_add(lococo_handle* h, const AttnParams& a, const CompressPa
     if (!sequence_available(h) || h->seq_count >= kMaxSeqSteps) return false;
     TcStepParams P;
     if (!build_step_params(h, a, p, &P)) return false;
+    P.items_per_unit = P.comp_per_unit + P.qtiles;
+    if ((int64_t)h->seq_items + (int64_t)P.items_per_unit * a.units > (int64_t)1 << 30) return false;
     if (h->seq_count == 0) {
         // take the next host slot; make sure the copy that last read it has been carried out
         h->seq_slot = (h->seq_slot + 1) % lococo_handle::kSeqSlots;
         cudaStreamCaptureStatus cap = cudaStreamCaptureStatusNone;
         cudaStreamIsCapturing(st, &cap);
         if (cap == cudaStreamCaptureStatusNone && h->seq_event[h->seq_slot]) cudaEventSynchronize(h->seq_event[h->seq_slot]);
+        h->seq_items = 0;
+        h->seq_per_unit = 0;
     }
+    h->seq_items += P.items_per_unit * a.units;
+    h->seq_per_unit += P.items_per_unit;
+    P.item_end = h->seq_items;
+    P.finished_target = h->seq_per_unit;
     TcStepParams* slot = reinterpret_cast<TcStepParams*>(h->seq_host) + (size_t)h->seq_slot * kMaxSeqSteps;
     slot[h->seq_count++] = P;
     return true;
@@ -1011,11 +1201,13 @@ int tensor_sequence_launch(lococo_handle* h, cudaStream_t st, void* prof) {
     TcSeqParams Q{};
     Q.steps = reinterpret_cast<const TcStepParams*>(h->ws + h->off_steps);
     Q.n_steps = n;
+    Q.total_items = h->seq_items;
     Q.work = reinterpret_cast<int*>(h->ws + h->off_sync);
-    Q.barrier = Q.work + kMaxSeqSteps;
+    Q.finished = Q.work + 64;
+    Q.version = Q.finished + h->units;
     Q.status = reinterpret_cast<int*>(h->ws + h->off_status);
     if (cudaMemcpyAsync(h->ws + h->off_steps, slot, (size_t)n * sizeof(TcStepParams), cudaMemcpyHostToDevice, st) != cudaSuccess ||
-        cudaMemsetAsync(h->ws + h->off_sync, 0, (size_t)(kMaxSeqSteps + 64) * sizeof(int), st) != cudaSuccess)
+        cudaMemsetAsync(h->ws + h->off_sync, 0, (size_t)(64 + 2 * h->units) * sizeof(int), st) != cudaSuccess)
         return -1;
     cudaStreamCaptureStatus cap = cudaStreamCaptureStatusNone;
     cudaStreamIsCapturing(st, &cap);
@@ -1024,16 +1216,11 @@ int tensor_sequence_launch(lococo_handle* h, cudaStream_t st, void* prof) {
             return -1;
         cudaEventRecord(h->seq_event[h->seq_slot], st);
     }
-    void* args[] = {&Q};
     prof_begin(prof, 3, st);
-    const cudaError_t e = cudaLaunchCooperativeKernel(reinterpret_cast<void*>(sequence_tc_kernel), dim3(h->coop_grid),
-                                                      dim3(kAttnThreads), args, kMaxSmem, st);
+    sequence_tc_kernel<<<std::min(h->coop_grid, Q.total_items), kAttnThreads, kMaxSmem, st>>>(Q);
+    const bool ok = cudaGetLastError() == cudaSuccess;
     prof_end(prof, st);
-    if (e != cudaSuccess) {
-        cudaGetLastError();
-        return -1;
-    }
-    return 1;
+    return ok ? 1 : -1;
 }
 
 void tensor_sequence_release(lococo_handle* h) {
@@ -1059,6 +1246,7 @@ int tensor_attention(lococo_handle* h, const AttnParams& p, cudaStream_t st) {
     TcAttnParams P{};
     P.base = p;
     P.status = reinterpret_cast<int*>(h->ws + h->off_status);
+    fill_attention_maps(&P);
     dim3 grid((p.b + 127) / 128, p.units);
     prof_begin(p.prof, 1, st);
     attention_tc_kernel<<<grid, kAttnThreads, kAttnSmem, st>>>(P);
