@@ -573,6 +573,9 @@ __device__ __forceinline__ void attention_body(const TcAttnParams& P, const CUte
         float m_used = 0.f, lrun = 0.f;
         const int vis = live ? p.c + row + 1 : 1;   // visible columns of this row
         const float sc2 = p.scale * 1.4426950408889634f;
+        // the two threads of a row exchange their maxima rounded to bf16, one slot per tile parity:
+        // both then derive the same reference maximum, which only has to be near the true one
+        __nv_bfloat16* xmax = reinterpret_cast<__nv_bfloat16*>(xchg);   // [2 parities][2 halves][128 rows]
         for (int jt = 0; jt < ntiles; ++jt) {
             const int b = jt & 1;
             mbar_wait(s_full(b), (jt >> 1) & 1, P.status, failed, 9);
@@ -580,29 +583,48 @@ __device__ __forceinline__ void attention_body(const TcAttnParams& P, const CUte
             const uint32_t s_addr = lane_base + b * 128 + half * 64;
             const int j0 = jt * 128 + half * 64;
             const bool need_mask = jt * 128 + 128 > p.c + r0;
-            // pass 1: maximum of this thread's 64 scaled, masked logits, shared with the partner
-            float tmax = -INFINITY;
+            if (jt >= 2) mbar_wait(pv_done(b), ((jt >> 1) - 1) & 1, P.status, failed, 11);   // P buffer b is free
+            uint8_t* pdst = p_ptr + b * kPBytes + rl * 16;
+            // One sweep over this thread's 64 logits: P = exp2(s - m) in bf16 into the A-operand layout
+            // [key group][row][8 keys], with the reference maximum m carried over from the earlier tiles,
+            // and the tile's own maximum on the side. Only if that maximum turns out to exceed m by more
+            // than the threshold (always for the first tile, rarely later) is m raised, O rescaled and
+            // the sweep repeated; a P that overflowed in the discarded sweep is simply overwritten.
+            float lsum = 0.f;
+            for (int attempt = 0; attempt < 2; ++attempt) {
+                float tmax = -INFINITY;
+                lsum = 0.f;
 #pragma unroll
-            for (int c0 = 0; c0 < 64; c0 += 32) {
-                uint32_t v[32];
-                tmem_ld32(s_addr + c0, v);
-                tmem_ld_wait();
+                for (int c0 = 0; c0 < 64; c0 += 32) {
+                    uint32_t v[32];
+                    tmem_ld32(s_addr + c0, v);
+                    tmem_ld_wait();
 #pragma unroll
-                for (int e = 0; e < 32; ++e) {
-                    const float s2 = __uint_as_float(v[e]) * sc2;
-                    if (!need_mask || j0 + c0 + e < vis) tmax = fmaxf(tmax, s2);
+                    for (int e = 0; e < 32; e += 8) {
+                        uint32_t pk[4];
+#pragma unroll
+                        for (int x = 0; x < 8; x += 2) {
+                            const int ja = j0 + c0 + e + x;
+                            const float sa = __uint_as_float(v[e + x]) * sc2, sb2 = __uint_as_float(v[e + x + 1]) * sc2;
+                            float pa = exp2f(sa - m_used), pb = exp2f(sb2 - m_used);
+                            if (need_mask && ja >= vis) pa = 0.f; else tmax = fmaxf(tmax, sa);
+                            if (need_mask && ja + 1 >= vis) pb = 0.f; else tmax = fmaxf(tmax, sb2);
+                            const __nv_bfloat162 pr = __floats2bfloat162_rn(pa, pb);
+                            pk[x >> 1] = *reinterpret_cast<const uint32_t*>(&pr);
+                            lsum += __low2float(pr) + __high2float(pr);
+                        }
+                        *reinterpret_cast<uint4*>(pdst + ((half * 64 + c0 + e) >> 3) * 2048) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
+                    }
                 }
-            }
-            xchg[half * 128 + rl] = tmax;
-            asm volatile("bar.sync 1, 256;" ::: "memory");
-            const float mt = fmaxf(tmax, xchg[(half ^ 1) * 128 + rl]);
-            asm volatile("bar.sync 1, 256;" ::: "memory");      // the slot is rewritten for the next tile
-            if (jt == 0) {
-                m_used = mt;        // finite: column 0 is visible to every row
-            } else {
-                // raise the reference maximum only for a large jump; O in TMEM is rescaled to match
-                const bool bump = mt > m_used + kRescaleThreshold;
-                if (__any_sync(0xffffffffu, bump)) {
+                if (attempt == 1) break;
+                const __nv_bfloat16 mine = __float2bfloat16_rn(tmax);
+                xmax[b * 256 + half * 128 + rl] = mine;
+                asm volatile("bar.sync 1, 256;" ::: "memory");
+                const float mt = fmaxf(__bfloat162float(mine), __bfloat162float(xmax[b * 256 + (half ^ 1) * 128 + rl]));
+                // column 0 is visible to every row, so mt of the first tile is finite
+                const bool bump = jt == 0 || mt > m_used + kRescaleThreshold;
+                if (!__any_sync(0xffffffffu, bump)) break;
+                if (jt > 0) {
                     const float f = bump ? exp2f(m_used - mt) : 1.f;
                     mbar_wait(pv_done((jt - 1) & 1), ((jt - 1) >> 1) & 1, P.status, failed, 10);
                     tc_fence_after();
@@ -617,34 +639,8 @@ __device__ __forceinline__ void attention_body(const TcAttnParams& P, const CUte
                     }
                     tmem_st_wait();
                     lrun *= f;
-                    if (bump) m_used = mt;
                 }
-            }
-            // pass 2: P = exp2(s - m), bf16, into the A-operand layout [key group][row][8 keys]
-            if (jt >= 2) mbar_wait(pv_done(b), ((jt >> 1) - 1) & 1, P.status, failed, 11);
-            uint8_t* pdst = p_ptr + b * kPBytes + rl * 16;
-            float lsum = 0.f;
-#pragma unroll
-            for (int c0 = 0; c0 < 64; c0 += 32) {
-                uint32_t v[32];
-                tmem_ld32(s_addr + c0, v);
-                tmem_ld_wait();
-#pragma unroll
-                for (int e = 0; e < 32; e += 8) {
-                    uint32_t pk[4];
-#pragma unroll
-                    for (int x = 0; x < 8; x += 2) {
-                        const int ja = j0 + c0 + e + x;
-                        float pa = exp2f(__uint_as_float(v[e + x]) * sc2 - m_used);
-                        float pb = exp2f(__uint_as_float(v[e + x + 1]) * sc2 - m_used);
-                        if (need_mask && ja >= vis) pa = 0.f;
-                        if (need_mask && ja + 1 >= vis) pb = 0.f;
-                        const __nv_bfloat162 pr = __floats2bfloat162_rn(pa, pb);
-                        pk[x >> 1] = *reinterpret_cast<const uint32_t*>(&pr);
-                        lsum += __low2float(pr) + __high2float(pr);
-                    }
-                    *reinterpret_cast<uint4*>(pdst + ((half * 64 + c0 + e) >> 3) * 2048) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
-                }
+                if (bump) m_used = mt;
             }
             lrun += lsum;
             tc_fence_before();
@@ -652,6 +648,7 @@ __device__ __forceinline__ void attention_body(const TcAttnParams& P, const CUte
             fence_proxy_async();
             mbar_arrive(p_full(b));
         }
+        asm volatile("bar.sync 1, 256;" ::: "memory");      // every exchange slot has been read: the sums reuse the space
         // the last PV has updated O
         mbar_wait(pv_done((ntiles - 1) & 1), ((ntiles - 1) >> 1) & 1, P.status, failed, 12);
         tc_fence_after();
