@@ -345,8 +345,20 @@ __device__ __forceinline__ void finalize_tile(const TcCompressParams& P, float (
     }
 }
 
+// Launched so that it may start while the kernel before it in the stream drains (programmatic
+// dependent launch): its CTAs take SMs as they fall free, let the kernel after them do the same, and
+// only then wait for the earlier kernel's results.
+__device__ __forceinline__ void overlap_with_neighbours() {
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+}
+__device__ __forceinline__ void wait_for_earlier_kernels() {
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+}
+
 __global__ void __launch_bounds__(256) finalize_parts_kernel(TcCompressParams P) {
     __shared__ float tk[32][33], tv[32][33], inv_s[32];
+    overlap_with_neighbours();
+    wait_for_earlier_kernels();
     finalize_tile(P, tk, tv, inv_s, blockIdx.x, blockIdx.y, blockIdx.z);
 }
 
@@ -724,7 +736,9 @@ __device__ __forceinline__ void step_item(const TcStepParams& P, uint8_t* smem, 
 __global__ void __launch_bounds__(kAttnThreads, 1) chunk_step_tc_kernel(const __grid_constant__ TcStepParams P) {
     extern __shared__ __align__(128) uint8_t smem[];
     __shared__ uint32_t tmem_slot;
+    overlap_with_neighbours();
     const uint32_t tmem = cta_tmem_acquire(&tmem_slot);
+    wait_for_earlier_kernels();
     step_item(P, smem, tmem, false, blockIdx.x);
     cta_tmem_release(tmem);
 }
@@ -1013,13 +1027,32 @@ static bool build_compress_params(lococo_handle* h, const CompressParams& p, boo
     return true;
 }
 
+// Launch that lets the kernel begin while its predecessor in the stream is still draining; the kernel
+// itself waits (wait_for_earlier_kernels) before it touches anything the predecessor produces.
+template <typename Param>
+static cudaError_t launch_overlapped(void (*kernel)(Param), dim3 grid, dim3 block, size_t smem, cudaStream_t st, const Param& arg) {
+    cudaLaunchConfig_t cfg{};
+    cfg.gridDim = grid;
+    cfg.blockDim = block;
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, kernel, arg);
+}
+
 // finalize (+ optional mixing-weight output) after the compress CTAs of either launch form
 static int finish_compress(const TcCompressParams& P, cudaStream_t st) {
     const CompressParams& p = P.base;
     int launches = 0;
     dim3 fgrid(p.M / 32, kD / 32, p.units);
-    finalize_parts_kernel<<<fgrid, 256, 0, st>>>(P);
-    if (cudaGetLastError() != cudaSuccess) return -1;
+    if (launch_overlapped(finalize_parts_kernel, fgrid, dim3(256), 0, st, P) != cudaSuccess) {
+        cudaGetLastError();
+        return -1;
+    }
     ++launches;
     if (p.W_out) {
         const int r = simt_write_weights(p.R, p.s, p.W_out, (int64_t)p.units * p.M, p.S, st);
@@ -1133,8 +1166,8 @@ int tensor_chunk_step(lococo_handle* h, const AttnParams& a, const CompressParam
     }
     const int blocks = P.n_attn + a.units * P.comp_per_unit;
     prof_begin(p.prof, 2, st);
-    chunk_step_tc_kernel<<<blocks, kAttnThreads, kMaxSmem, st>>>(P);
-    const bool ok = cudaGetLastError() == cudaSuccess;
+    const bool ok = launch_overlapped(chunk_step_tc_kernel, dim3(blocks), dim3(kAttnThreads), kMaxSmem, st, P) == cudaSuccess;
+    if (!ok) cudaGetLastError();
     prof_end(p.prof, st);
     if (!ok) return -1;
     const int r = finish_compress(P.comp, st);
