@@ -193,9 +193,11 @@ lococo_status lococo_host_staging_bytes(const lococo_handle* handle, int32_t L, 
 /*
  * lococo_process_sequence on HOST buffers: contiguous [batch, heads, L, d] Q, K, V are
  * copied to the device staging area, the loop runs from an empty cache, and O plus the
- * final cache ([batch, heads, M, d] each, optional) are copied back.  Host buffers
- * should be pinned for the copies to be asynchronous.  Synchronises `stream` before
- * returning; final_cache_len (host) receives the fill count.
+ * final cache ([batch, heads, M, d] each, optional) are copied back.  The three legs are
+ * pipelined chunk by chunk on streams the handle owns (inputs of chunk n+1, the step of
+ * chunk n, the output of chunk n-1), ordered after the work already queued on `stream`.
+ * Host buffers should be pinned for the copies to be asynchronous.  Synchronises `stream`
+ * before returning; final_cache_len (host) receives the fill count.
  */
 lococo_status lococo_process_sequence_host(lococo_handle* handle, const void* Q_host, const void* K_host,
                                            const void* V_host, int32_t L, int32_t B, void* O_host,

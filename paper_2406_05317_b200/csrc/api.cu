@@ -260,6 +260,10 @@ lococo_status lococo_destroy(lococo_handle* h) {
     h->prof.release();
     if (h->loop_graph.exec) cudaGraphExecDestroy(h->loop_graph.exec);
     tensor_sequence_release(h);
+    for (int i = 0; i < h->host_ev_n; ++i) cudaEventDestroy(h->host_ev[i]);
+    delete[] h->host_ev;
+    if (h->host_in) cudaStreamDestroy(h->host_in);
+    if (h->host_out) cudaStreamDestroy(h->host_out);
     delete h;
     return LOCOCO_OK;
 }
@@ -507,17 +511,63 @@ lococo_status lococo_process_sequence_host(lococo_handle* h, const void* Qh, con
     char* base = static_cast<char*>(staging);
     char *dQ = base, *dK = base + seq, *dV = base + 2 * seq, *dO = base + 3 * seq;
     char *dKc = base + 4 * seq, *dVc = dKc + cache;
-    if (cudaMemcpyAsync(dQ, Qh, seq_bytes, cudaMemcpyHostToDevice, st) != cudaSuccess ||
-        cudaMemcpyAsync(dK, Kh, seq_bytes, cudaMemcpyHostToDevice, st) != cudaSuccess ||
-        cudaMemcpyAsync(dV, Vh, seq_bytes, cudaMemcpyHostToDevice, st) != cudaSuccess)
+    // Chunk by chunk on three streams: the copy of chunk n+1 to the device, the step of chunk n
+    // (Algorithm 2 needs nothing beyond chunk n and the cache) and the copy of chunk n-1's output back
+    // run at the same time, so the call costs about as much as its longest leg (normally the inputs).
+    const int n_chunks = (L + B - 1) / B;
+    if (!h->host_in && (cudaStreamCreateWithFlags(&h->host_in, cudaStreamNonBlocking) != cudaSuccess ||
+                        cudaStreamCreateWithFlags(&h->host_out, cudaStreamNonBlocking) != cudaSuccess))
         return LOCOCO_ERR_CUDA;
+    if (h->host_ev_n < 2 * n_chunks + 2) {
+        cudaEvent_t* ev = new (std::nothrow) cudaEvent_t[2 * n_chunks + 2]();
+        if (!ev) return LOCOCO_ERR_CUDA;
+        for (int i = 0; i < h->host_ev_n; ++i) ev[i] = h->host_ev[i];
+        for (int i = h->host_ev_n; i < 2 * n_chunks + 2; ++i)
+            if (cudaEventCreateWithFlags(&ev[i], cudaEventDisableTiming) != cudaSuccess) {
+                for (int j = h->host_ev_n; j < i; ++j) cudaEventDestroy(ev[j]);
+                delete[] ev;
+                return LOCOCO_ERR_CUDA;
+            }
+        delete[] h->host_ev;
+        h->host_ev = ev;
+        h->host_ev_n = 2 * n_chunks + 2;
+    }
+    cudaEvent_t* ev_in = h->host_ev;                 // chunk n is on the device
+    cudaEvent_t* ev_done = h->host_ev + n_chunks;    // chunk n's output is complete
+    cudaEvent_t ev_start = h->host_ev[2 * n_chunks], ev_out = h->host_ev[2 * n_chunks + 1];
+    const size_t row = (size_t)cfg.head_dim * h->elt, pitch = (size_t)L * row;
+    // the staging area is free once the work already queued on `stream` is done
+    if (cudaEventRecord(ev_start, st) != cudaSuccess || cudaStreamWaitEvent(h->host_in, ev_start, 0) != cudaSuccess ||
+        cudaStreamWaitEvent(h->host_out, ev_start, 0) != cudaSuccess)
+        return LOCOCO_ERR_CUDA;
+    for (int n = 0; n < n_chunks; ++n) {
+        const size_t off = (size_t)n * B * row;
+        const size_t width = (size_t)std::min(B, L - n * B) * row;
+        if (cudaMemcpy2DAsync(dQ + off, pitch, static_cast<const char*>(Qh) + off, pitch, width, h->units, cudaMemcpyHostToDevice, h->host_in) != cudaSuccess ||
+            cudaMemcpy2DAsync(dK + off, pitch, static_cast<const char*>(Kh) + off, pitch, width, h->units, cudaMemcpyHostToDevice, h->host_in) != cudaSuccess ||
+            cudaMemcpy2DAsync(dV + off, pitch, static_cast<const char*>(Vh) + off, pitch, width, h->units, cudaMemcpyHostToDevice, h->host_in) != cudaSuccess ||
+            cudaEventRecord(ev_in[n], h->host_in) != cudaSuccess)
+            return LOCOCO_ERR_CUDA;
+    }
     int c = 0;
-    s = lococo_process_sequence(h, contiguous(dQ, cfg.heads, L, cfg.head_dim), contiguous(dK, cfg.heads, L, cfg.head_dim),
-                                contiguous(dV, cfg.heads, L, cfg.head_dim), L, B,
-                                contiguous(dO, cfg.heads, L, cfg.head_dim), contiguous(dKc, cfg.heads, cfg.M, cfg.head_dim),
-                                contiguous(dVc, cfg.heads, cfg.M, cfg.head_dim), &c, nullptr, stream);
-    if (s) return s;
-    if (cudaMemcpyAsync(Oh, dO, seq_bytes, cudaMemcpyDeviceToHost, st) != cudaSuccess) return LOCOCO_ERR_CUDA;
+    const lococo_tensor tQ = contiguous(dQ, cfg.heads, L, cfg.head_dim), tK = contiguous(dK, cfg.heads, L, cfg.head_dim);
+    const lococo_tensor tV = contiguous(dV, cfg.heads, L, cfg.head_dim), tO = contiguous(dO, cfg.heads, L, cfg.head_dim);
+    const lococo_tensor tKc = contiguous(dKc, cfg.heads, cfg.M, cfg.head_dim), tVc = contiguous(dVc, cfg.heads, cfg.M, cfg.head_dim);
+    for (int n = 0; n < n_chunks; ++n) {
+        const int t0 = n * B, b = std::min(B, L - t0);
+        const size_t off = (size_t)t0 * row;
+        if (cudaStreamWaitEvent(st, ev_in[n], 0) != cudaSuccess) return LOCOCO_ERR_CUDA;
+        auto from = [&](lococo_tensor t) {
+            t.ptr = static_cast<char*>(t.ptr) + off;
+            return t;
+        };
+        s = run_chunk_loop(h, from(tQ), from(tK), from(tV), b, B, from(tO), tKc, tVc, &c, nullptr, st);
+        if (s) return s;
+        if (cudaEventRecord(ev_done[n], st) != cudaSuccess || cudaStreamWaitEvent(h->host_out, ev_done[n], 0) != cudaSuccess ||
+            cudaMemcpy2DAsync(static_cast<char*>(Oh) + off, pitch, dO + off, pitch, (size_t)b * row, h->units, cudaMemcpyDeviceToHost, h->host_out) != cudaSuccess)
+            return LOCOCO_ERR_CUDA;
+    }
+    if (cudaEventRecord(ev_out, h->host_out) != cudaSuccess || cudaStreamWaitEvent(st, ev_out, 0) != cudaSuccess) return LOCOCO_ERR_CUDA;
     if (Kc_h && cudaMemcpyAsync(Kc_h, dKc, cache_bytes, cudaMemcpyDeviceToHost, st) != cudaSuccess) return LOCOCO_ERR_CUDA;
     if (Vc_h && cudaMemcpyAsync(Vc_h, dVc, cache_bytes, cudaMemcpyDeviceToHost, st) != cudaSuccess) return LOCOCO_ERR_CUDA;
     if (cudaStreamSynchronize(st) != cudaSuccess) return LOCOCO_ERR_CUDA;

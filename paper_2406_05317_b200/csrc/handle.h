@@ -37,6 +37,10 @@ struct lococo_handle {
     unsigned char* seq_host = nullptr;
     cudaEvent_t seq_event[kSeqSlots] = {};
     int seq_slot = 0, seq_count = 0;
+    // lococo_process_sequence_host: copy streams and per-chunk events (created on first use)
+    cudaStream_t host_in = nullptr, host_out = nullptr;
+    cudaEvent_t* host_ev = nullptr;
+    int host_ev_n = 0;
     int seq_items = 0, seq_per_unit = 0;   // items queued so far: all units, one unit
     int coop_grid = 0;      // 0: not probed yet, -1: persistent kernel unavailable, > 0: CTAs that fit the device
     int64_t launches = 0;
