@@ -24,6 +24,9 @@ if str(ROOT) not in sys.path:
 METRIC = "chunk-step tokens/sec per layer (32 heads)"
 UNIT = "tokens/s"
 WORKLOAD = "cfg2"
+# dram__bytes_read.sum + dram__bytes_write.sum of one chunk_step_tc_kernel launch at this workload (ncu
+# capture of the committed kernel, steady-state step): 36.9 MB read + 0.5 MB written
+STEP_KERNEL_DRAM_BYTES = 37.4e6
 
 
 # ------------------------------------------------------------------ algorithmic work
@@ -308,7 +311,8 @@ def run_ours(args):
                           "frac": roof_ms / (total_ms / args.steps), "peak_source": peaks["source"] + " burst"},
         "roofline": {"bound": "tensor", "kernel": kernel, "flops_per_launch": flops_per_launch,
                      "achieved": achieved, "peak": peaks["bf16_tflops"], "unit": "TFLOP/s",
-                     "frac": (achieved / peaks["bf16_tflops"]) if achieved else None, "traffic": None,
+                     "frac": (achieved / peaks["bf16_tflops"]) if achieved else None,
+                     "traffic": STEP_KERNEL_DRAM_BYTES if (step_n and not seq_n) else None,
                      "peak_source": peaks["source"] + " burst", "launches": dom_n,
                      "us_per_launch": dom_per_launch_ms * 1e3},
     }
