@@ -1,0 +1,257 @@
+// A batched bf16 GEMM on the 5th-generation tensor cores for the contractions of the backward pass:
+//   D[z][m][n] (+)= alpha * sum_k A[m][k] * B[n][k]
+// Operands come in through the tensor copy engine (128-byte swizzle) with tensor maps built by the
+// caller, so "A[m][k]" is whatever the caller's map and coordinate rule make of it: either operand
+// may be K-major (rows of K elements) or MN-major (rows of M/N elements, one row per k), and the
+// coordinates of the box of K step s, output tile (tm, tn) and batch z are affine in
+// (tm, tn % n_inner, tn / n_inner, s % s_inner, s / s_inner, z). That is enough for plain batched
+// GEMMs, for sums over several units (the weight gradient), for row-shifted windows of one tensor
+// (a convolution tap = a row offset; loads may start at negative rows and read zeros there) and for
+// maps with overlapping strides (an im2col view that is never materialised).
+// One CTA = one 128 x 128 output tile: warp 5 lane 0 feeds a 3-stage ring (32 KB per stage), warp 4
+// lane 0 issues four K=16 MMAs per stage into 128 TMEM columns, warps 0-3 write the tile out.
+// Two CTAs fit an SM, so one tile's epilogue overlaps the other's main loop.
+#pragma once
+#include <cuda.h>
+
+#include <cstdint>
+
+#include "tc_common.cuh"
+
+namespace lococo {
+namespace gemm {
+
+using namespace tc;
+
+struct Coord {      // one box coordinate = c0 + tm*TM + tni*(TN % n_inner) + tno*(TN / n_inner) + si*(s % s_inner) + so*(s / s_inner) + z*Z
+    int c0, tm, tni, tno, si, so, z;
+};
+struct Operand {
+    CUtensorMap map;   // K-major: box {64 k, 128 rows}; MN-major: box {64 m/n, 64 k}, loaded at x and x + 64
+    Coord c[4];
+    int mn_major;
+    int pad[3];
+};
+enum Mode { kStoreF32 = 0, kAtomicF32 = 1, kStoreBF16 = 2, kAddF32 = 3 };
+struct alignas(64) Params {
+    Operand A, B;
+    int n_inner, s_inner;        // decomposition of the N tile index and of the K step index
+    int steps, splits;           // K steps (64 wide) in total; CTAs that share them (blockIdx.z = z * splits + split)
+    void* out;
+    int64_t out_z, out_m;        // element strides of the batch and of a row
+    int out_n_inner;             // column n lands at (n % out_n_inner) * out_n_in + (n / out_n_inner) * out_n_out
+    int64_t out_n_in, out_n_out;
+    int M, N;                    // valid rows and columns
+    int mode;
+    float alpha;
+    int* status;
+};
+
+constexpr int kThreads = 192;
+constexpr int kStages = 3;
+constexpr uint32_t kOperandBytes = 16384;
+constexpr uint32_t kStageBytes2 = 2 * kOperandBytes;
+constexpr uint32_t kSmem = kStages * kStageBytes2 + 1024 + 128;
+
+__device__ __forceinline__ int coord_of(const Coord& c, int tm, int tn, int n_inner, int s, int s_inner, int z) {
+    return c.c0 + c.tm * tm + c.tni * (tn % n_inner) + c.tno * (tn / n_inner) + c.si * (s % s_inner) + c.so * (s / s_inner) + c.z * z;
+}
+
+__global__ void __launch_bounds__(kThreads, 2) gemm_kernel(const __grid_constant__ Params P) {
+    extern __shared__ __align__(128) uint8_t smem_raw[];
+    __shared__ uint32_t tmem_slot;
+    uint8_t* smem = smem_raw + ((1024u - (smem_u32(smem_raw) & 1023u)) & 1023u);
+    uint64_t* bars = reinterpret_cast<uint64_t*>(smem + kStages * kStageBytes2);
+    volatile int* failed = reinterpret_cast<volatile int*>(bars + 2 * kStages + 1);
+    const uint32_t ring = smem_u32(smem), bar_full = smem_u32(bars), bar_empty = bar_full + 8 * kStages, bar_acc = bar_empty + 8 * kStages;
+    const int tid = threadIdx.x, warp = tid >> 5;
+    const int tm = blockIdx.x, tn = blockIdx.y;
+    const int z = blockIdx.z / P.splits, split = blockIdx.z % P.splits;
+    const int per = (P.steps + P.splits - 1) / P.splits;
+    const int s_begin = split * per, s_end = min(P.steps, s_begin + per);
+
+    if (tid == 128) {
+        for (int s = 0; s < kStages; ++s) {
+            mbar_init(bar_full + 8 * s, 1);
+            mbar_init(bar_empty + 8 * s, 1);
+        }
+        mbar_init(bar_acc, 1);
+        *failed = 0;
+        fence_barrier_init();
+    }
+    if (warp == 0) {
+        tmem_alloc(smem_u32(&tmem_slot), 128);
+        tmem_relinquish();
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem = *reinterpret_cast<volatile uint32_t*>(&tmem_slot);
+
+    if (tid == 160) {
+        // ---- producer
+        for (int s = s_begin, g = 0; s < s_end; ++s, ++g) {
+            const int st = g % kStages;
+            if (g >= kStages) mbar_wait(bar_empty + 8 * st, ((g / kStages) - 1) & 1, P.status, failed, 30);
+            mbar_expect_tx(bar_full + 8 * st, kStageBytes2);
+            const uint32_t dst = ring + st * kStageBytes2;
+#pragma unroll
+            for (int op = 0; op < 2; ++op) {
+                const Operand& O = op ? P.B : P.A;
+                const uint32_t d = dst + op * kOperandBytes;
+                const int tile = op ? tn : tm;
+                (void)tile;
+                const int x = coord_of(O.c[0], tm, tn, P.n_inner, s, P.s_inner, z), y = coord_of(O.c[1], tm, tn, P.n_inner, s, P.s_inner, z);
+                const int c2 = coord_of(O.c[2], tm, tn, P.n_inner, s, P.s_inner, z), c3 = coord_of(O.c[3], tm, tn, P.n_inner, s, P.s_inner, z);
+                if (O.mn_major) {
+                    tma_load_4d(d, &O.map, x, y, c2, c3, bar_full + 8 * st);
+                    tma_load_4d(d + kOperandBytes / 2, &O.map, x + 64, y, c2, c3, bar_full + 8 * st);
+                } else {
+                    tma_load_4d(d, &O.map, x, y, c2, c3, bar_full + 8 * st);
+                }
+            }
+        }
+    } else if (tid == 128) {
+        // ---- MMA issuer
+        const uint32_t idesc = instr_desc_bf16(128, P.A.mn_major != 0, P.B.mn_major != 0);
+        for (int s = s_begin, g = 0; s < s_end; ++s, ++g) {
+            const int st = g % kStages;
+            mbar_wait(bar_full + 8 * st, (g / kStages) & 1, P.status, failed, 31);
+            tc_fence_after();
+            const uint32_t a_addr = ring + st * kStageBytes2, b_addr = a_addr + kOperandBytes;
+            // K-major: 32 bytes per 16-element step inside the 128-byte row, 8-row groups 1024 bytes apart.
+            // MN-major: 16 k rows (two 8-row groups) per step, the two 64-wide halves 8 KB apart.
+            const uint64_t a0 = P.A.mn_major ? smem_desc_sw128(a_addr, kOperandBytes / 2, 1024) : smem_desc_sw128(a_addr, 16, 1024);
+            const uint64_t b0 = P.B.mn_major ? smem_desc_sw128(b_addr, kOperandBytes / 2, 1024) : smem_desc_sw128(b_addr, 16, 1024);
+            const uint32_t a_step = P.A.mn_major ? 2048u >> 4 : 32u >> 4, b_step = P.B.mn_major ? 2048u >> 4 : 32u >> 4;
+#pragma unroll
+            for (int kk = 0; kk < 4; ++kk) umma_ss(tmem, a0 + kk * a_step, b0 + kk * b_step, idesc, (g | kk) != 0);
+            umma_commit(bar_empty + 8 * st);
+        }
+        umma_commit(bar_acc);
+    }
+    if (warp < 4) {
+        // ---- epilogue: thread = one row of the tile
+        __syncwarp();
+        const bool any = s_end > s_begin;
+        if (any) {
+            mbar_wait(bar_acc, 0, P.status, failed, 32);
+            tc_fence_after();
+        }
+        const int row = tm * 128 + tid;
+        const uint32_t lane_addr = tmem + ((uint32_t)(warp * 32) << 16);
+        const int64_t base = (int64_t)z * P.out_z + (int64_t)row * P.out_m;
+        const bool contiguous = P.out_n_in == 1 && P.out_n_inner % 32 == 0;
+#pragma unroll 1
+        for (int c0 = 0; c0 < 128; c0 += 32) {
+            uint32_t v[32];
+            if (any) {
+                tmem_ld32(lane_addr + c0, v);
+                tmem_ld_wait();
+            } else {
+#pragma unroll
+                for (int e = 0; e < 32; ++e) v[e] = 0u;
+            }
+            const int n0 = tn * 128 + c0;
+            if (row >= P.M || n0 >= P.N || (!any && P.mode != kStoreF32 && P.mode != kStoreBF16)) continue;
+            const int64_t col0 = (int64_t)(n0 % P.out_n_inner) * P.out_n_in + (int64_t)(n0 / P.out_n_inner) * P.out_n_out;
+            if (contiguous && n0 + 32 <= P.N) {
+                if (P.mode == kStoreF32) {
+                    float4* o = reinterpret_cast<float4*>(static_cast<float*>(P.out) + base + col0);
+#pragma unroll
+                    for (int e = 0; e < 32; e += 4)
+                        o[e >> 2] = make_float4(__uint_as_float(v[e]) * P.alpha, __uint_as_float(v[e + 1]) * P.alpha,
+                                                __uint_as_float(v[e + 2]) * P.alpha, __uint_as_float(v[e + 3]) * P.alpha);
+                } else if (P.mode == kAddF32) {
+                    float4* o = reinterpret_cast<float4*>(static_cast<float*>(P.out) + base + col0);
+#pragma unroll
+                    for (int e = 0; e < 32; e += 4) {
+                        float4 t = o[e >> 2];
+                        t.x += __uint_as_float(v[e]) * P.alpha; t.y += __uint_as_float(v[e + 1]) * P.alpha;
+                        t.z += __uint_as_float(v[e + 2]) * P.alpha; t.w += __uint_as_float(v[e + 3]) * P.alpha;
+                        o[e >> 2] = t;
+                    }
+                } else if (P.mode == kStoreBF16) {
+                    uint4* o = reinterpret_cast<uint4*>(static_cast<__nv_bfloat16*>(P.out) + base + col0);
+#pragma unroll
+                    for (int e = 0; e < 32; e += 8)
+                        o[e >> 3] = make_uint4(pack_bf16(__uint_as_float(v[e]) * P.alpha, __uint_as_float(v[e + 1]) * P.alpha),
+                                               pack_bf16(__uint_as_float(v[e + 2]) * P.alpha, __uint_as_float(v[e + 3]) * P.alpha),
+                                               pack_bf16(__uint_as_float(v[e + 4]) * P.alpha, __uint_as_float(v[e + 5]) * P.alpha),
+                                               pack_bf16(__uint_as_float(v[e + 6]) * P.alpha, __uint_as_float(v[e + 7]) * P.alpha));
+                } else {
+                    float* o = static_cast<float*>(P.out) + base + col0;
+#pragma unroll
+                    for (int e = 0; e < 32; ++e) atomicAdd(o + e, __uint_as_float(v[e]) * P.alpha);
+                }
+            } else {
+#pragma unroll 1
+                for (int e = 0; e < 32; ++e) {
+                    const int n = n0 + e;
+                    if (n >= P.N) break;
+                    const int64_t col = (int64_t)(n % P.out_n_inner) * P.out_n_in + (int64_t)(n / P.out_n_inner) * P.out_n_out;
+                    const float x = __uint_as_float(v[e]) * P.alpha;
+                    if (P.mode == kStoreF32) static_cast<float*>(P.out)[base + col] = x;
+                    else if (P.mode == kAddF32) static_cast<float*>(P.out)[base + col] += x;
+                    else if (P.mode == kStoreBF16) static_cast<__nv_bfloat16*>(P.out)[base + col] = __float2bfloat16_rn(x);
+                    else atomicAdd(static_cast<float*>(P.out) + base + col, x);
+                }
+            }
+        }
+    }
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 0) tmem_dealloc(tmem, 128);
+    if (tid == 128) {
+        for (int s = 0; s < 2 * kStages + 1; ++s) mbar_inval(bar_full + 8 * s);
+    }
+}
+
+// ---- host side
+using EncodeTiledFn = CUresult (*)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
+                                   const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                   CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+inline EncodeTiledFn encode_tiled() {
+    static EncodeTiledFn fn = [] {
+        void* sym = nullptr;
+        cudaDriverEntryPointQueryResult res;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &sym, cudaEnableDefault, &res) != cudaSuccess ||
+            res != cudaDriverEntryPointSuccess) {
+            cudaGetLastError();
+            sym = nullptr;
+        }
+        return reinterpret_cast<EncodeTiledFn>(sym);
+    }();
+    return fn;
+}
+
+// bf16 tensor of rank 4: extents dims[0..3] (dims[0] innermost, contiguous), byte strides of dims 1..3.
+// K-major operands take boxes of 64 x 128, MN-major operands boxes of 64 x 64.
+inline bool make_map(CUtensorMap* map, const void* base, const uint64_t dims[4], const uint64_t strides[3], bool mn_major) {
+    EncodeTiledFn fn = encode_tiled();
+    if (!fn || (reinterpret_cast<uintptr_t>(base) & 15u)) return false;
+    cuuint64_t d[4], s[3];
+    for (int i = 0; i < 4; ++i) d[i] = dims[i] ? dims[i] : 1;
+    for (int i = 0; i < 3; ++i) {
+        s[i] = strides[i];
+        if (s[i] == 0 || s[i] % 16 != 0 || s[i] >= ((cuuint64_t)1 << 40)) return false;
+    }
+    const cuuint32_t box[4] = {64, mn_major ? 64u : 128u, 1, 1};
+    const cuuint32_t estr[4] = {1, 1, 1, 1};
+    return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(base), d, s, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+              CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+// Launch over (m_tiles, n_tiles, batch * splits). Returns false when the launch was refused.
+inline bool launch(const Params& P, int m_tiles, int n_tiles, int batch, cudaStream_t st) {
+    static bool attr_set = false;
+    if (!attr_set) {
+        if (cudaFuncSetAttribute(gemm_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmem) != cudaSuccess) return false;
+        attr_set = true;
+    }
+    gemm_kernel<<<dim3(m_tiles, n_tiles, batch * P.splits), kThreads, kSmem, st>>>(P);
+    return cudaGetLastError() == cudaSuccess;
+}
+
+}  // namespace gemm
+}  // namespace lococo
