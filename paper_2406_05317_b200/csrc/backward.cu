@@ -13,6 +13,7 @@
 // All arithmetic is fp32 on CUDA cores; storage type T is float or bf16.
 #include <algorithm>
 
+#include "backward.h"
 #include "handle.h"
 
 namespace lococo {
@@ -20,24 +21,6 @@ namespace lococo {
 int simt_conv_rowsum(int dtype, const CompressParams& p, cudaStream_t st);
 
 namespace {
-
-struct BwdStep {
-    CatView xk, xv;            // [saved cache; chunk]
-    View q, o, d_o;            // this chunk's queries, outputs, output gradients
-    View dq, dk, dv;           // this chunk's gradients (outputs)
-    int heads, units, d, M, k, c_in, c, b, S;
-    int weights_per_head;
-    const void* g_packed;      // [sets][k][M][c_in]
-    float scale;
-    const float* lse;          // this chunk's log-sum-exp, [units][lse_stride]
-    int64_t lse_stride;
-    float *R, *s;              // recomputed ReLU'd logits [units][M][S] and denominators [units][M]
-    float* dA;                 // [units][M][S]: dw, then dA in place
-    float* delta;              // [units][b]: <dO_r, O_r>
-    float *gK, *gV;            // [units][M][d] gradient w.r.t. the cache (after the step in, before the step out)
-    float *dXK, *dXV;          // [units][S][d]
-    float *dG, *dbias;         // [sets][M][c_in][k], [sets][M]
-};
 
 __global__ void zero_kernel(float* p, int64_t n) {
     for (int64_t i = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; i < n; i += (int64_t)gridDim.x * blockDim.x) p[i] = 0.f;
@@ -517,9 +500,15 @@ __global__ void bwd_init_g_kernel(View gk_in, View gv_in, float* gK, float* gV, 
 bool launched() { return cudaGetLastError() == cudaSuccess; }
 
 // All kernels of one reversed step. Returns the number of launches or -1.
+// `tb` (tensor-core scratch) non-null: the contractions run as tcgen05 GEMMs (tensor_backward.cu).
 template <typename T>
-int backward_step(const BwdStep& p, const CompressParams& fwd, int dtype, cudaStream_t st) {
+int backward_step(lococo_handle* h, const BwdStep& p, const CompressParams& fwd, int dtype, int B, char* tb, cudaStream_t st) {
     int n = 0;
+    if (tb) {
+        const int r = tensor_backward_pack(h, p, B, tb, st);
+        if (r < 0) return -1;
+        n += r;
+    }
     const int64_t dx = (int64_t)p.units * p.S * p.d;
     const int zb = (int)std::min<int64_t>((dx + 255) / 256, 4096);
     if (p.c + p.b <= p.M) {
@@ -531,6 +520,11 @@ int backward_step(const BwdStep& p, const CompressParams& fwd, int dtype, cudaSt
         zero_kernel<<<zb, 256, 0, st>>>(p.dXV, dx);
         if (!launched()) return -1;
         n += 2;
+        if (tb) {
+            const int r = tensor_backward_compress(h, p, fwd, B, tb, st);
+            if (r < 0) return -1;
+            n += r;
+        } else {
         const int r = simt_conv_rowsum(dtype, fwd, st);   // R and s of the forward, recomputed
         if (r < 0) return -1;
         n += r;
@@ -549,9 +543,15 @@ int backward_step(const BwdStep& p, const CompressParams& fwd, int dtype, cudaSt
         bwd_dZ_kernel<T><<<dim3((p.S + 63) / 64, (p.c_in + 63) / 64, p.units), 256, smem, st>>>(p);
         if (!launched()) return -1;
         n += 2;
+        }
     }
     bwd_delta_kernel<T><<<(p.units * p.b + 7) / 8, 256, 0, st>>>(p);
-    if (p.d == 128) {
+    if (tb) {
+        if (!launched()) return -1;
+        const int r = tensor_backward_attention(h, p, B, tb, st);
+        if (r < 0) return -1;
+        n += r - 2;
+    } else if (p.d == 128) {
         bwd_attn_dq_kernel<T, 128><<<dim3((p.b + 31) / 32, p.units), 128, 0, st>>>(p);
         bwd_attn_dkv_kernel<T, 128><<<dim3((p.S + 31) / 32, p.units), 128, 0, st>>>(p);
     } else {
@@ -593,7 +593,7 @@ View bdev(const lococo_tensor& t, int64_t tokens, size_t elt) {
 }
 
 struct Scratch {
-    size_t gK, gV, dXK, dXV, dA, delta, total;
+    size_t gK, gV, dXK, dXV, dA, delta, tensor, total;
 };
 
 Scratch scratch_layout(const lococo_handle* h, int B) {
@@ -607,6 +607,8 @@ Scratch scratch_layout(const lococo_handle* h, int B) {
     s.dXV = off;   off = align256(off + units * Smax * c.head_dim * sizeof(float));
     s.dA = off;    off = align256(off + units * c.M * Smax * sizeof(float));
     s.delta = off; off = align256(off + units * (size_t)B * sizeof(float));
+    s.tensor = off;
+    if (tensor_backward_supported(h)) off = align256(off + tensor_backward_scratch_bytes(h, B));
     s.total = off;
     return s;
 }
@@ -652,6 +654,12 @@ lococo_status lococo_process_sequence_backward(lococo_handle* h, lococo_tensor Q
     const char* sv = static_cast<const char*>(saved);
     const float* lse_all = reinterpret_cast<const float*>(sv + 2 * snap_all);
 
+    char* tb = tensor_backward_supported(h) ? sc + sl.tensor : nullptr;
+    if (tb) {
+        const int r = tensor_backward_prepare(h, B, tb, st);
+        if (r < 0) return LOCOCO_ERR_CUDA;
+        h->launches += r;
+    }
     int launched_n = cfg.dtype == LOCOCO_F32
                          ? init_g<float>(bdev(dKc_final, 0, e), bdev(dVc_final, 0, e), gK, gV, cfg.heads, h->units, cfg.M, cfg.head_dim, st)
                          : init_g<__nv_bfloat16>(bdev(dKc_final, 0, e), bdev(dVc_final, 0, e), gK, gV, cfg.heads, h->units, cfg.M,
@@ -698,8 +706,8 @@ lococo_status lococo_process_sequence_backward(lococo_handle* h, lococo_tensor Q
         f.S = p.S; f.weights_per_head = cfg.weights_per_head; f.g_packed = p.g_packed;
         f.bias = h->has_bias ? reinterpret_cast<const float*>(h->ws + h->off_bias) : nullptr;
         f.eps = cfg.norm_eps; f.R = p.R; f.s = p.s;
-        const int r = cfg.dtype == LOCOCO_F32 ? backward_step<float>(p, f, cfg.dtype, st)
-                                              : backward_step<__nv_bfloat16>(p, f, cfg.dtype, st);
+        const int r = cfg.dtype == LOCOCO_F32 ? backward_step<float>(h, p, f, cfg.dtype, B, nullptr, st)
+                                              : backward_step<__nv_bfloat16>(h, p, f, cfg.dtype, B, tb, st);
         if (r < 0) return LOCOCO_ERR_CUDA;
         h->launches += r;
     }

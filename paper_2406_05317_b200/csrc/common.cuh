@@ -57,6 +57,7 @@ struct CompressParams {
     float* UK;             // [units][M][d] unnormalised blends
     float* UV;
     float* W_out;          // optional [units][M][S]
+    int keep_R;            // also leave R in place on paths that would not store it (the backward's recompute)
     void* prof;            // host only: Profiler* or nullptr
 };
 

@@ -4,7 +4,7 @@
 // caller, so "A[m][k]" is whatever the caller's map and coordinate rule make of it: either operand
 // may be K-major (rows of K elements) or MN-major (rows of M/N elements, one row per k), and the
 // coordinates of the box of K step s, output tile (tm, tn) and batch z are affine in
-// (tm, tn % n_inner, tn / n_inner, s % s_inner, s / s_inner, z). That is enough for plain batched
+// (tm, tn % n_inner, tn / n_inner, s % s_inner, s / s_inner, z % z_inner, z / z_inner). That is enough for plain batched
 // GEMMs, for sums over several units (the weight gradient), for row-shifted windows of one tensor
 // (a convolution tap = a row offset; loads may start at negative rows and read zeros there) and for
 // maps with overlapping strides (an im2col view that is never materialised).
@@ -23,8 +23,9 @@ namespace gemm {
 
 using namespace tc;
 
-struct Coord {      // one box coordinate = c0 + tm*TM + tni*(TN % n_inner) + tno*(TN / n_inner) + si*(s % s_inner) + so*(s / s_inner) + z*Z
-    int c0, tm, tni, tno, si, so, z;
+struct Coord {      // one box coordinate = c0 + tm*TM + tni*(TN % n_inner) + tno*(TN / n_inner) + si*(s % s_inner) + so*(s / s_inner)
+                    //                      + zi*(Z % z_inner) + zo*(Z / z_inner)
+    int c0, tm, tni, tno, si, so, zi, zo;
 };
 struct Operand {
     CUtensorMap map;   // K-major: box {64 k, 128 rows}; MN-major: box {64 m/n, 64 k}, loaded at x and x + 64
@@ -35,10 +36,10 @@ struct Operand {
 enum Mode { kStoreF32 = 0, kAtomicF32 = 1, kStoreBF16 = 2, kAddF32 = 3 };
 struct alignas(64) Params {
     Operand A, B;
-    int n_inner, s_inner;        // decomposition of the N tile index and of the K step index
+    int n_inner, s_inner, z_inner;   // decomposition of the N tile index, of the K step index and of the batch index
     int steps, splits;           // K steps (64 wide) in total; CTAs that share them (blockIdx.z = z * splits + split)
     void* out;
-    int64_t out_z, out_m;        // element strides of the batch and of a row
+    int64_t out_zi, out_zo, out_m;   // element strides of batch % z_inner, batch / z_inner and of a row
     int out_n_inner;             // column n lands at (n % out_n_inner) * out_n_in + (n / out_n_inner) * out_n_out
     int64_t out_n_in, out_n_out;
     int M, N;                    // valid rows and columns
@@ -53,8 +54,9 @@ constexpr uint32_t kOperandBytes = 16384;
 constexpr uint32_t kStageBytes2 = 2 * kOperandBytes;
 constexpr uint32_t kSmem = kStages * kStageBytes2 + 1024 + 128;
 
-__device__ __forceinline__ int coord_of(const Coord& c, int tm, int tn, int n_inner, int s, int s_inner, int z) {
-    return c.c0 + c.tm * tm + c.tni * (tn % n_inner) + c.tno * (tn / n_inner) + c.si * (s % s_inner) + c.so * (s / s_inner) + c.z * z;
+__device__ __forceinline__ int coord_of(const Coord& c, const Params& P, int tm, int tn, int s, int z) {
+    return c.c0 + c.tm * tm + c.tni * (tn % P.n_inner) + c.tno * (tn / P.n_inner) + c.si * (s % P.s_inner) + c.so * (s / P.s_inner) +
+           c.zi * (z % P.z_inner) + c.zo * (z / P.z_inner);
 }
 
 __global__ void __launch_bounds__(kThreads, 2) gemm_kernel(const __grid_constant__ Params P) {
@@ -99,10 +101,8 @@ __global__ void __launch_bounds__(kThreads, 2) gemm_kernel(const __grid_constant
             for (int op = 0; op < 2; ++op) {
                 const Operand& O = op ? P.B : P.A;
                 const uint32_t d = dst + op * kOperandBytes;
-                const int tile = op ? tn : tm;
-                (void)tile;
-                const int x = coord_of(O.c[0], tm, tn, P.n_inner, s, P.s_inner, z), y = coord_of(O.c[1], tm, tn, P.n_inner, s, P.s_inner, z);
-                const int c2 = coord_of(O.c[2], tm, tn, P.n_inner, s, P.s_inner, z), c3 = coord_of(O.c[3], tm, tn, P.n_inner, s, P.s_inner, z);
+                const int x = coord_of(O.c[0], P, tm, tn, s, z), y = coord_of(O.c[1], P, tm, tn, s, z);
+                const int c2 = coord_of(O.c[2], P, tm, tn, s, z), c3 = coord_of(O.c[3], P, tm, tn, s, z);
                 if (O.mn_major) {
                     tma_load_4d(d, &O.map, x, y, c2, c3, bar_full + 8 * st);
                     tma_load_4d(d + kOperandBytes / 2, &O.map, x + 64, y, c2, c3, bar_full + 8 * st);
@@ -140,7 +140,7 @@ __global__ void __launch_bounds__(kThreads, 2) gemm_kernel(const __grid_constant
         }
         const int row = tm * 128 + tid;
         const uint32_t lane_addr = tmem + ((uint32_t)(warp * 32) << 16);
-        const int64_t base = (int64_t)z * P.out_z + (int64_t)row * P.out_m;
+        const int64_t base = (int64_t)(z % P.z_inner) * P.out_zi + (int64_t)(z / P.z_inner) * P.out_zo + (int64_t)row * P.out_m;
         const bool contiguous = P.out_n_in == 1 && P.out_n_inner % 32 == 0;
 #pragma unroll 1
         for (int c0 = 0; c0 < 128; c0 += 32) {

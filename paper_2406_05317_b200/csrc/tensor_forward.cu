@@ -1017,7 +1017,7 @@ static bool build_compress_params(lococo_handle* h, const CompressParams& p, boo
     P.gimage = reinterpret_cast<const __nv_bfloat16*>(h->ws + h->off_gimage);
     P.part_U = reinterpret_cast<float*>(h->ws + h->off_part);
     P.part_s = P.part_U + (size_t)p.units * SB * max_parts * 2 * kSlots * kD;
-    P.R_store = p.W_out ? p.R : nullptr;
+    P.R_store = (p.W_out || p.keep_R) ? p.R : nullptr;
     P.status = reinterpret_cast<int*>(h->ws + h->off_status);
     P.n_tile = pl.n_tile; P.tiles = pl.tiles; P.parts = pl.parts; P.tiles_per_part = pl.tiles_per_part;
     P.part_stride = fused ? max_parts : pl.parts;   // fixed regions where steps with different plans share a launch
