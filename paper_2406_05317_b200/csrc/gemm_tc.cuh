@@ -33,7 +33,9 @@ struct Operand {
     int mn_major;
     int pad[3];
 };
-enum Mode { kStoreF32 = 0, kAtomicF32 = 1, kStoreBF16 = 2, kAddF32 = 3 };
+// kSoftmaxBF16: out = exp2(acc * scale2 - rowvec[row] * log2 e) where column < causal_c + row + 1, else 0 (bf16)
+// kDsBF16:      out = aux * (acc - rowvec[row]) * alpha             under the same mask (aux: bf16, laid out like out)
+enum Mode { kStoreF32 = 0, kAtomicF32 = 1, kStoreBF16 = 2, kAddF32 = 3, kSoftmaxBF16 = 4, kDsBF16 = 5 };
 struct alignas(64) Params {
     Operand A, B;
     int n_inner, s_inner, z_inner;   // decomposition of the N tile index, of the K step index and of the batch index
@@ -46,6 +48,15 @@ struct alignas(64) Params {
     int mode;
     float alpha;
     int* status;
+    // causal structure (rows = queries, columns = keys; row r sees columns < causal_c + r + 1)
+    int causal_tiles;            // 1: output tiles entirely beyond the limit skip their K loop (and come out as zeros)
+    int causal_c;
+    int k_lo_on, k_lo_c0;        // K loop starts at step max(0, (tm * 128 + k_lo_c0) / 64)
+    int k_hi_on, k_hi_c0;        // K loop ends before step (tm * 128 + k_hi_c0 + 63) / 64
+    const float* rowvec;         // per (batch, row) value of the two fused modes
+    int64_t rowvec_z;
+    const void* aux;
+    float scale2;
 };
 
 constexpr int kThreads = 192;
@@ -70,7 +81,11 @@ __global__ void __launch_bounds__(kThreads, 2) gemm_kernel(const __grid_constant
     const int tm = blockIdx.x, tn = blockIdx.y;
     const int z = blockIdx.z / P.splits, split = blockIdx.z % P.splits;
     const int per = (P.steps + P.splits - 1) / P.splits;
-    const int s_begin = split * per, s_end = min(P.steps, s_begin + per);
+    int s_begin = split * per, s_end = min(P.steps, s_begin + per);
+    if (P.k_lo_on) s_begin = max(s_begin, max(0, tm * 128 + P.k_lo_c0) / 64);
+    if (P.k_hi_on) s_end = min(s_end, max(0, tm * 128 + P.k_hi_c0 + 63) / 64);
+    if (P.causal_tiles && tn * 128 >= P.causal_c + tm * 128 + 128) s_end = s_begin;
+    if (s_end < s_begin) s_end = s_begin;
 
     if (tid == 128) {
         for (int s = 0; s < kStages; ++s) {
@@ -142,6 +157,11 @@ __global__ void __launch_bounds__(kThreads, 2) gemm_kernel(const __grid_constant
         const uint32_t lane_addr = tmem + ((uint32_t)(warp * 32) << 16);
         const int64_t base = (int64_t)(z % P.z_inner) * P.out_zi + (int64_t)(z / P.z_inner) * P.out_zo + (int64_t)row * P.out_m;
         const bool contiguous = P.out_n_in == 1 && P.out_n_inner % 32 == 0;
+        const bool fused = P.mode == kSoftmaxBF16 || P.mode == kDsBF16;
+        const int mode = fused ? (int)kStoreBF16 : P.mode;
+        const float alpha = fused ? 1.f : P.alpha;
+        const float rv = fused && row < P.M ? P.rowvec[(int64_t)z * P.rowvec_z + row] : 0.f;
+        const int vis = P.causal_c + row + 1;
 #pragma unroll 1
         for (int c0 = 0; c0 < 128; c0 += 32) {
             uint32_t v[32];
@@ -153,36 +173,63 @@ __global__ void __launch_bounds__(kThreads, 2) gemm_kernel(const __grid_constant
                 for (int e = 0; e < 32; ++e) v[e] = 0u;
             }
             const int n0 = tn * 128 + c0;
-            if (row >= P.M || n0 >= P.N || (!any && P.mode != kStoreF32 && P.mode != kStoreBF16)) continue;
+            if (row >= P.M || n0 >= P.N || (!any && mode != kStoreF32 && mode != kStoreBF16)) continue;
             const int64_t col0 = (int64_t)(n0 % P.out_n_inner) * P.out_n_in + (int64_t)(n0 / P.out_n_inner) * P.out_n_out;
+            if (P.mode == kSoftmaxBF16) {
+                const float l2 = rv * 1.4426950408889634f;
+#pragma unroll
+                for (int e = 0; e < 32; ++e)
+                    v[e] = __float_as_uint(n0 + e < vis ? exp2f(__uint_as_float(v[e]) * P.scale2 - l2) : 0.f);
+            } else if (P.mode == kDsBF16) {
+                const __nv_bfloat16* a = static_cast<const __nv_bfloat16*>(P.aux) + base + col0;
+                if (n0 + 32 <= P.N) {
+#pragma unroll
+                    for (int e = 0; e < 32; e += 8) {
+                        const uint4 q = *reinterpret_cast<const uint4*>(a + e);
+                        const uint32_t w[4] = {q.x, q.y, q.z, q.w};
+#pragma unroll
+                        for (int x = 0; x < 8; ++x) {
+                            const float pr = n0 + e + x < vis ? __uint_as_float((x & 1) ? (w[x >> 1] & 0xffff0000u) : (w[x >> 1] << 16)) : 0.f;
+                            v[e + x] = __float_as_uint(pr * (__uint_as_float(v[e + x]) - rv) * P.alpha);
+                        }
+                    }
+                } else {
+#pragma unroll 1
+                    for (int e = 0; e < 32; ++e) {
+                        float pr = 0.f;
+                        if (n0 + e < vis && n0 + e < P.N) pr = __bfloat162float(a[e]);
+                        v[e] = __float_as_uint(pr * (__uint_as_float(v[e]) - rv) * P.alpha);
+                    }
+                }
+            }
             if (contiguous && n0 + 32 <= P.N) {
-                if (P.mode == kStoreF32) {
+                if (mode == kStoreF32) {
                     float4* o = reinterpret_cast<float4*>(static_cast<float*>(P.out) + base + col0);
 #pragma unroll
                     for (int e = 0; e < 32; e += 4)
-                        o[e >> 2] = make_float4(__uint_as_float(v[e]) * P.alpha, __uint_as_float(v[e + 1]) * P.alpha,
-                                                __uint_as_float(v[e + 2]) * P.alpha, __uint_as_float(v[e + 3]) * P.alpha);
-                } else if (P.mode == kAddF32) {
+                        o[e >> 2] = make_float4(__uint_as_float(v[e]) * alpha, __uint_as_float(v[e + 1]) * alpha,
+                                                __uint_as_float(v[e + 2]) * alpha, __uint_as_float(v[e + 3]) * alpha);
+                } else if (mode == kAddF32) {
                     float4* o = reinterpret_cast<float4*>(static_cast<float*>(P.out) + base + col0);
 #pragma unroll
                     for (int e = 0; e < 32; e += 4) {
                         float4 t = o[e >> 2];
-                        t.x += __uint_as_float(v[e]) * P.alpha; t.y += __uint_as_float(v[e + 1]) * P.alpha;
-                        t.z += __uint_as_float(v[e + 2]) * P.alpha; t.w += __uint_as_float(v[e + 3]) * P.alpha;
+                        t.x += __uint_as_float(v[e]) * alpha; t.y += __uint_as_float(v[e + 1]) * alpha;
+                        t.z += __uint_as_float(v[e + 2]) * alpha; t.w += __uint_as_float(v[e + 3]) * alpha;
                         o[e >> 2] = t;
                     }
-                } else if (P.mode == kStoreBF16) {
+                } else if (mode == kStoreBF16) {
                     uint4* o = reinterpret_cast<uint4*>(static_cast<__nv_bfloat16*>(P.out) + base + col0);
 #pragma unroll
                     for (int e = 0; e < 32; e += 8)
-                        o[e >> 3] = make_uint4(pack_bf16(__uint_as_float(v[e]) * P.alpha, __uint_as_float(v[e + 1]) * P.alpha),
-                                               pack_bf16(__uint_as_float(v[e + 2]) * P.alpha, __uint_as_float(v[e + 3]) * P.alpha),
-                                               pack_bf16(__uint_as_float(v[e + 4]) * P.alpha, __uint_as_float(v[e + 5]) * P.alpha),
-                                               pack_bf16(__uint_as_float(v[e + 6]) * P.alpha, __uint_as_float(v[e + 7]) * P.alpha));
+                        o[e >> 3] = make_uint4(pack_bf16(__uint_as_float(v[e]) * alpha, __uint_as_float(v[e + 1]) * alpha),
+                                               pack_bf16(__uint_as_float(v[e + 2]) * alpha, __uint_as_float(v[e + 3]) * alpha),
+                                               pack_bf16(__uint_as_float(v[e + 4]) * alpha, __uint_as_float(v[e + 5]) * alpha),
+                                               pack_bf16(__uint_as_float(v[e + 6]) * alpha, __uint_as_float(v[e + 7]) * alpha));
                 } else {
                     float* o = static_cast<float*>(P.out) + base + col0;
 #pragma unroll
-                    for (int e = 0; e < 32; ++e) atomicAdd(o + e, __uint_as_float(v[e]) * P.alpha);
+                    for (int e = 0; e < 32; ++e) atomicAdd(o + e, __uint_as_float(v[e]) * alpha);
                 }
             } else {
 #pragma unroll 1
@@ -190,10 +237,10 @@ __global__ void __launch_bounds__(kThreads, 2) gemm_kernel(const __grid_constant
                     const int n = n0 + e;
                     if (n >= P.N) break;
                     const int64_t col = (int64_t)(n % P.out_n_inner) * P.out_n_in + (int64_t)(n / P.out_n_inner) * P.out_n_out;
-                    const float x = __uint_as_float(v[e]) * P.alpha;
-                    if (P.mode == kStoreF32) static_cast<float*>(P.out)[base + col] = x;
-                    else if (P.mode == kAddF32) static_cast<float*>(P.out)[base + col] += x;
-                    else if (P.mode == kStoreBF16) static_cast<__nv_bfloat16*>(P.out)[base + col] = __float2bfloat16_rn(x);
+                    const float x = __uint_as_float(v[e]) * alpha;
+                    if (mode == kStoreF32) static_cast<float*>(P.out)[base + col] = x;
+                    else if (mode == kAddF32) static_cast<float*>(P.out)[base + col] += x;
+                    else if (mode == kStoreBF16) static_cast<__nv_bfloat16*>(P.out)[base + col] = __float2bfloat16_rn(x);
                     else atomicAdd(static_cast<float*>(P.out) + base + col, x);
                 }
             }

@@ -9,9 +9,10 @@
 //     dG         += sum over units and positions of dA (*) Z          the im2col view of Z is a tensor
 //                                                                     map with overlapping strides
 //     dZ (in dX) += sum over taps of shift_t(dA^T) G_t                a tap = a row offset of the box
-//   attention (Eq. 1 reversed), in blocks of up to 1024 queries, logits and probabilities materialised:
-//     Sraw = Q X_K^T, dP = dO X_V^T, P = exp(scale Sraw - lse), dS = scale P (dP - delta)
-//     dX_V += P^T dO, dX_K += dS^T Q, dQ = dS X_K
+//   attention (Eq. 1 reversed), in blocks of up to 1024 queries, P and dS materialised in bf16:
+//     P = exp(scale Q X_K^T - lse), dS = scale P (dO X_V^T - delta)   softmax and its gradient fused into the
+//                                                                     GEMM epilogues; masked tiles skipped
+//     dX_V += P^T dO, dX_K += dS^T Q, dQ = dS X_K                     K loops cut at the causal limit
 // Gradients that enter a GEMM are rounded to bf16 (fp32 accumulation), like the forward's operands.
 #include <algorithm>
 
@@ -30,7 +31,7 @@ int round_up(int x, int m) { return (x + m - 1) / m * m; }
 
 struct Layout {
     int Sp, Sp2, QB;
-    size_t xpad, gkv, wb, dab, dat, gt, dummy_k, dummy_v, dw, sraw, dpf, pb, dsb, total;
+    size_t xpad, gkv, wb, dab, dat, gt, dummy_k, dummy_v, dw, pb, dsb, total;
 };
 
 Layout layout_of(const lococo_handle* h, int B) {
@@ -52,8 +53,6 @@ Layout layout_of(const lococo_handle* h, int B) {
     L.dummy_k = take(U * c.M * kD * 2);
     L.dummy_v = take(U * c.M * kD * 2);
     L.dw = take(U * c.M * L.Sp * 4);
-    L.sraw = take(U * (size_t)L.QB * L.Sp * 4);
-    L.dpf = take(U * (size_t)L.QB * L.Sp * 4);
     L.pb = take(U * (size_t)L.QB * L.Sp * 2);
     L.dsb = take(U * (size_t)L.QB * L.Sp * 2);
     L.total = off;
@@ -154,27 +153,6 @@ __global__ void __launch_bounds__(256) transpose_kernel(const __nv_bfloat16* in,
         const int j = j0 + r;
         if (j < Sp) out[((int64_t)u * Sp + j) * M + i0 + tx] = tile[tx][r];
     }
-}
-
-// One block per (unit, query row of the block): P and dS in bf16, zero at and beyond the causal limit.
-__global__ void __launch_bounds__(256) attn_row_kernel(BwdStep p, const float* sraw, const float* dpf, __nv_bfloat16* pb,
-                                                       __nv_bfloat16* dsb, int q0, int qb, int QB, int Sp) {
-    const int u = blockIdx.y, r = blockIdx.x;
-    const int64_t row = ((int64_t)u * QB + r) * Sp;
-    const int vis = p.c + q0 + r + 1;
-    const float lse = p.lse[(int64_t)u * p.lse_stride + q0 + r] * 1.4426950408889634f;
-    const float delta = p.delta[(int64_t)u * p.b + q0 + r];
-    const float sc2 = p.scale * 1.4426950408889634f;
-    for (int j = threadIdx.x; j < Sp; j += 256) {
-        float P = 0.f, dS = 0.f;
-        if (j < vis) {
-            P = exp2f(sraw[row + j] * sc2 - lse);
-            dS = P * (dpf[row + j] - delta) * p.scale;
-        }
-        pb[row + j] = __float2bfloat16_rn(P);
-        dsb[row + j] = __float2bfloat16_rn(dS);
-    }
-    (void)qb;
 }
 
 // ------------------------------------------------------------------ GEMM set-up helpers
@@ -336,8 +314,6 @@ int tensor_backward_attention(lococo_handle* h, const BwdStep& p, int B, char* s
     const Layout L = layout_of(h, B);
     const int U = p.units, H = p.heads, batch = U / H, S = p.S, pad = (p.k - 1) / 2;
     __nv_bfloat16* xpad = reinterpret_cast<__nv_bfloat16*>(sc + L.xpad);
-    float* sraw = reinterpret_cast<float*>(sc + L.sraw);
-    float* dpf = reinterpret_cast<float*>(sc + L.dpf);
     __nv_bfloat16* pb = reinterpret_cast<__nv_bfloat16*>(sc + L.pb);
     __nv_bfloat16* dsb = reinterpret_cast<__nv_bfloat16*>(sc + L.dsb);
     const Tensor4 t_xpad{xpad, {256, (uint64_t)L.Sp2, (uint64_t)U, 1}, {512, (uint64_t)L.Sp2 * 512, (uint64_t)U * L.Sp2 * 512}};
@@ -348,23 +324,30 @@ int tensor_backward_attention(lococo_handle* h, const BwdStep& p, int B, char* s
         const int qb = std::min(L.QB, p.b - q0), q_tiles = (qb + 127) / 128;
         const int Sv = std::min(S, p.c + q0 + qb);          // keys any query of the block can see
         const int sv_tiles = (Sv + 127) / 128;
-        for (int which = 0; which < 2; ++which) {           // Sraw = Q X_K^T, dP = dO X_V^T
+        // P = exp(scale Q X_K^T - lse) and dS = scale P (dO X_V^T - delta): the softmax and its gradient are
+        // applied to the accumulator tile, under the causal mask, and only bf16 P and dS reach memory
+        for (int which = 0; which < 2; ++which) {
             gemm::Params G = base_params(h);
             if (!operand(G.A, which ? t_do : t_q, false) || !operand(G.B, t_xpad, false)) return -1;
             G.z_inner = H;
             G.A.c[0].si = 64; G.A.c[1].c0 = q0; G.A.c[1].tm = 128; G.A.c[2].zi = 1; G.A.c[3].zo = 1;
             G.B.c[0].c0 = which * kD; G.B.c[0].si = 64; G.B.c[1].c0 = pad; G.B.c[1].tni = 128; G.B.c[2].zi = 1; G.B.c[2].zo = H;
             G.steps = 2;
-            G.out = which ? dpf : sraw; G.out_zi = (int64_t)L.QB * L.Sp; G.out_zo = (int64_t)H * L.QB * L.Sp; G.out_m = L.Sp;
-            G.M = qb; G.N = Sv; G.mode = gemm::kStoreF32;
+            G.out = which ? dsb : pb; G.out_zi = (int64_t)L.QB * L.Sp; G.out_zo = (int64_t)H * L.QB * L.Sp; G.out_m = L.Sp;
+            G.M = qb; G.N = Sv;
+            G.causal_tiles = 1; G.causal_c = p.c + q0;
+            if (which) {
+                G.mode = gemm::kDsBF16; G.aux = pb; G.alpha = p.scale;
+                G.rowvec = p.delta + q0; G.rowvec_z = p.b;
+            } else {
+                G.mode = gemm::kSoftmaxBF16; G.scale2 = p.scale * 1.4426950408889634f;
+                G.rowvec = p.lse + q0; G.rowvec_z = p.lse_stride;
+            }
             if (!gemm::launch(G, q_tiles, sv_tiles, U, st)) return -1;
             ++n;
         }
-        attn_row_kernel<<<dim3(qb, U), 256, 0, st>>>(p, sraw, dpf, pb, dsb, q0, qb, L.QB, L.Sp);
-        if (!launched()) return -1;
-        ++n;
-        const Tensor4 t_pb{pb, {(uint64_t)L.Sp, (uint64_t)qb, (uint64_t)U, 1}, {(uint64_t)L.Sp * 2, (uint64_t)L.QB * L.Sp * 2, (uint64_t)U * L.QB * L.Sp * 2}};
-        const Tensor4 t_dsb{dsb, {(uint64_t)L.Sp, (uint64_t)qb, (uint64_t)U, 1}, {(uint64_t)L.Sp * 2, (uint64_t)L.QB * L.Sp * 2, (uint64_t)U * L.QB * L.Sp * 2}};
+        const Tensor4 t_pb{pb, {(uint64_t)Sv, (uint64_t)qb, (uint64_t)U, 1}, {(uint64_t)L.Sp * 2, (uint64_t)L.QB * L.Sp * 2, (uint64_t)U * L.QB * L.Sp * 2}};
+        const Tensor4 t_dsb{dsb, {(uint64_t)Sv, (uint64_t)qb, (uint64_t)U, 1}, {(uint64_t)L.Sp * 2, (uint64_t)L.QB * L.Sp * 2, (uint64_t)U * L.QB * L.Sp * 2}};
         for (int which = 0; which < 2; ++which) {           // dX_V += P^T dO, dX_K += dS^T Q
             gemm::Params G = base_params(h);
             if (!operand(G.A, which ? t_dsb : t_pb, true) || !operand(G.B, which ? t_q : t_do, true)) return -1;
@@ -372,6 +355,7 @@ int tensor_backward_attention(lococo_handle* h, const BwdStep& p, int B, char* s
             G.A.c[0].tm = 128; G.A.c[1].si = 64; G.A.c[2].zi = 1; G.A.c[2].zo = H;
             G.B.c[0].tni = 128; G.B.c[1].c0 = q0; G.B.c[1].si = 64; G.B.c[2].zi = 1; G.B.c[3].zo = 1;
             G.steps = (qb + 63) / 64;
+            G.k_lo_on = 1; G.k_lo_c0 = -(p.c + q0);          // query rows that cannot see this key tile contribute nothing
             G.out = which ? p.dXK : p.dXV; G.out_zi = (int64_t)S * kD; G.out_zo = (int64_t)H * S * kD; G.out_m = kD;
             G.M = Sv; G.N = kD; G.mode = gemm::kAddF32;
             if (!gemm::launch(G, sv_tiles, 1, U, st)) return -1;
@@ -384,6 +368,7 @@ int tensor_backward_attention(lococo_handle* h, const BwdStep& p, int B, char* s
             G.A.c[0].si = 64; G.A.c[1].tm = 128; G.A.c[2].zi = 1; G.A.c[2].zo = H;
             G.B.c[0].tni = 128; G.B.c[1].c0 = pad; G.B.c[1].si = 64; G.B.c[2].zi = 1; G.B.c[2].zo = H;
             G.steps = (Sv + 63) / 64;
+            G.k_hi_on = 1; G.k_hi_c0 = p.c + q0 + 128;       // keys beyond the last query of the tile are masked
             G.out = reinterpret_cast<__nv_bfloat16*>(p.dq.ptr) + (int64_t)q0 * p.dq.st;
             G.out_zi = p.dq.sh; G.out_zo = p.dq.sb; G.out_m = p.dq.st;
             G.M = qb; G.N = kD; G.mode = gemm::kStoreBF16;
