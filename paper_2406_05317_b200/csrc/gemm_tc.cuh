@@ -8,8 +8,8 @@
 // GEMMs, for sums over several units (the weight gradient), for row-shifted windows of one tensor
 // (a convolution tap = a row offset; loads may start at negative rows and read zeros there) and for
 // maps with overlapping strides (an im2col view that is never materialised).
-// One CTA = one 128 x 128 output tile: warp 5 lane 0 feeds a 3-stage ring (32 KB per stage), warp 4
-// lane 0 issues four K=16 MMAs per stage into 128 TMEM columns, warps 0-3 write the tile out.
+// One CTA = one 128 x 128 output tile: one lane feeds a 3-stage ring (32 KB per stage), one lane issues
+// four K=16 MMAs per stage into 128 TMEM columns, eight warps write the tile out (two per 32 rows).
 // Two CTAs fit an SM, so one tile's epilogue overlaps the other's main loop.
 #pragma once
 #include <cuda.h>
@@ -59,7 +59,7 @@ struct alignas(64) Params {
     float scale2;
 };
 
-constexpr int kThreads = 192;
+constexpr int kThreads = 320;                      // 8 epilogue warps, the MMA-issue warp, the producer warp
 constexpr int kStages = 3;
 constexpr uint32_t kOperandBytes = 16384;
 constexpr uint32_t kStageBytes2 = 2 * kOperandBytes;
@@ -87,7 +87,7 @@ __global__ void __launch_bounds__(kThreads, 2) gemm_kernel(const __grid_constant
     if (P.causal_tiles && tn * 128 >= P.causal_c + tm * 128 + 128) s_end = s_begin;
     if (s_end < s_begin) s_end = s_begin;
 
-    if (tid == 128) {
+    if (tid == 256) {
         for (int s = 0; s < kStages; ++s) {
             mbar_init(bar_full + 8 * s, 1);
             mbar_init(bar_empty + 8 * s, 1);
@@ -105,7 +105,7 @@ __global__ void __launch_bounds__(kThreads, 2) gemm_kernel(const __grid_constant
     tc_fence_after();
     const uint32_t tmem = *reinterpret_cast<volatile uint32_t*>(&tmem_slot);
 
-    if (tid == 160) {
+    if (tid == 288) {
         // ---- producer
         for (int s = s_begin, g = 0; s < s_end; ++s, ++g) {
             const int st = g % kStages;
@@ -126,7 +126,7 @@ __global__ void __launch_bounds__(kThreads, 2) gemm_kernel(const __grid_constant
                 }
             }
         }
-    } else if (tid == 128) {
+    } else if (tid == 256) {
         // ---- MMA issuer
         const uint32_t idesc = instr_desc_bf16(128, P.A.mn_major != 0, P.B.mn_major != 0);
         for (int s = s_begin, g = 0; s < s_end; ++s, ++g) {
@@ -145,7 +145,7 @@ __global__ void __launch_bounds__(kThreads, 2) gemm_kernel(const __grid_constant
         }
         umma_commit(bar_acc);
     }
-    if (warp < 4) {
+    if (warp < 8) {
         // ---- epilogue: thread = one row of the tile
         __syncwarp();
         const bool any = s_end > s_begin;
@@ -153,8 +153,10 @@ __global__ void __launch_bounds__(kThreads, 2) gemm_kernel(const __grid_constant
             mbar_wait(bar_acc, 0, P.status, failed, 32);
             tc_fence_after();
         }
-        const int row = tm * 128 + tid;
-        const uint32_t lane_addr = tmem + ((uint32_t)(warp * 32) << 16);
+        // warp w reads TMEM lanes 32 * (w % 4) ..., i.e. those rows of the tile; warps 4-7 take columns 64-127
+        const int row = tm * 128 + (tid & 127);
+        const uint32_t lane_addr = tmem + ((uint32_t)((warp & 3) * 32) << 16);
+        const int c_begin = (tid >> 7) * 64;
         const int64_t base = (int64_t)(z % P.z_inner) * P.out_zi + (int64_t)(z / P.z_inner) * P.out_zo + (int64_t)row * P.out_m;
         const bool contiguous = P.out_n_in == 1 && P.out_n_inner % 32 == 0;
         const bool fused = P.mode == kSoftmaxBF16 || P.mode == kDsBF16;
@@ -163,7 +165,7 @@ __global__ void __launch_bounds__(kThreads, 2) gemm_kernel(const __grid_constant
         const float rv = fused && row < P.M ? P.rowvec[(int64_t)z * P.rowvec_z + row] : 0.f;
         const int vis = P.causal_c + row + 1;
 #pragma unroll 1
-        for (int c0 = 0; c0 < 128; c0 += 32) {
+        for (int c0 = c_begin; c0 < c_begin + 64; c0 += 32) {
             uint32_t v[32];
             if (any) {
                 tmem_ld32(lane_addr + c0, v);
@@ -249,7 +251,7 @@ __global__ void __launch_bounds__(kThreads, 2) gemm_kernel(const __grid_constant
     tc_fence_before();
     __syncthreads();
     if (warp == 0) tmem_dealloc(tmem, 128);
-    if (tid == 128) {
+    if (tid == 256) {
         for (int s = 0; s < 2 * kStages + 1; ++s) mbar_inval(bar_full + 8 * s);
     }
 }
