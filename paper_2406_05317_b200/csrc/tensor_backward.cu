@@ -4,8 +4,8 @@
 //   cache update (Eq. 4-7 reversed)
 //     R, s        recomputed by the forward's own tcgen05 conv kernel (R left in place)
 //     dw          = [gK | gV] [X_K | X_V]^T                          per unit, K = 2d
-//     dA, w       row kernel: dA = [R>0] (dw - <dw, w>_row) / s, w = R / s, both rounded to bf16
-//     dX         += w^T [gK | gV]                                     per unit, K = M
+//     dA          row kernel: dA = [R>0] (dw - <dw, w>_row) / s with w = R / s, rounded to bf16
+//     dX         += w^T [gK | gV] = R^T ([gK | gV] / s)               per unit, K = M; R is exact in bf16
 //     dG         += sum over units and positions of dA (*) Z          the im2col view of Z is a tensor
 //                                                                     map with overlapping strides
 //     dZ (in dX) += sum over taps of shift_t(dA^T) G_t                a tap = a row offset of the box
@@ -13,7 +13,8 @@
 //     P = exp(scale Q X_K^T - lse), dS = scale P (dO X_V^T - delta)   softmax and its gradient fused into the
 //                                                                     GEMM epilogues; masked tiles skipped
 //     dX_V += P^T dO, dX_K += dS^T Q, dQ = dS X_K                     K loops cut at the causal limit
-// Gradients that enter a GEMM are rounded to bf16 (fp32 accumulation), like the forward's operands.
+// Gradients that enter a GEMM are rounded to bf16 (fp32 accumulation), like the forward's operands; the
+// cache gradient, which every earlier step inherits, enters as two bf16 terms (value + remainder).
 #include <algorithm>
 
 #include "backward.h"
@@ -31,7 +32,7 @@ int round_up(int x, int m) { return (x + m - 1) / m * m; }
 
 struct Layout {
     int Sp, Sp2, QB;
-    size_t xpad, gkv, wb, dab, dat, gt, dummy_k, dummy_v, dw, pb, dsb, total;
+    size_t xpad, gkv, gkv_lo, gs, gs_lo, wb, dab, dat, gt, dummy_k, dummy_v, dw, pb, dsb, total;
 };
 
 Layout layout_of(const lococo_handle* h, int B) {
@@ -46,6 +47,9 @@ Layout layout_of(const lococo_handle* h, int B) {
     auto take = [&](size_t bytes) { const size_t o = off; off = align256(off + bytes); return o; };
     L.xpad = take(U * L.Sp2 * 256 * 2);
     L.gkv = take(U * c.M * 256 * 2);
+    L.gkv_lo = take(U * c.M * 256 * 2);
+    L.gs = take(U * c.M * 256 * 2);
+    L.gs_lo = take(U * c.M * 256 * 2);
     L.wb = take(U * c.M * L.Sp * 2);
     L.dab = take(U * c.M * L.Sp * 2);
     L.dat = take(U * (size_t)L.Sp * c.M * 2);
@@ -77,13 +81,25 @@ __global__ void pack_x_kernel(BwdStep p, __nv_bfloat16* xpad, int Sp2, int pad) 
     }
 }
 
-// gKV[u][i] = [gK[u][i] | gV[u][i]] in bf16.
-__global__ void pack_g_kernel(const float* gK, const float* gV, __nv_bfloat16* gkv, int64_t rows) {
+// gKV[u][i] = [gK[u][i] | gV[u][i]] in bf16, and the part of it that bf16 drops, also in bf16: dw is
+// followed by the subtraction dw - <dw, w> (Eq. 7 reversed), which cancels most of it, so dw is
+// computed from both parts (two GEMMs) and carries the gradient to about 16 bits.
+// The same split of g / s (row i divided by the denominator s_i of Eq. 7): the blend's own gradient is
+// dX = w^T g = R^T (g / s), and R is exact in bf16 (the forward rounded it), so that GEMM loses nothing.
+__global__ void pack_g_kernel(const float* gK, const float* gV, const float* s, __nv_bfloat16* gkv, __nv_bfloat16* gkv_lo,
+                              __nv_bfloat16* gs, __nv_bfloat16* gs_lo, int64_t rows) {
     const int64_t total = rows * 256;
     for (int64_t x = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; x < total; x += (int64_t)gridDim.x * blockDim.x) {
         const int64_t r = x / 256;
         const int ch = (int)(x % 256);
-        gkv[x] = __float2bfloat16_rn(ch < kD ? gK[r * kD + ch] : gV[r * kD + ch - kD]);
+        const float g = ch < kD ? gK[r * kD + ch] : gV[r * kD + ch - kD];
+        const __nv_bfloat16 hi = __float2bfloat16_rn(g);
+        gkv[x] = hi;
+        gkv_lo[x] = __float2bfloat16_rn(g - __bfloat162float(hi));
+        const float q = g / s[r];
+        const __nv_bfloat16 qh = __float2bfloat16_rn(q);
+        gs[x] = qh;
+        gs_lo[x] = __float2bfloat16_rn(q - __bfloat162float(qh));
     }
 }
 
@@ -97,8 +113,8 @@ __global__ void pack_gt_kernel(const __nv_bfloat16* gp, __nv_bfloat16* gt, int M
     for (int r = threadIdx.y; r < 32; r += blockDim.y) gt[plane + (int64_t)(c0 + r) * M + i0 + threadIdx.x] = tile[threadIdx.x][r];
 }
 
-// One block per (unit, slot) row: dA = [R>0] (dw - <dw, w>) / s, w = R / s (Eq. 7 reversed), both in bf16
-// and zero from column S up to the row stride; dbias += sum of dA.
+// One block per (unit, slot) row: dA = [R>0] (dw - <dw, w>) / s with w = R / s (Eq. 7 reversed), in bf16,
+// and R itself as bf16 (exact); both zero from column S up to the row stride; dbias += sum of dA.
 __global__ void __launch_bounds__(256) da_row_kernel(BwdStep p, const float* dw, __nv_bfloat16* dab, __nv_bfloat16* wb, int Sp) {
     __shared__ float red[8];
     const int64_t row = blockIdx.x;                          // u * M + i
@@ -118,7 +134,7 @@ __global__ void __launch_bounds__(256) da_row_kernel(BwdStep p, const float* dw,
         float da = 0.f, w = 0.f;
         if (j < p.S) {
             const float r = Rr[j];
-            w = r * inv_s;
+            w = r;
             da = r > 0.f ? (dwr[j] - dot) * inv_s : 0.f;
         }
         dab[row * Sp + j] = __float2bfloat16_rn(da);
@@ -217,6 +233,7 @@ int tensor_backward_compress(lococo_handle* h, const BwdStep& p, const CompressP
     const int sets = p.weights_per_head ? H : 1, in_set = U / sets;
     __nv_bfloat16* xpad = reinterpret_cast<__nv_bfloat16*>(sc + L.xpad);
     __nv_bfloat16* gkv = reinterpret_cast<__nv_bfloat16*>(sc + L.gkv);
+    __nv_bfloat16* gkv_lo = reinterpret_cast<__nv_bfloat16*>(sc + L.gkv_lo);
     __nv_bfloat16* wb = reinterpret_cast<__nv_bfloat16*>(sc + L.wb);
     __nv_bfloat16* dab = reinterpret_cast<__nv_bfloat16*>(sc + L.dab);
     __nv_bfloat16* dat = reinterpret_cast<__nv_bfloat16*>(sc + L.dat);
@@ -234,7 +251,8 @@ int tensor_backward_compress(lococo_handle* h, const BwdStep& p, const CompressP
     if (r < 0) return -1;
     n += r;
 
-    pack_g_kernel<<<std::min<int64_t>(((int64_t)U * M * 256 + 255) / 256, 4096), 256, 0, st>>>(p.gK, p.gV, gkv, (int64_t)U * M);
+    pack_g_kernel<<<std::min<int64_t>(((int64_t)U * M * 256 + 255) / 256, 4096), 256, 0, st>>>(p.gK, p.gV, p.s, gkv, gkv_lo, reinterpret_cast<__nv_bfloat16*>(sc + L.gs),
+                                                                                       reinterpret_cast<__nv_bfloat16*>(sc + L.gs_lo), (int64_t)U * M);
     if (!launched()) return -1;
     ++n;
 
@@ -242,14 +260,15 @@ int tensor_backward_compress(lococo_handle* h, const BwdStep& p, const CompressP
     const Tensor4 t_xpad{xpad, {256, (uint64_t)L.Sp2, (uint64_t)U, 1}, {512, (uint64_t)L.Sp2 * 512, (uint64_t)U * L.Sp2 * 512}};
     const int m_tiles = M / 128, s_tiles = (S + 127) / 128;
 
-    {   // dw[u] = gKV[u] Xcat[u]^T
+    for (int part = 0; part < 2; ++part) {   // dw[u] = gKV[u] Xcat[u]^T, leading part then remainder
         gemm::Params G = base_params(h);
-        if (!operand(G.A, t_gkv, false) || !operand(G.B, t_xpad, false)) return -1;
+        const Tensor4 t_lo{gkv_lo, {256, (uint64_t)M, (uint64_t)U, 1}, {512, (uint64_t)M * 512, (uint64_t)U * M * 512}};
+        if (!operand(G.A, part ? t_lo : t_gkv, false) || !operand(G.B, t_xpad, false)) return -1;
         G.A.c[0].si = 64; G.A.c[1].tm = 128; G.A.c[2].zi = 1;
         G.B.c[0].si = 64; G.B.c[1].c0 = pad; G.B.c[1].tni = 128; G.B.c[2].zi = 1;
         G.steps = 4;
         G.out = dw; G.out_zi = (int64_t)M * L.Sp; G.out_m = L.Sp;
-        G.M = M; G.N = S; G.mode = gemm::kStoreF32;
+        G.M = M; G.N = S; G.mode = part ? gemm::kAddF32 : gemm::kStoreF32;
         if (!gemm::launch(G, m_tiles, s_tiles, U, st)) return -1;
         ++n;
     }
@@ -260,9 +279,10 @@ int tensor_backward_compress(lococo_handle* h, const BwdStep& p, const CompressP
 
     const Tensor4 t_wb{wb, {(uint64_t)L.Sp, (uint64_t)M, (uint64_t)U, 1}, {(uint64_t)L.Sp * 2, (uint64_t)M * L.Sp * 2, (uint64_t)U * M * L.Sp * 2}};
     const Tensor4 t_dab{dab, {(uint64_t)L.Sp, (uint64_t)M, (uint64_t)U, 1}, {(uint64_t)L.Sp * 2, (uint64_t)M * L.Sp * 2, (uint64_t)U * M * L.Sp * 2}};
-    {   // dX[u] += w[u]^T gKV[u]   (columns 0-127 -> dX_K, 128-255 -> dX_V)
+    for (int part = 0; part < 2; ++part) {   // dX[u] += R[u]^T (g / s)[u]   (columns 0-127 -> dX_K, 128-255 -> dX_V)
         gemm::Params G = base_params(h);
-        if (!operand(G.A, t_wb, true) || !operand(G.B, t_gkv, true)) return -1;
+        const Tensor4 t_gs{sc + (part ? L.gs_lo : L.gs), {256, (uint64_t)M, (uint64_t)U, 1}, {512, (uint64_t)M * 512, (uint64_t)U * M * 512}};
+        if (!operand(G.A, t_wb, true) || !operand(G.B, t_gs, true)) return -1;
         G.A.c[0].tm = 128; G.A.c[1].si = 64; G.A.c[2].zi = 1;
         G.B.c[0].tni = 128; G.B.c[1].si = 64; G.B.c[2].zi = 1;
         G.steps = M / 64;

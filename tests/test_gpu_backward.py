@@ -87,3 +87,19 @@ def test_backward_shared_weights_fp32_batch():
     w = wl.Workload("bwd_shared", 33, batch=3, heads=2, d=128, M=32, B=40, k=9, L=130, dtype="f32",
                     weights_per_head=False, qkv_scale=0.5, g_std=0.05)
     check_backward(w)
+
+
+def test_backward_bf16_tensor_path_shared_weights_batch_stacked_input_ragged():
+    # tensor-core backward: several sequences share one weight set (the weight gradient sums over all
+    # units), keys stacked on values as the conv input (c_in = 2d), chunk length not a multiple of 64
+    w = wl.Workload("bwd_tc_shared", 34, batch=2, heads=3, d=128, M=128, B=200, k=7, L=700, dtype="bf16",
+                    weights_per_head=False, qkv_scale=0.3, g_std=0.05, c_in_mult=2)
+    check_backward(w)
+
+
+def test_backward_bf16_tensor_path_per_head_fill_then_partial_cache_bias():
+    # tensor-core backward: per-head weights with a batch, two fill steps, a first compress step on a
+    # partly filled cache (c = 192 < M), ragged last chunk, bias gradient
+    w = wl.Workload("bwd_tc_fill", 35, batch=2, heads=2, d=128, M=256, B=96, k=5, L=420, dtype="bf16",
+                    weights_per_head=True, qkv_scale=0.0884, g_std=0.02)
+    check_backward(w, bias=True)
