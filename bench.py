@@ -324,9 +324,61 @@ def run_ours(args):
         out["cpu_baseline"] = {"value": value, "unit": UNIT, "cores": threads, "kind": "oracle",
                                "sample": f"{heads_sample} of {w.heads} heads, all {w.n_chunks} chunks, "
                                          f"{times[0]:.1f} s, scaled by {w.heads}/{heads_sample}"}
+        out["backward"] = time_backward()
     print(json.dumps(out))
     if world > 1:
         dist.destroy_process_group()
+
+
+def time_backward(name="cfg5", runs=2):
+    """Secondary figure (not the headline metric): forward with snapshots + backward through all chunk
+    steps at the fine-tuning shape (cfg5 = cfg4 shapes), device-resident seeded inputs, CUDA events."""
+    import torch
+
+    from paper_2406_05317_b200 import api, workloads as wl
+    w = wl.CONFIGS[name]
+    ctx = api.Lococo(w.batch, w.heads, w.d, w.M, w.k, w.B, dtype=torch.bfloat16, c_in=w.c_in,
+                     weights_per_head=w.weights_per_head)
+    G, _ = wl.make_weights(w)
+    ctx.set_weights(torch.from_numpy(G).cuda().to(torch.bfloat16))
+    g = torch.Generator(device="cuda").manual_seed(5000)
+    shape = (w.batch, w.heads, w.L, w.d)
+    rnd = lambda sh, s=1.0: (torch.randn(sh, device="cuda", generator=g) * s).to(torch.bfloat16)
+    Q, K, V, PO = rnd(shape, w.qkv_scale), rnd(shape, w.qkv_scale), rnd(shape, w.qkv_scale), rnd(shape)
+    cshape = (w.batch, w.heads, w.M, w.d)
+    PK, PV = rnd(cshape), rnd(cshape)
+    O, gQ, gK, gV = (torch.empty_like(Q) for _ in range(4))
+    Kc, Vc = torch.zeros(cshape, dtype=torch.bfloat16, device="cuda"), torch.zeros(cshape, dtype=torch.bfloat16, device="cuda")
+    gG = torch.zeros(G.shape, dtype=torch.float32, device="cuda")
+    saved = torch.empty(ctx.saved_bytes(w.L, w.B), dtype=torch.uint8, device="cuda")
+    scratch = torch.empty(ctx.backward_scratch_bytes(w.L, w.B), dtype=torch.uint8, device="cuda")
+    side = torch.cuda.Stream()
+    torch.cuda.synchronize()
+    fwd_ms = bwd_ms = 0.0
+    with torch.cuda.stream(side):
+        for it in range(1 + runs):
+            e = [torch.cuda.Event(enable_timing=True) for _ in range(3)]
+            Kc.zero_(); Vc.zero_()
+            e[0].record()
+            ctx.process_sequence(Q, K, V, w.B, O, Kc, Vc, 0, saved)
+            e[1].record()
+            ctx.process_sequence_backward(Q, K, V, O, w.B, saved, PO, PK, PV, gQ, gK, gV, gG, None, scratch)
+            e[2].record()
+            e[2].synchronize()
+            if it:
+                fwd_ms += e[0].elapsed_time(e[1]) / runs
+                bwd_ms += e[1].elapsed_time(e[2]) / runs
+    assert ctx.device_status() == api.OK
+    conv_f, blend_f, attn_f = sequence_flops(w)
+    fwd_flops = w.batch * w.heads * (conv_f + blend_f + attn_f)
+    # recompute of the conv + two conv-sized gradients, two blend-sized pairs, 2.5 x the attention
+    bwd_flops = w.batch * w.heads * (3.0 * conv_f + 2.0 * blend_f + 2.5 * attn_f)
+    peaks = measured_peaks()
+    return {"workload": f"{name}: 32 heads, d=128, M={w.M}, B={w.B}, k={w.k}, L={w.L}, shared conv weights, forward with cache "
+                        "snapshots + backward through all chunk steps", "forward_ms": fwd_ms, "backward_ms": bwd_ms,
+            "tokens_per_s_fwd_bwd": w.batch * w.L / ((fwd_ms + bwd_ms) * 1e-3),
+            "backward_tflops": bwd_flops / (bwd_ms * 1e-3) / 1e12, "backward_frac_of_peak": bwd_flops / (bwd_ms * 1e-3) / 1e12 / peaks["bf16_tflops"],
+            "forward_tflops": fwd_flops / (fwd_ms * 1e-3) / 1e12}
 
 
 def main():
