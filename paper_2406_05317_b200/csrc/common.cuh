@@ -57,7 +57,8 @@ struct CompressParams {
     float* UK;             // [units][M][d] unnormalised blends
     float* UV;
     float* W_out;          // optional [units][M][S]
-    int keep_R;            // also leave R in place on paths that would not store it (the backward's recompute)
+    void* R16;             // optional bf16 copy of R, [units][M][R16_stride] (the backward's recompute; tensor-core path only)
+    int R16_stride;        // multiple of 8
     void* prof;            // host only: Profiler* or nullptr
 };
 

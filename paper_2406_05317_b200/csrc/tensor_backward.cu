@@ -114,15 +114,16 @@ __global__ void pack_gt_kernel(const __nv_bfloat16* gp, __nv_bfloat16* gt, int M
 }
 
 // One block per (unit, slot) row: dA = [R>0] (dw - <dw, w>) / s with w = R / s (Eq. 7 reversed), in bf16,
-// and R itself as bf16 (exact); both zero from column S up to the row stride; dbias += sum of dA.
-__global__ void __launch_bounds__(256) da_row_kernel(BwdStep p, const float* dw, __nv_bfloat16* dab, __nv_bfloat16* wb, int Sp) {
+// zero from column S up to the row stride; R comes from the recompute in bf16 (rows of Sp, zero beyond S);
+// dbias += sum of dA.
+__global__ void __launch_bounds__(256) da_row_kernel(BwdStep p, const float* dw, __nv_bfloat16* dab, const __nv_bfloat16* rb, int Sp) {
     __shared__ float red[8];
     const int64_t row = blockIdx.x;                          // u * M + i
     const float* dwr = dw + row * Sp;
-    const float* Rr = p.R + row * p.S;
+    const __nv_bfloat16* Rr = rb + row * Sp;
     const float inv_s = 1.f / p.s[row];
     float acc = 0.f;
-    for (int j = threadIdx.x; j < p.S; j += 256) acc = fmaf(Rr[j], dwr[j], acc);
+    for (int j = threadIdx.x; j < p.S; j += 256) acc = fmaf(__bfloat162float(Rr[j]), dwr[j], acc);
     for (int of = 16; of > 0; of >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, of);
     if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = acc;
     __syncthreads();
@@ -131,14 +132,9 @@ __global__ void __launch_bounds__(256) da_row_kernel(BwdStep p, const float* dw,
     dot *= inv_s;                                            // <dw, w>
     float bsum = 0.f;
     for (int j = threadIdx.x; j < Sp; j += 256) {
-        float da = 0.f, w = 0.f;
-        if (j < p.S) {
-            const float r = Rr[j];
-            w = r;
-            da = r > 0.f ? (dwr[j] - dot) * inv_s : 0.f;
-        }
+        float da = 0.f;
+        if (j < p.S && __bfloat162float(Rr[j]) > 0.f) da = (dwr[j] - dot) * inv_s;
         dab[row * Sp + j] = __float2bfloat16_rn(da);
-        wb[row * Sp + j] = __float2bfloat16_rn(w);
         bsum += da;
     }
     if (p.dbias) {
@@ -234,6 +230,7 @@ int tensor_backward_compress(lococo_handle* h, const BwdStep& p, const CompressP
     __nv_bfloat16* xpad = reinterpret_cast<__nv_bfloat16*>(sc + L.xpad);
     __nv_bfloat16* gkv = reinterpret_cast<__nv_bfloat16*>(sc + L.gkv);
     __nv_bfloat16* gkv_lo = reinterpret_cast<__nv_bfloat16*>(sc + L.gkv_lo);
+    if (L.gs_lo - L.gs != L.gkv_lo - L.gkv) return -1;
     __nv_bfloat16* wb = reinterpret_cast<__nv_bfloat16*>(sc + L.wb);
     __nv_bfloat16* dab = reinterpret_cast<__nv_bfloat16*>(sc + L.dab);
     __nv_bfloat16* dat = reinterpret_cast<__nv_bfloat16*>(sc + L.dat);
@@ -245,7 +242,8 @@ int tensor_backward_compress(lococo_handle* h, const BwdStep& p, const CompressP
     f.k_out = View{sc + L.dummy_k, (int64_t)H * M * kD, (int64_t)M * kD, kD};
     f.v_out = View{sc + L.dummy_v, (int64_t)H * M * kD, (int64_t)M * kD, kD};
     f.W_out = nullptr;
-    f.keep_R = 1;
+    f.R16 = wb;             // R in bf16 (exact: the forward rounds it), rows of Sp
+    f.R16_stride = L.Sp;
     f.prof = nullptr;
     const int r = tensor_compress(h, f, st);
     if (r < 0) return -1;
@@ -256,19 +254,20 @@ int tensor_backward_compress(lococo_handle* h, const BwdStep& p, const CompressP
     if (!launched()) return -1;
     ++n;
 
-    const Tensor4 t_gkv{gkv, {256, (uint64_t)M, (uint64_t)U, 1}, {512, (uint64_t)M * 512, (uint64_t)U * M * 512}};
     const Tensor4 t_xpad{xpad, {256, (uint64_t)L.Sp2, (uint64_t)U, 1}, {512, (uint64_t)L.Sp2 * 512, (uint64_t)U * L.Sp2 * 512}};
     const int m_tiles = M / 128, s_tiles = (S + 127) / 128;
 
-    for (int part = 0; part < 2; ++part) {   // dw[u] = gKV[u] Xcat[u]^T, leading part then remainder
+    const uint64_t part_stride = L.gkv_lo - L.gkv;          // value and remainder lie the same distance apart in both pairs
+    {   // dw[u] = gKV[u] Xcat[u]^T: one K loop over the value's and then the remainder's 2d channels
         gemm::Params G = base_params(h);
-        const Tensor4 t_lo{gkv_lo, {256, (uint64_t)M, (uint64_t)U, 1}, {512, (uint64_t)M * 512, (uint64_t)U * M * 512}};
-        if (!operand(G.A, part ? t_lo : t_gkv, false) || !operand(G.B, t_xpad, false)) return -1;
-        G.A.c[0].si = 64; G.A.c[1].tm = 128; G.A.c[2].zi = 1;
+        const Tensor4 t_g2{gkv, {256, (uint64_t)M, (uint64_t)U, 2}, {512, (uint64_t)M * 512, part_stride}};
+        if (!operand(G.A, t_g2, false) || !operand(G.B, t_xpad, false)) return -1;
+        G.s_inner = 4;
+        G.A.c[0].si = 64; G.A.c[1].tm = 128; G.A.c[2].zi = 1; G.A.c[3].so = 1;
         G.B.c[0].si = 64; G.B.c[1].c0 = pad; G.B.c[1].tni = 128; G.B.c[2].zi = 1;
-        G.steps = 4;
+        G.steps = 8;
         G.out = dw; G.out_zi = (int64_t)M * L.Sp; G.out_m = L.Sp;
-        G.M = M; G.N = S; G.mode = part ? gemm::kAddF32 : gemm::kStoreF32;
+        G.M = M; G.N = S; G.mode = gemm::kStoreF32;
         if (!gemm::launch(G, m_tiles, s_tiles, U, st)) return -1;
         ++n;
     }
@@ -279,13 +278,14 @@ int tensor_backward_compress(lococo_handle* h, const BwdStep& p, const CompressP
 
     const Tensor4 t_wb{wb, {(uint64_t)L.Sp, (uint64_t)M, (uint64_t)U, 1}, {(uint64_t)L.Sp * 2, (uint64_t)M * L.Sp * 2, (uint64_t)U * M * L.Sp * 2}};
     const Tensor4 t_dab{dab, {(uint64_t)L.Sp, (uint64_t)M, (uint64_t)U, 1}, {(uint64_t)L.Sp * 2, (uint64_t)M * L.Sp * 2, (uint64_t)U * M * L.Sp * 2}};
-    for (int part = 0; part < 2; ++part) {   // dX[u] += R[u]^T (g / s)[u]   (columns 0-127 -> dX_K, 128-255 -> dX_V)
+    {   // dX[u] += R[u]^T (g / s)[u]   (columns 0-127 -> dX_K, 128-255 -> dX_V); K loop over the slots, twice
         gemm::Params G = base_params(h);
-        const Tensor4 t_gs{sc + (part ? L.gs_lo : L.gs), {256, (uint64_t)M, (uint64_t)U, 1}, {512, (uint64_t)M * 512, (uint64_t)U * M * 512}};
-        if (!operand(G.A, t_wb, true) || !operand(G.B, t_gs, true)) return -1;
+        const Tensor4 t_gs2{sc + L.gs, {256, (uint64_t)M, (uint64_t)U, 2}, {512, (uint64_t)M * 512, part_stride}};
+        if (!operand(G.A, t_wb, true) || !operand(G.B, t_gs2, true)) return -1;
+        G.s_inner = M / 64;
         G.A.c[0].tm = 128; G.A.c[1].si = 64; G.A.c[2].zi = 1;
-        G.B.c[0].tni = 128; G.B.c[1].si = 64; G.B.c[2].zi = 1;
-        G.steps = M / 64;
+        G.B.c[0].tni = 128; G.B.c[1].si = 64; G.B.c[2].zi = 1; G.B.c[3].so = 1;
+        G.steps = 2 * (M / 64);
         G.out = p.dXK; G.out_zi = (int64_t)S * kD; G.out_m = kD;
         G.out_n_inner = kD; G.out_n_in = 1; G.out_n_out = p.dXV - p.dXK;
         G.M = S; G.N = 256; G.mode = gemm::kAddF32;

@@ -244,6 +244,19 @@ __device__ __forceinline__ void compress_body(const TcCompressParams& P, uint8_t
             }
             umma_commit(bar_blend);
         }
+        // R as the blends read it (bf16, [position group][slot][8 positions]) also goes out row by row
+        // when the backward pass asked for it: a slot's groups are consecutive 16-byte pieces of its row
+        if (p.R16) {
+            const int groups = n_tile / 8;
+            __nv_bfloat16* r16 = static_cast<__nv_bfloat16*>(p.R16) + ((int64_t)u * p.M + sb * kSlots) * p.R16_stride + j0;
+            for (int x = tid; x < kSlots * groups; x += blockDim.x) {
+                const int sl = x / groups, gq = x % groups;
+                if (j0 + gq * 8 < p.R16_stride)
+                    *reinterpret_cast<uint4*>(r16 + (int64_t)sl * p.R16_stride + gq * 8) =
+                        *reinterpret_cast<const uint4*>(ring_ptr + gq * 2048 + sl * 16);
+            }
+            __syncthreads();     // the ring is reused (row sums, next tile) once the blends are done
+        }
         // the staged tiles and the ring are reused by the next tile only after the blends read them
         mbar_wait(bar_blend, tile_it & 1, P.status, failed, 4);
     }
@@ -1017,7 +1030,7 @@ static bool build_compress_params(lococo_handle* h, const CompressParams& p, boo
     P.gimage = reinterpret_cast<const __nv_bfloat16*>(h->ws + h->off_gimage);
     P.part_U = reinterpret_cast<float*>(h->ws + h->off_part);
     P.part_s = P.part_U + (size_t)p.units * SB * max_parts * 2 * kSlots * kD;
-    P.R_store = (p.W_out || p.keep_R) ? p.R : nullptr;
+    P.R_store = p.W_out ? p.R : nullptr;
     P.status = reinterpret_cast<int*>(h->ws + h->off_status);
     P.n_tile = pl.n_tile; P.tiles = pl.tiles; P.parts = pl.parts; P.tiles_per_part = pl.tiles_per_part;
     P.part_stride = fused ? max_parts : pl.parts;   // fixed regions where steps with different plans share a launch
