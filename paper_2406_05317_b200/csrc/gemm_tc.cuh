@@ -33,11 +33,13 @@ struct Operand {
     int mn_major;
     int pad[3];
 };
-// kSoftmaxBF16: out = exp2(acc * scale2 - rowvec[row] * log2 e) where column < causal_c + row + 1, else 0 (bf16)
-// kDsBF16:      out = aux * (acc - rowvec[row]) * alpha             under the same mask (aux: bf16, laid out like out)
-enum Mode { kStoreF32 = 0, kAtomicF32 = 1, kStoreBF16 = 2, kAddF32 = 3, kSoftmaxBF16 = 4, kDsBF16 = 5 };
+// kPairBF16: TWO products per tile, acc = A B^T and acc2 = A2 B2^T (same coordinates rule, second accumulator);
+//            out  = p = exp2(acc * scale2 - rowvec[row] * log2 e) where column < causal_c + row + 1, else 0 (bf16)
+//            out2 = p * (acc2 - rowvec2[row]) * alpha under the same mask (p in fp32: not rounded in between)
+enum Mode { kStoreF32 = 0, kAtomicF32 = 1, kStoreBF16 = 2, kAddF32 = 3, kPairBF16 = 4 };
 struct alignas(64) Params {
     Operand A, B;
+    Operand A2, B2;              // second product of kPairBF16
     int n_inner, s_inner, z_inner;   // decomposition of the N tile index, of the K step index and of the batch index
     int steps, splits;           // K steps (64 wide) in total; CTAs that share them (blockIdx.z = z * splits + split)
     void* out;
@@ -53,10 +55,12 @@ struct alignas(64) Params {
     int causal_c;
     int k_lo_on, k_lo_c0;        // K loop starts at step max(0, (tm * 128 + k_lo_c0) / 64)
     int k_hi_on, k_hi_c0;        // K loop ends before step (tm * 128 + k_hi_c0 + 63) / 64
-    const float* rowvec;         // per (batch, row) value of the two fused modes
+    const float* rowvec;         // per (batch, row) values of kPairBF16
     int64_t rowvec_z;
-    const void* aux;
     float scale2;
+    void* out2;                  // kPairBF16
+    const float* rowvec2;
+    int64_t rowvec2_z;
 };
 
 constexpr int kThreads = 320;                      // 8 epilogue warps, the MMA-issue warp, the producer warp
@@ -86,6 +90,7 @@ __global__ void __launch_bounds__(kThreads, 2) gemm_kernel(const __grid_constant
     if (P.k_hi_on) s_end = min(s_end, max(0, tm * 128 + P.k_hi_c0 + 63) / 64);
     if (P.causal_tiles && tn * 128 >= P.causal_c + tm * 128 + 128) s_end = s_begin;
     if (s_end < s_begin) s_end = s_begin;
+    const int passes = P.mode == kPairBF16 ? 2 : 1;
 
     if (tid == 256) {
         for (int s = 0; s < kStages; ++s) {
@@ -97,7 +102,7 @@ __global__ void __launch_bounds__(kThreads, 2) gemm_kernel(const __grid_constant
         fence_barrier_init();
     }
     if (warp == 0) {
-        tmem_alloc(smem_u32(&tmem_slot), 128);
+        tmem_alloc(smem_u32(&tmem_slot), 256);
         tmem_relinquish();
     }
     tc_fence_before();
@@ -107,14 +112,16 @@ __global__ void __launch_bounds__(kThreads, 2) gemm_kernel(const __grid_constant
 
     if (tid == 288) {
         // ---- producer
-        for (int s = s_begin, g = 0; s < s_end; ++s, ++g) {
+        int g = 0;
+        for (int pass = 0; pass < passes; ++pass)
+        for (int s = s_begin; s < s_end; ++s, ++g) {
             const int st = g % kStages;
             if (g >= kStages) mbar_wait(bar_empty + 8 * st, ((g / kStages) - 1) & 1, P.status, failed, 30);
             mbar_expect_tx(bar_full + 8 * st, kStageBytes2);
             const uint32_t dst = ring + st * kStageBytes2;
 #pragma unroll
             for (int op = 0; op < 2; ++op) {
-                const Operand& O = op ? P.B : P.A;
+                const Operand& O = pass ? (op ? P.B2 : P.A2) : (op ? P.B : P.A);
                 const uint32_t d = dst + op * kOperandBytes;
                 const int x = coord_of(O.c[0], P, tm, tn, s, z), y = coord_of(O.c[1], P, tm, tn, s, z);
                 const int c2 = coord_of(O.c[2], P, tm, tn, s, z), c3 = coord_of(O.c[3], P, tm, tn, s, z);
@@ -128,19 +135,23 @@ __global__ void __launch_bounds__(kThreads, 2) gemm_kernel(const __grid_constant
         }
     } else if (tid == 256) {
         // ---- MMA issuer
-        const uint32_t idesc = instr_desc_bf16(128, P.A.mn_major != 0, P.B.mn_major != 0);
-        for (int s = s_begin, g = 0; s < s_end; ++s, ++g) {
+        int g = 0;
+        for (int pass = 0; pass < passes; ++pass)
+        for (int s = s_begin; s < s_end; ++s, ++g) {
+            const Operand& OA = pass ? P.A2 : P.A;
+            const Operand& OB = pass ? P.B2 : P.B;
+            const uint32_t idesc = instr_desc_bf16(128, OA.mn_major != 0, OB.mn_major != 0);
             const int st = g % kStages;
             mbar_wait(bar_full + 8 * st, (g / kStages) & 1, P.status, failed, 31);
             tc_fence_after();
             const uint32_t a_addr = ring + st * kStageBytes2, b_addr = a_addr + kOperandBytes;
             // K-major: 32 bytes per 16-element step inside the 128-byte row, 8-row groups 1024 bytes apart.
             // MN-major: 16 k rows (two 8-row groups) per step, the two 64-wide halves 8 KB apart.
-            const uint64_t a0 = P.A.mn_major ? smem_desc_sw128(a_addr, kOperandBytes / 2, 1024) : smem_desc_sw128(a_addr, 16, 1024);
-            const uint64_t b0 = P.B.mn_major ? smem_desc_sw128(b_addr, kOperandBytes / 2, 1024) : smem_desc_sw128(b_addr, 16, 1024);
-            const uint32_t a_step = P.A.mn_major ? 2048u >> 4 : 32u >> 4, b_step = P.B.mn_major ? 2048u >> 4 : 32u >> 4;
+            const uint64_t a0 = OA.mn_major ? smem_desc_sw128(a_addr, kOperandBytes / 2, 1024) : smem_desc_sw128(a_addr, 16, 1024);
+            const uint64_t b0 = OB.mn_major ? smem_desc_sw128(b_addr, kOperandBytes / 2, 1024) : smem_desc_sw128(b_addr, 16, 1024);
+            const uint32_t a_step = OA.mn_major ? 2048u >> 4 : 32u >> 4, b_step = OB.mn_major ? 2048u >> 4 : 32u >> 4;
 #pragma unroll
-            for (int kk = 0; kk < 4; ++kk) umma_ss(tmem, a0 + kk * a_step, b0 + kk * b_step, idesc, (g | kk) != 0);
+            for (int kk = 0; kk < 4; ++kk) umma_ss(tmem + pass * 128, a0 + kk * a_step, b0 + kk * b_step, idesc, (s != s_begin || kk != 0));
             umma_commit(bar_empty + 8 * st);
         }
         umma_commit(bar_acc);
@@ -159,11 +170,49 @@ __global__ void __launch_bounds__(kThreads, 2) gemm_kernel(const __grid_constant
         const int c_begin = (tid >> 7) * 64;
         const int64_t base = (int64_t)(z % P.z_inner) * P.out_zi + (int64_t)(z / P.z_inner) * P.out_zo + (int64_t)row * P.out_m;
         const bool contiguous = P.out_n_in == 1 && P.out_n_inner % 32 == 0;
-        const bool fused = P.mode == kSoftmaxBF16 || P.mode == kDsBF16;
-        const int mode = fused ? (int)kStoreBF16 : P.mode;
-        const float alpha = fused ? 1.f : P.alpha;
-        const float rv = fused && row < P.M ? P.rowvec[(int64_t)z * P.rowvec_z + row] : 0.f;
-        const int vis = P.causal_c + row + 1;
+        if (P.mode == kPairBF16) {
+            const float l2 = row < P.M ? P.rowvec[(int64_t)z * P.rowvec_z + row] * 1.4426950408889634f : 0.f;
+            const float dl = row < P.M ? P.rowvec2[(int64_t)z * P.rowvec2_z + row] : 0.f;
+            const int lim = min(P.N, P.causal_c + row + 1);       // columns this row sees
+#pragma unroll 1
+            for (int c0 = c_begin; c0 < c_begin + 64; c0 += 16) {
+                uint32_t v[16], w[16];
+                if (any) {
+                    tmem_ld16(lane_addr + c0, v);
+                    tmem_ld16(lane_addr + 128 + c0, w);
+                    tmem_ld_wait();
+                }
+                const int n0 = tn * 128 + c0;
+                if (row >= P.M || n0 >= P.N) continue;
+                __nv_bfloat16* o1 = static_cast<__nv_bfloat16*>(P.out) + base + n0;
+                __nv_bfloat16* o2 = static_cast<__nv_bfloat16*>(P.out2) + base + n0;
+                uint32_t pk[8], dk[8];
+#pragma unroll
+                for (int e = 0; e < 16; e += 2) {
+                    const bool on0 = any && n0 + e < lim, on1 = any && n0 + e + 1 < lim;
+                    const float p0 = on0 ? exp2f(__uint_as_float(v[e]) * P.scale2 - l2) : 0.f;
+                    const float p1 = on1 ? exp2f(__uint_as_float(v[e + 1]) * P.scale2 - l2) : 0.f;
+                    const float d0 = on0 ? p0 * (__uint_as_float(w[e]) - dl) * P.alpha : 0.f;
+                    const float d1 = on1 ? p1 * (__uint_as_float(w[e + 1]) - dl) * P.alpha : 0.f;
+                    pk[e >> 1] = pack_bf16(p0, p1);
+                    dk[e >> 1] = pack_bf16(d0, d1);
+                }
+                if (n0 + 16 <= P.N) {
+                    *reinterpret_cast<uint4*>(o1) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
+                    *reinterpret_cast<uint4*>(o1 + 8) = make_uint4(pk[4], pk[5], pk[6], pk[7]);
+                    *reinterpret_cast<uint4*>(o2) = make_uint4(dk[0], dk[1], dk[2], dk[3]);
+                    *reinterpret_cast<uint4*>(o2 + 8) = make_uint4(dk[4], dk[5], dk[6], dk[7]);
+                } else {
+                    for (int e = 0; e < 16 && n0 + e < P.N; ++e) {
+                        const uint32_t a = pk[e >> 1], d = dk[e >> 1];
+                        reinterpret_cast<uint16_t*>(o1)[e] = (uint16_t)((e & 1) ? (a >> 16) : (a & 0xffffu));
+                        reinterpret_cast<uint16_t*>(o2)[e] = (uint16_t)((e & 1) ? (d >> 16) : (d & 0xffffu));
+                    }
+                }
+            }
+        } else {
+        const int mode = P.mode;
+        const float alpha = P.alpha;
 #pragma unroll 1
         for (int c0 = c_begin; c0 < c_begin + 64; c0 += 32) {
             uint32_t v[32];
@@ -177,33 +226,6 @@ __global__ void __launch_bounds__(kThreads, 2) gemm_kernel(const __grid_constant
             const int n0 = tn * 128 + c0;
             if (row >= P.M || n0 >= P.N || (!any && mode != kStoreF32 && mode != kStoreBF16)) continue;
             const int64_t col0 = (int64_t)(n0 % P.out_n_inner) * P.out_n_in + (int64_t)(n0 / P.out_n_inner) * P.out_n_out;
-            if (P.mode == kSoftmaxBF16) {
-                const float l2 = rv * 1.4426950408889634f;
-#pragma unroll
-                for (int e = 0; e < 32; ++e)
-                    v[e] = __float_as_uint(n0 + e < vis ? exp2f(__uint_as_float(v[e]) * P.scale2 - l2) : 0.f);
-            } else if (P.mode == kDsBF16) {
-                const __nv_bfloat16* a = static_cast<const __nv_bfloat16*>(P.aux) + base + col0;
-                if (n0 + 32 <= P.N) {
-#pragma unroll
-                    for (int e = 0; e < 32; e += 8) {
-                        const uint4 q = *reinterpret_cast<const uint4*>(a + e);
-                        const uint32_t w[4] = {q.x, q.y, q.z, q.w};
-#pragma unroll
-                        for (int x = 0; x < 8; ++x) {
-                            const float pr = n0 + e + x < vis ? __uint_as_float((x & 1) ? (w[x >> 1] & 0xffff0000u) : (w[x >> 1] << 16)) : 0.f;
-                            v[e + x] = __float_as_uint(pr * (__uint_as_float(v[e + x]) - rv) * P.alpha);
-                        }
-                    }
-                } else {
-#pragma unroll 1
-                    for (int e = 0; e < 32; ++e) {
-                        float pr = 0.f;
-                        if (n0 + e < vis && n0 + e < P.N) pr = __bfloat162float(a[e]);
-                        v[e] = __float_as_uint(pr * (__uint_as_float(v[e]) - rv) * P.alpha);
-                    }
-                }
-            }
             if (contiguous && n0 + 32 <= P.N) {
                 if (mode == kStoreF32) {
                     float4* o = reinterpret_cast<float4*>(static_cast<float*>(P.out) + base + col0);
@@ -247,10 +269,11 @@ __global__ void __launch_bounds__(kThreads, 2) gemm_kernel(const __grid_constant
                 }
             }
         }
+        }
     }
     tc_fence_before();
     __syncthreads();
-    if (warp == 0) tmem_dealloc(tmem, 128);
+    if (warp == 0) tmem_dealloc(tmem, 256);
     if (tid == 256) {
         for (int s = 0; s < 2 * kStages + 1; ++s) mbar_inval(bar_full + 8 * s);
     }

@@ -10,8 +10,8 @@
 //                                                                     map with overlapping strides
 //     dZ (in dX) += sum over taps of shift_t(dA^T) G_t                a tap = a row offset of the box
 //   attention (Eq. 1 reversed), in blocks of up to 1024 queries, P and dS materialised in bf16:
-//     P = exp(scale Q X_K^T - lse), dS = scale P (dO X_V^T - delta)   softmax and its gradient fused into the
-//                                                                     GEMM epilogues; masked tiles skipped
+//     P = exp(scale Q X_K^T - lse), dS = scale P (dO X_V^T - delta)   one launch, two accumulators per tile, softmax
+//                                                                     and its gradient in the epilogue; masked tiles skipped
 //     dX_V += P^T dO, dX_K += dS^T Q, dQ = dS X_K                     K loops cut at the causal limit
 // Gradients that enter a GEMM are rounded to bf16 (fp32 accumulation), like the forward's operands; the
 // cache gradient, which every earlier step inherits, enters as two bf16 terms (value + remainder).
@@ -344,25 +344,28 @@ int tensor_backward_attention(lococo_handle* h, const BwdStep& p, int B, char* s
         const int qb = std::min(L.QB, p.b - q0), q_tiles = (qb + 127) / 128;
         const int Sv = std::min(S, p.c + q0 + qb);          // keys any query of the block can see
         const int sv_tiles = (Sv + 127) / 128;
-        // P = exp(scale Q X_K^T - lse) and dS = scale P (dO X_V^T - delta): the softmax and its gradient are
-        // applied to the accumulator tile, under the causal mask, and only bf16 P and dS reach memory
-        for (int which = 0; which < 2; ++which) {
+        // P = exp(scale Q X_K^T - lse) and dS = scale P (dO X_V^T - delta): ONE launch computes both products
+        // of a tile into two accumulators and applies the softmax and its gradient to them, under the causal
+        // mask; only bf16 P and dS reach memory
+        {
             gemm::Params G = base_params(h);
-            if (!operand(G.A, which ? t_do : t_q, false) || !operand(G.B, t_xpad, false)) return -1;
+            if (!operand(G.A, t_q, false) || !operand(G.B, t_xpad, false) || !operand(G.A2, t_do, false) || !operand(G.B2, t_xpad, false))
+                return -1;
             G.z_inner = H;
-            G.A.c[0].si = 64; G.A.c[1].c0 = q0; G.A.c[1].tm = 128; G.A.c[2].zi = 1; G.A.c[3].zo = 1;
-            G.B.c[0].c0 = which * kD; G.B.c[0].si = 64; G.B.c[1].c0 = pad; G.B.c[1].tni = 128; G.B.c[2].zi = 1; G.B.c[2].zo = H;
+            for (int which = 0; which < 2; ++which) {
+                gemm::Operand& A = which ? G.A2 : G.A;
+                gemm::Operand& Bo = which ? G.B2 : G.B;
+                A.c[0].si = 64; A.c[1].c0 = q0; A.c[1].tm = 128; A.c[2].zi = 1; A.c[3].zo = 1;
+                Bo.c[0].c0 = which * kD; Bo.c[0].si = 64; Bo.c[1].c0 = pad; Bo.c[1].tni = 128; Bo.c[2].zi = 1; Bo.c[2].zo = H;
+            }
             G.steps = 2;
-            G.out = which ? dsb : pb; G.out_zi = (int64_t)L.QB * L.Sp; G.out_zo = (int64_t)H * L.QB * L.Sp; G.out_m = L.Sp;
+            G.out = pb; G.out2 = dsb;
+            G.out_zi = (int64_t)L.QB * L.Sp; G.out_zo = (int64_t)H * L.QB * L.Sp; G.out_m = L.Sp;
             G.M = qb; G.N = Sv;
             G.causal_tiles = 1; G.causal_c = p.c + q0;
-            if (which) {
-                G.mode = gemm::kDsBF16; G.aux = pb; G.alpha = p.scale;
-                G.rowvec = p.delta + q0; G.rowvec_z = p.b;
-            } else {
-                G.mode = gemm::kSoftmaxBF16; G.scale2 = p.scale * 1.4426950408889634f;
-                G.rowvec = p.lse + q0; G.rowvec_z = p.lse_stride;
-            }
+            G.mode = gemm::kPairBF16; G.alpha = p.scale; G.scale2 = p.scale * 1.4426950408889634f;
+            G.rowvec = p.lse + q0; G.rowvec_z = p.lse_stride;
+            G.rowvec2 = p.delta + q0; G.rowvec2_z = p.b;
             if (!gemm::launch(G, q_tiles, sv_tiles, U, st)) return -1;
             ++n;
         }
