@@ -303,7 +303,13 @@ int tensor_backward_compress(lococo_handle* h, const BwdStep& p, const CompressP
         G.B.c[0].tni = 128; G.B.c[1].si = 64; G.B.c[2].tno = 1; G.B.c[3].so = unit_so; G.B.c[3].zi = unit_zi;
         G.steps = in_set * G.s_inner;
         const int tiles = m_tiles * (k * C / 128) * sets;
-        G.splits = std::max(1, std::min(G.steps, (296 + tiles - 1) / tiles));
+        // K splits: fill whole waves of the 2 x 148 CTA slots (the split partials meet in atomics)
+        double best = 0.0;
+        for (int sp = 1; sp <= 16 && (sp == 1 || G.steps / sp >= 32); ++sp) {   // a split keeps at least 32 K steps
+            const int ctas = tiles * sp, waves = (ctas + 295) / 296;
+            const double fill = (double)ctas / (waves * 296.0) - 0.002 * sp;
+            if (fill > best) { best = fill; G.splits = sp; }
+        }
         G.out = p.dG; G.out_zi = (int64_t)M * C * k; G.out_m = (int64_t)C * k;
         G.out_n_inner = C; G.out_n_in = k; G.out_n_out = 1;
         G.M = M; G.N = k * C; G.mode = gemm::kAtomicF32;
