@@ -93,6 +93,15 @@ def test_cfg4_slice(api, orc, path):
     check_sequence(api, orc, wl.CONFIGS["cfg4"].slice(heads=2, B=1024, L=3072), path)
 
 
+@pytest.mark.parametrize("path", [0, 1])
+def test_generation_mode_chunk_of_one_token(api, orc, path):
+    # B = 1 (the generation stage of Section 3.3 sets the segment length to 1): 128 fill steps, then every step compresses
+    # S = M + 1 positions back into M slots
+    w = wl.Workload("decode", 12, batch=2, heads=2, d=128, M=128, B=1, k=21, L=160, dtype="bf16",
+                    weights_per_head=False, qkv_scale=0.0884, g_std=0.02)
+    check_sequence(api, orc, w, path)
+
+
 @pytest.mark.parametrize("dtype", ["f32", "bf16"])
 def test_ragged_everything(api, orc, dtype):
     # sizes that are multiples of nothing: M=40, B=37, L=301 (last chunk short), k=7,
