@@ -135,18 +135,19 @@ lococo_status attention_impl(lococo_handle* h, View q, View kc, View vc, int c, 
     return count(h, simt_attention(h->cfg.dtype, p, st));
 }
 
-// One step of Algorithm 2's loop with an in-place cache: Step 3 with the old cache, then the
-// update. On the tensor-core path both run as one launch (they are independent of each other).
+// One step of Algorithm 2's loop: Step 3 with the old cache (kc, vc), then the update into (ko, vo), which
+// may be the old cache itself. On the tensor-core path both run as one launch (they are independent of
+// each other; with a separate output cache the compress CTAs can write it directly).
 lococo_status step_impl(lococo_handle* h, View q, View kc, View vc, int c, View kn, View vn, int b, View o, float* lse,
-                        int64_t lse_stride, cudaStream_t st) {
+                        int64_t lse_stride, View ko, View vo, cudaStream_t st) {
     if (h->use_tensor && c + b > h->cfg.M) {
         const AttnParams a = make_attn_params(h, q, kc, vc, c, kn, vn, b, o, lse, lse_stride);
-        const CompressParams p = make_compress_params(h, kc, vc, c, kn, vn, b, kc, vc, nullptr);
+        const CompressParams p = make_compress_params(h, kc, vc, c, kn, vn, b, ko, vo, nullptr);
         if (tensor_attention_supported(h, a) && tensor_compress_supported(h, p)) return count(h, tensor_chunk_step(h, a, p, st));
     }
     lococo_status s = attention_impl(h, q, kc, vc, c, kn, vn, b, o, lse, lse_stride, st);
     if (s) return s;
-    return compress_impl(h, kc, vc, c, kn, vn, b, kc, vc, nullptr, st);
+    return compress_impl(h, kc, vc, c, kn, vn, b, ko, vo, nullptr, st);
 }
 
 bool chunk_args_ok(const lococo_handle* h, int c, int b) {
@@ -367,13 +368,20 @@ lococo_status run_chunk_loop(lococo_handle* h, lococo_tensor Q, lococo_tensor K,
     const size_t snap_step = (size_t)h->units * cfg.M * cfg.head_dim * e;
     const size_t snap_all = align_up((size_t)n_chunks * snap_step, 256);
     char* sv = static_cast<char*>(saved);
+    // The cache the next step reads: the caller's, or (tensor-core path, while steps can write their
+    // result directly) the workspace's second cache; the two alternate, so a step never writes the cache
+    // its own attention CTAs are reading. The final cache is always handed back in the caller's tensors.
+    View cur_k = dev(K_cache), cur_v = dev(V_cache);
+    const lococo_tensor alt_k_t = contiguous(h->ws + h->off_alt_k, cfg.heads, cfg.M, cfg.head_dim);
+    const lococo_tensor alt_v_t = contiguous(h->ws + h->off_alt_v, cfg.heads, cfg.M, cfg.head_dim);
+    bool in_alt = false;
     for (int n = 0; n < n_chunks; ++n) {
         const int t0 = n * B;
         const int b = L - t0 < B ? L - t0 : B;
         if (sv) {
             lococo_tensor sk = contiguous(sv + (size_t)n * snap_step, cfg.heads, cfg.M, cfg.head_dim);
             lococo_tensor svv = contiguous(sv + snap_all + (size_t)n * snap_step, cfg.heads, cfg.M, cfg.head_dim);
-            FillParams f{dev(K_cache), dev(V_cache), dev(sk), dev(svv), cfg.heads, h->units, cfg.head_dim, 0, cfg.M};
+            FillParams f{cur_k, cur_v, dev(sk), dev(svv), cfg.heads, h->units, cfg.head_dim, 0, cfg.M};
             lococo_status s = count(h, simt_fill(cfg.dtype, f, st));
             if (s) return s;
         }
@@ -391,13 +399,33 @@ lococo_status run_chunk_loop(lococo_handle* h, lococo_tensor Q, lococo_tensor K,
         if (!queued) {
             lococo_status s = count(h, tensor_sequence_launch(h, st, h->prof.on ? &h->prof : nullptr));   // flush what is queued, in order
             if (s) return s;
-            s = step_impl(h, qn, dev(K_cache), dev(V_cache), c, kn, vn, b, on, lse, L, st);
+            View out_k = cur_k, out_v = cur_v;
+            bool direct = false;
+            if (h->use_tensor && !h->persistent_loop && c + b > cfg.M) {
+                const CompressParams p = make_compress_params(h, cur_k, cur_v, c, kn, vn, b, cur_k, cur_v, nullptr);
+                direct = tensor_compress_supported(h, p) && tensor_step_direct(h, p);
+            }
+            if (direct) {
+                out_k = in_alt ? dev(K_cache) : dev(alt_k_t);
+                out_v = in_alt ? dev(V_cache) : dev(alt_v_t);
+            }
+            s = step_impl(h, qn, cur_k, cur_v, c, kn, vn, b, on, lse, L, out_k, out_v, st);
             if (s) return s;
+            if (direct) {
+                cur_k = out_k;
+                cur_v = out_v;
+                in_alt = !in_alt;
+            }
         }
         c = c + b <= cfg.M ? c + b : cfg.M;
     }
     lococo_status s = count(h, tensor_sequence_launch(h, st, h->prof.on ? &h->prof : nullptr));
     if (s) return s;
+    if (in_alt) {   // hand the final cache back
+        FillParams f{cur_k, cur_v, dev(K_cache), dev(V_cache), cfg.heads, h->units, cfg.head_dim, 0, cfg.M};
+        s = count(h, simt_fill(cfg.dtype, f, st));
+        if (s) return s;
+    }
     *c_inout = c;
     return LOCOCO_OK;
 }

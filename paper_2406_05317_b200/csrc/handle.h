@@ -32,6 +32,7 @@ struct lococo_handle {
     size_t ws_need = 0;
     size_t off_status = 0, off_gpack = 0, off_bias = 0, off_s = 0, off_UK = 0, off_UV = 0, off_R = 0;
     size_t off_gimage = 0, off_part = 0, off_steps = 0, off_sync = 0;  // tensor-core path
+    size_t off_alt_k = 0, off_alt_v = 0;   // second cache (the chunk loop alternates between the caller's and this one)
     // persistent chunk loop: step descriptors staged in pinned host memory (a small ring, one slot per call)
     static constexpr int kSeqSlots = 4;
     unsigned char* seq_host = nullptr;
@@ -65,6 +66,7 @@ void tensor_layout_workspace(lococo_handle* h, size_t* off);
 int tensor_pack_weights(lococo_handle* h, const void* G, cudaStream_t st);
 bool tensor_compress_supported(const lococo_handle* h, const CompressParams& p);
 int tensor_compress(lococo_handle* h, const CompressParams& p, cudaStream_t st);
+bool tensor_step_direct(lococo_handle* h, const CompressParams& p);
 bool tensor_attention_supported(const lococo_handle* h, const AttnParams& p);
 int tensor_attention(lococo_handle* h, const AttnParams& p, cudaStream_t st);
 int tensor_chunk_step(lococo_handle* h, const AttnParams& a, const CompressParams& p, cudaStream_t st);

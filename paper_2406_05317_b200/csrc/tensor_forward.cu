@@ -39,6 +39,8 @@ struct TcCompressParams {
     float* part_U;                // [units][slot blocks][parts][2][128 channels][128 slots]
     float* part_s;                // [units][slot blocks][parts][128]
     int part_stride;              // partial sets reserved per (unit, slot block): >= parts
+    int direct;                   // 1 (only with parts == 1 and an output that is not the input cache): the CTA
+                                  // normalises and writes the cache rows itself, no partials, no finalize pass
     float* R_store;               // optional [units][M][S]
     int* status;
     int n_tile, tiles, parts, tiles_per_part, halves, stages, rows_pad, slot_blocks;
@@ -261,6 +263,33 @@ __device__ __forceinline__ void compress_body(const TcCompressParams& P, uint8_t
         mbar_wait(bar_blend, tile_it & 1, P.status, failed, 4);
     }
 
+    if (P.direct && tile_it > 0) {
+        // ---- this CTA saw every position of its slots: Eq. 7 after Eq. 4-5 here, same arithmetic as finalize_tile
+        tc_fence_after();
+        float* sums = reinterpret_cast<float*>(ring_ptr);      // [3 groups][128 rows]; the ring is idle now
+        sums[eg * kSlots + rl] = ssum;
+        __syncthreads();
+        const float tot = sums[rl] + sums[kSlots + rl] + sums[2 * kSlots + rl] + p.eps;
+        const float inv = 1.f / tot;
+        if (eg == 0) p.s[(int64_t)u * p.M + slot] = tot;
+        const uint32_t lane_addr = tmem + ((uint32_t)((warp & 3) * 32) << 16);
+#pragma unroll 1
+        for (int piece = eg; piece < 2 * (kD / 32); piece += 3) {
+            const int mat = piece & 1, c0 = (piece >> 1) * 32;
+            const View& out = mat ? p.v_out : p.k_out;
+            __nv_bfloat16* orow = unit_base_mut<__nv_bfloat16>(out, n, h) + (int64_t)slot * out.st + c0;
+            uint32_t a[32];
+            tmem_ld32(lane_addr + (mat ? kColUV : kColUK) + c0, a);
+            tmem_ld_wait();
+#pragma unroll
+            for (int e = 0; e < 32; e += 8)
+                *reinterpret_cast<uint4*>(orow + e) =
+                    make_uint4(pack_bf16(__uint_as_float(a[e]) * inv, __uint_as_float(a[e + 1]) * inv),
+                               pack_bf16(__uint_as_float(a[e + 2]) * inv, __uint_as_float(a[e + 3]) * inv),
+                               pack_bf16(__uint_as_float(a[e + 4]) * inv, __uint_as_float(a[e + 5]) * inv),
+                               pack_bf16(__uint_as_float(a[e + 6]) * inv, __uint_as_float(a[e + 7]) * inv));
+        }
+    } else
     // ---- partial blends and row sums of this CTA's tiles
     if (tile_it > 0) {
         tc_fence_after();
@@ -1000,6 +1029,10 @@ void tensor_layout_workspace(lococo_handle* h, size_t* off) {
     *off = align(*off + (size_t)kMaxSeqSteps * sizeof(TcStepParams));
     h->off_sync = *off;
     *off = align(*off + (size_t)(64 + 2 * h->units) * sizeof(int));   // item counter, then per unit: finished, version
+    h->off_alt_k = *off;
+    *off = align(*off + (size_t)h->units * c.M * kD * 2);
+    h->off_alt_v = *off;
+    *off = align(*off + (size_t)h->units * c.M * kD * 2);
 }
 
 int tensor_pack_weights(lococo_handle* h, const void* G, cudaStream_t st) {
@@ -1177,14 +1210,24 @@ int tensor_chunk_step(lococo_handle* h, const AttnParams& a, const CompressParam
             return -1;
         attr_set = true;
     }
+    // one CTA per (unit, slot block) and an output cache that is not the input: no partials, no finalize pass
+    P.comp.direct = P.comp.parts == 1 && p.W_out == nullptr && p.k_out.ptr != p.xk.cache.ptr && p.v_out.ptr != p.xv.cache.ptr;
     const int blocks = P.n_attn + a.units * P.comp_per_unit;
     prof_begin(p.prof, 2, st);
     const bool ok = launch_overlapped(chunk_step_tc_kernel, dim3(blocks), dim3(kAttnThreads), kMaxSmem, st, P) == cudaSuccess;
     if (!ok) cudaGetLastError();
     prof_end(p.prof, st);
     if (!ok) return -1;
+    if (P.comp.direct) return 1;
     const int r = finish_compress(P.comp, st);
     return r < 0 ? -1 : 1 + r;
+}
+
+// Whether a chunk step with these parameters can write the new cache straight from its compress CTAs
+// (given an output cache that is not the input).
+bool tensor_step_direct(lococo_handle* h, const CompressParams& p) {
+    Plan pl;
+    return h->use_tensor && p.W_out == nullptr && make_plan(p.S, p.k, p.c_in / 128, p.units, p.M / kSlots, true, &pl) && pl.parts == 1;
 }
 
 // ---- persistent chunk loop
