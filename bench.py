@@ -325,6 +325,7 @@ def run_ours(args):
                                "sample": f"{heads_sample} of {w.heads} heads, all {w.n_chunks} chunks, "
                                          f"{times[0]:.1f} s, scaled by {w.heads}/{heads_sample}"}
         out["backward"] = time_backward()
+        out["layer_stack"] = time_layer_stack()
     print(json.dumps(out))
     if world > 1:
         dist.destroy_process_group()
@@ -379,6 +380,43 @@ def time_backward(name="cfg5", runs=2):
             "tokens_per_s_fwd_bwd": w.batch * w.L / ((fwd_ms + bwd_ms) * 1e-3),
             "backward_tflops": bwd_flops / (bwd_ms * 1e-3) / 1e12, "backward_frac_of_peak": bwd_flops / (bwd_ms * 1e-3) / 1e12 / peaks["bf16_tflops"],
             "forward_tflops": fwd_flops / (fwd_ms * 1e-3) / 1e12}
+
+
+def time_layer_stack(layers=32, runs=3):
+    """Secondary figure: the paper's own setting (Section 4.1: one conv weight set per layer shared by its heads,
+    keys stacked on values as the conv input) for a whole 32-layer prefill of 4096 tokens, one layer after the
+    other on one stream; the projections and MLPs around the attention are not part of this library."""
+    import torch
+
+    from paper_2406_05317_b200 import api, workloads as wl
+    w = wl.CONFIGS[WORKLOAD].slice(c_in_mult=2)
+    g = torch.Generator(device="cuda").manual_seed(7000)
+    shape = (w.batch, w.heads, w.L, w.d)
+    Q, K, V = ((torch.randn(shape, device="cuda", generator=g) * w.qkv_scale).to(torch.bfloat16) for _ in range(3))
+    O = torch.empty_like(Q)
+    ctxs, caches = [], []
+    for _ in range(layers):
+        ctx = api.Lococo(w.batch, w.heads, w.d, w.M, w.k, w.B, dtype=torch.bfloat16, c_in=w.c_in, weights_per_head=False)
+        ctx.set_weights((torch.randn((1, w.M, w.c_in, w.k), device="cuda", generator=g) * w.g_std).to(torch.bfloat16))
+        ctxs.append(ctx)
+        caches.append((torch.zeros(w.batch, w.heads, w.M, w.d, dtype=torch.bfloat16, device="cuda"),
+                       torch.zeros(w.batch, w.heads, w.M, w.d, dtype=torch.bfloat16, device="cuda")))
+    side = torch.cuda.Stream()
+    torch.cuda.synchronize()
+    ms = 0.0
+    with torch.cuda.stream(side):
+        for it in range(3 + runs):
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record()
+            for ctx, (Kc, Vc) in zip(ctxs, caches):
+                ctx.process_sequence(Q, K, V, w.B, O, Kc, Vc, 0)
+            b.record()
+            b.synchronize()
+            if it >= 3:
+                ms += a.elapsed_time(b) / runs
+    assert all(c.device_status() == api.OK for c in ctxs)
+    return {"workload": f"{layers} layers x ({WORKLOAD} shapes, conv weights shared by the heads of a layer, c_in = 2d), 4096-token prefill",
+            "ms": ms, "ms_per_layer": ms / layers, "tokens_per_s_all_layers": w.batch * w.L / (ms * 1e-3)}
 
 
 def main():
