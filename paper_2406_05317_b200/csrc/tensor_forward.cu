@@ -25,6 +25,21 @@ namespace {
 
 using namespace tc;
 
+// The kernels of the chunk loop are launched so that they may start while the kernel before them in the
+// stream drains (programmatic dependent launch): their CTAs take SMs as they fall free, let the kernel
+// after them do the same, and wait for the earlier kernels' results only where they first need them —
+// a step's attention CTAs before their cache tiles (which they process last), its compress CTAs before
+// they stage cache rows or, if their tiles lie in the chunk, before they store their partial blends
+// (the earlier finalize pass still reads that buffer). Everything before that point overlaps the tail
+// of the previous step and its finalize pass. Without the launch attribute the wait is a no-op.
+__device__ __forceinline__ void overlap_with_neighbours() {
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+}
+__device__ __forceinline__ void wait_for_earlier_kernels() {
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+}
+
+
 constexpr int kSlots = 128;              // slots per CTA (MMA M)
 constexpr int kD = 128;                  // head dimension
 constexpr int kStageBytes = 32768;       // one tap x 128 channels x 128 slots, bf16
@@ -83,6 +98,9 @@ __device__ __forceinline__ void compress_body(const TcCompressParams& P, uint8_t
     const int n_tile = P.n_tile, pad = (p.k - 1) / 2, rows = n_tile + p.k - 1;
     const int NS = P.stages;
     const uint32_t lbo_z = (uint32_t)P.rows_pad * 16u;
+    // does this CTA read cache rows (or write the cache itself)? then the earlier kernels come first
+    const bool touches_cache = P.direct || part * P.tiles_per_part * n_tile - pad < p.xk.c;
+    if (touches_cache) wait_for_earlier_kernels();
 
     uint8_t* ring_ptr = smem;
     uint8_t* zk_ptr = ring_ptr + (size_t)NS * kStageBytes;
@@ -292,6 +310,7 @@ __device__ __forceinline__ void compress_body(const TcCompressParams& P, uint8_t
     } else
     // ---- partial blends and row sums of this CTA's tiles
     if (tile_it > 0) {
+        if (!touches_cache) wait_for_earlier_kernels();      // the partial buffer may still be read by the last finalize pass
         tc_fence_after();
         float* sums = reinterpret_cast<float*>(ring_ptr);      // [3 groups][128 rows]; the ring is idle now
         sums[eg * kSlots + rl] = ssum;
@@ -387,16 +406,6 @@ __device__ __forceinline__ void finalize_tile(const TcCompressParams& P, float (
     }
 }
 
-// Launched so that it may start while the kernel before it in the stream drains (programmatic
-// dependent launch): its CTAs take SMs as they fall free, let the kernel after them do the same, and
-// only then wait for the earlier kernel's results.
-__device__ __forceinline__ void overlap_with_neighbours() {
-    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
-}
-__device__ __forceinline__ void wait_for_earlier_kernels() {
-    asm volatile("griddepcontrol.wait;" ::: "memory");
-}
-
 __global__ void __launch_bounds__(256) finalize_parts_kernel(TcCompressParams P) {
     __shared__ float tk[32][33], tv[32][33], inv_s[32];
     overlap_with_neighbours();
@@ -490,6 +499,10 @@ __device__ __forceinline__ void attention_body(const TcAttnParams& P, const CUte
     const int last_row = min(r0 + 127, p.b - 1);
     const int ncols = p.c + last_row + 1;           // columns any query of this tile can see
     const int ntiles = (ncols + 127) / 128;
+    // Key tiles are processed chunk first, cache last (the softmax does not care about the order): the tiles
+    // that hold cache rows are the only ones that depend on the previous step's result.
+    const int cache_tiles = min(ntiles, (p.c + 127) / 128);
+    auto tile_of = [&](int jt) { const int a = jt + cache_tiles; return a >= ntiles ? a - ntiles : a; };
 
     if (warp >= 9) {
         // ---------------- loader: one lane drives the copy engine; the three warps together stage what
@@ -532,7 +545,8 @@ __device__ __forceinline__ void attention_body(const TcAttnParams& P, const CUte
             const CatView& x = which ? p.xv : p.xk;
             const uint32_t dst = (which ? vs : ks) + buf * kTileBytes;
             const uint32_t bar = which ? v_full(buf) : k_full(buf);
-            const int jb = jt * 128;
+            const int jb = tile_of(jt) * 128;
+            if (jb < p.c) wait_for_earlier_kernels();          // cache rows: the previous step's result
             if (jb + 128 <= p.c) {
                 const int mi = kMapKCache + which;
                 if ((mask >> mi) & 1) {
@@ -585,6 +599,7 @@ __device__ __forceinline__ void attention_body(const TcAttnParams& P, const CUte
             mbar_wait(pv_done(b), ph, P.status, failed, 5);
             load_kv(t, b, 1);
         }
+        if (cache_tiles == 0) wait_for_earlier_kernels();   // keeps the chain of waits unbroken
     } else if (tid == kMma) {
         // ---------------- MMA issuer: S(0), then per tile S(t) followed by PV(t-1)
         const uint32_t idesc_s = instr_desc_bf16(128, false, false);
@@ -625,7 +640,7 @@ __device__ __forceinline__ void attention_body(const TcAttnParams& P, const CUte
     if (warp < 8) {
         // ---------------- softmax
         float m_used = 0.f, lrun = 0.f;
-        const int vis = live ? p.c + row + 1 : 1;   // visible columns of this row
+        const int vis = live ? p.c + row + 1 : (1 << 30);   // visible columns of this row (rows past the chunk are all zeros)
         const float sc2 = p.scale * 1.4426950408889634f;
         // the two threads of a row exchange their maxima rounded to bf16, one slot per tile parity:
         // both then derive the same reference maximum, which only has to be near the true one
@@ -635,8 +650,9 @@ __device__ __forceinline__ void attention_body(const TcAttnParams& P, const CUte
             mbar_wait(s_full(b), (jt >> 1) & 1, P.status, failed, 9);
             tc_fence_after();
             const uint32_t s_addr = lane_base + b * 128 + half * 64;
-            const int j0 = jt * 128 + half * 64;
-            const bool need_mask = jt * 128 + 128 > p.c + r0;
+            const int at = tile_of(jt);                   // the key tile this round works on
+            const int j0 = at * 128 + half * 64;
+            const bool need_mask = at * 128 + 128 > p.c + r0;
             if (jt >= 2) mbar_wait(pv_done(b), ((jt >> 1) - 1) & 1, P.status, failed, 11);   // P buffer b is free
             uint8_t* pdst = p_ptr + b * kPBytes + rl * 16;
             // One sweep over this thread's 64 logits: P = exp2(s - m) in bf16 into the A-operand layout
@@ -675,7 +691,7 @@ __device__ __forceinline__ void attention_body(const TcAttnParams& P, const CUte
                 xmax[b * 256 + half * 128 + rl] = mine;
                 asm volatile("bar.sync 1, 256;" ::: "memory");
                 const float mt = fmaxf(__bfloat162float(mine), __bfloat162float(xmax[b * 256 + (half ^ 1) * 128 + rl]));
-                // column 0 is visible to every row, so mt of the first tile is finite
+                // the first tile worked on holds a key every row sees (the chunk's first, or key 0), so mt is finite there
                 const bool bump = jt == 0 || mt > m_used + kRescaleThreshold;
                 if (!__any_sync(0xffffffffu, bump)) break;
                 if (jt > 0) {
@@ -780,8 +796,7 @@ __global__ void __launch_bounds__(kAttnThreads, 1) chunk_step_tc_kernel(const __
     __shared__ uint32_t tmem_slot;
     overlap_with_neighbours();
     const uint32_t tmem = cta_tmem_acquire(&tmem_slot);
-    wait_for_earlier_kernels();
-    step_item(P, smem, tmem, false, blockIdx.x);
+    step_item(P, smem, tmem, false, blockIdx.x);     // the bodies wait for the earlier kernels where they need them
     cta_tmem_release(tmem);
 }
 
