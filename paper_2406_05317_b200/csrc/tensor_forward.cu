@@ -100,7 +100,6 @@ __device__ __forceinline__ void compress_body(const TcCompressParams& P, uint8_t
     const uint32_t lbo_z = (uint32_t)P.rows_pad * 16u;
     // does this CTA read cache rows (or write the cache itself)? then the earlier kernels come first
     const bool touches_cache = P.direct || part * P.tiles_per_part * n_tile - pad < p.xk.c;
-    if (touches_cache) wait_for_earlier_kernels();
 
     uint8_t* ring_ptr = smem;
     uint8_t* zk_ptr = ring_ptr + (size_t)NS * kStageBytes;
@@ -158,7 +157,8 @@ __device__ __forceinline__ void compress_body(const TcCompressParams& P, uint8_t
         }
         // ---- 1. stage the key and value rows j0-pad .. j0+n_tile+pad-1 (zeros outside [0,S))
         // each thread owns one 8-channel group (q) and every (threads/16)-th row
-        auto stage_tile = [&](const CatView& xv_, uint32_t dst, int first, int step) {
+        // `rows_of`: 0 all rows, 1 only rows outside the cache (chunk rows and padding), 2 only cache rows
+        auto stage_tile = [&](const CatView& xv_, uint32_t dst, int first, int step, int rows_of = 0) {
             const int q = first & 15;
             const __nv_bfloat16* cbase = unit_base<__nv_bfloat16>(xv_.cache, n, h) + q * 8;
             const __nv_bfloat16* kbase = unit_base<__nv_bfloat16>(xv_.chunk, n, h) + q * 8;
@@ -167,16 +167,26 @@ __device__ __forceinline__ void compress_body(const TcCompressParams& P, uint8_t
                 const int j = j0 - pad + r;
                 const bool valid = j >= 0 && j < p.S;
                 const bool in_cache = valid && j < xv_.c;
+                if ((rows_of == 1 && in_cache) || (rows_of == 2 && !in_cache)) continue;
                 const __nv_bfloat16* src = !valid ? safe : (in_cache ? cbase + (int64_t)j * xv_.cache.st
                                                                      : kbase + (int64_t)(j - xv_.c) * xv_.chunk.st);
                 if (in_cache && cache_cg) cp_async16_cg(d0 + r * 16, src, 16u);
                 else cp_async16(d0 + r * 16, src, valid ? 16u : 0u);
             }
         };
-        stage_tile(p.xk, zk, tid, nthr16);
         // the value tile is a conv input only when c_in = 2d; otherwise it is needed by the
         // blend only and is staged by the epilogue warps while the conv runs
-        if (P.halves == 2) stage_tile(p.xv, zv, tid, nthr16);
+        if (touches_cache) {
+            // chunk rows (and the weight ring's first stages) before the wait for the previous step, cache rows after
+            stage_tile(p.xk, zk, tid, nthr16, 1);
+            if (P.halves == 2) stage_tile(p.xv, zv, tid, nthr16, 1);
+            wait_for_earlier_kernels();
+            stage_tile(p.xk, zk, tid, nthr16, 2);
+            if (P.halves == 2) stage_tile(p.xv, zv, tid, nthr16, 2);
+        } else {
+            stage_tile(p.xk, zk, tid, nthr16);
+            if (P.halves == 2) stage_tile(p.xv, zv, tid, nthr16);
+        }
         cp_async_wait_all();
         fence_proxy_async();
         __syncthreads();
