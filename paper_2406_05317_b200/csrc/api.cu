@@ -364,6 +364,7 @@ lococo_status run_chunk_loop(lococo_handle* h, lococo_tensor Q, lococo_tensor K,
     const size_t e = h->elt;
     int c = *c_inout;
     h->seq_count = 0;   // nothing is left queued from a call that failed half-way
+    h->chain_open = false;
     const int n_chunks = (L + B - 1) / B;
     const size_t snap_step = (size_t)h->units * cfg.M * cfg.head_dim * e;
     const size_t snap_all = align_up((size_t)n_chunks * snap_step, 256);

@@ -25,6 +25,9 @@ struct lococo_handle {
     size_t elt = 0;         // bytes per stored element
     float scale = 0.f;      // softmax scale in effect
     bool use_tensor = false;
+    // true once a kernel of this library has been launched in the current call: only then may the next one be
+    // launched as a programmatic dependent (its early, pre-wait reads must not race with a foreign kernel)
+    bool chain_open = false;
     bool persistent_loop = false;   // chunk loop as one cooperative launch (LOCOCO_PATH_TENSOR_PERSISTENT)
     bool weights_set = false;
     bool has_bias = false;

@@ -1101,7 +1101,8 @@ static bool build_compress_params(lococo_handle* h, const CompressParams& p, boo
 // Launch that lets the kernel begin while its predecessor in the stream is still draining; the kernel
 // itself waits (wait_for_earlier_kernels) before it touches anything the predecessor produces.
 template <typename Param>
-static cudaError_t launch_overlapped(void (*kernel)(Param), dim3 grid, dim3 block, size_t smem, cudaStream_t st, const Param& arg) {
+static cudaError_t launch_overlapped(void (*kernel)(Param), dim3 grid, dim3 block, size_t smem, cudaStream_t st, const Param& arg,
+                                     bool overlap = true) {
     cudaLaunchConfig_t cfg{};
     cfg.gridDim = grid;
     cfg.blockDim = block;
@@ -1111,7 +1112,7 @@ static cudaError_t launch_overlapped(void (*kernel)(Param), dim3 grid, dim3 bloc
     attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
-    cfg.numAttrs = 1;
+    cfg.numAttrs = overlap ? 1 : 0;
     return cudaLaunchKernelEx(&cfg, kernel, arg);
 }
 
@@ -1239,7 +1240,10 @@ int tensor_chunk_step(lococo_handle* h, const AttnParams& a, const CompressParam
     P.comp.direct = P.comp.parts == 1 && p.W_out == nullptr && p.k_out.ptr != p.xk.cache.ptr && p.v_out.ptr != p.xv.cache.ptr;
     const int blocks = P.n_attn + a.units * P.comp_per_unit;
     prof_begin(p.prof, 2, st);
-    const bool ok = launch_overlapped(chunk_step_tc_kernel, dim3(blocks), dim3(kAttnThreads), kMaxSmem, st, P) == cudaSuccess;
+    // the step's CTAs read the chunk before they wait for earlier kernels: the first step of a call is therefore
+    // launched in plain stream order, after whatever the caller ran before (it may have produced Q, K, V)
+    const bool ok = launch_overlapped(chunk_step_tc_kernel, dim3(blocks), dim3(kAttnThreads), kMaxSmem, st, P, h->chain_open) == cudaSuccess;
+    h->chain_open = true;
     if (!ok) cudaGetLastError();
     prof_end(p.prof, st);
     if (!ok) return -1;
