@@ -957,7 +957,8 @@ __global__ void __launch_bounds__(kAttnThreads, 1) sequence_tc_kernel(const __gr
             __syncthreads();
         }
         // within a unit: compress CTAs first (the longest), then the attention tiles, longest first
-        if (r < P.comp_per_unit) compress_body(P.comp, smem, tmem, false, r % P.comp.parts, r / P.comp.parts, u);
+        // (cache rows rewritten by other SMs earlier in this same kernel are read around L1)
+        if (r < P.comp_per_unit) compress_body(P.comp, smem, tmem, n > 0, r % P.comp.parts, r / P.comp.parts, u);
         else attention_body(P.attn, Q.steps[n].attn.maps, true, smem, tmem, P.qtiles - 1 - (r - P.comp_per_unit), u);
         __syncthreads();
         if (threadIdx.x == 0) {

@@ -93,6 +93,17 @@ def test_cfg4_slice(api, orc, path):
     check_sequence(api, orc, wl.CONFIGS["cfg4"].slice(heads=2, B=1024, L=3072), path)
 
 
+def test_tensor_path_ragged_chunks_direct_cache_write(api, orc):
+    # tensor-core path with sizes that are multiples of nothing the kernels tile by: B = 100, a short last
+    # chunk, a first compress step on a partly filled cache (c = 100), several sequences; with this many
+    # units every compress CTA sees all positions of its slots and writes the new cache itself, so the loop
+    # alternates between the caller's cache and the workspace's (11 compress steps: the result ends up in
+    # the workspace's cache and is copied back)
+    w = wl.Workload("tc_ragged", 13, batch=3, heads=2, d=128, M=128, B=100, k=9, L=1177, dtype="bf16",
+                    weights_per_head=True, qkv_scale=0.0884, g_std=0.02)
+    check_sequence(api, orc, w, 0, bias=True)
+
+
 @pytest.mark.parametrize("path", [0, 1])
 def test_generation_mode_chunk_of_one_token(api, orc, path):
     # B = 1 (the generation stage of Section 3.3 sets the segment length to 1): 128 fill steps, then every step compresses
