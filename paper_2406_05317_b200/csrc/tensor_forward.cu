@@ -685,19 +685,21 @@ __device__ __forceinline__ void attention_body(const TcAttnParams& P, const CUte
 #pragma unroll
                         for (int x = 0; x < 8; x += 2) {
                             const int ja = j0 + c0 + e + x;
-                            const float sa = __uint_as_float(v[e + x]) * sc2, sb2 = __uint_as_float(v[e + x + 1]) * sc2;
-                            float pa = exp2f(sa - m_used), pb = exp2f(sb2 - m_used);
-                            if (need_mask && ja >= vis) pa = 0.f; else tmax = fmaxf(tmax, sa);
-                            if (need_mask && ja + 1 >= vis) pb = 0.f; else tmax = fmaxf(tmax, sb2);
+                            // one FMA per logit: exp2(s * scale - m); the maximum is tracked on the raw logits
+                            // and scaled once per tile (the scale is positive)
+                            const float ra = __uint_as_float(v[e + x]), rb = __uint_as_float(v[e + x + 1]);
+                            float pa = exp2f(fmaf(ra, sc2, -m_used)), pb = exp2f(fmaf(rb, sc2, -m_used));
+                            if (need_mask && ja >= vis) pa = 0.f; else tmax = fmaxf(tmax, ra);
+                            if (need_mask && ja + 1 >= vis) pb = 0.f; else tmax = fmaxf(tmax, rb);
                             const __nv_bfloat162 pr = __floats2bfloat162_rn(pa, pb);
                             pk[x >> 1] = *reinterpret_cast<const uint32_t*>(&pr);
-                            lsum += __low2float(pr) + __high2float(pr);
+                            lsum += pa + pb;   // the row sum takes the unrounded terms (fp32)
                         }
                         *reinterpret_cast<uint4*>(pdst + ((half * 64 + c0 + e) >> 3) * 2048) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
                     }
                 }
                 if (attempt == 1) break;
-                const __nv_bfloat16 mine = __float2bfloat16_rn(tmax);
+                const __nv_bfloat16 mine = __float2bfloat16_rn(tmax * sc2);
                 xmax[b * 256 + half * 128 + rl] = mine;
                 asm volatile("bar.sync 1, 256;" ::: "memory");
                 const float mt = fmaxf(__bfloat162float(mine), __bfloat162float(xmax[b * 256 + (half ^ 1) * 128 + rl]));
