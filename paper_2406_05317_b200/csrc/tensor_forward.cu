@@ -16,6 +16,7 @@
 #include <cuda.h>   // tensor map types only: the encoder is looked up at run time
 
 #include <algorithm>
+#include <type_traits>
 
 #include "handle.h"
 #include "tc_common.cuh"
@@ -671,9 +672,10 @@ __device__ __forceinline__ void attention_body(const TcAttnParams& P, const CUte
             // than the threshold (always for the first tile, rarely later) is m raised, O rescaled and
             // the sweep repeated; a P that overflowed in the discarded sweep is simply overwritten.
             float lsum = 0.f;
-            for (int attempt = 0; attempt < 2; ++attempt) {
-                float tmax = -INFINITY;
-                lsum = 0.f;
+            // (compiled twice: tiles that the causal limit crosses test every column, the others none)
+            auto sweep = [&](auto masked, float& tmax) {
+                constexpr bool kMasked = decltype(masked)::value;
+                float sum = 0.f;
 #pragma unroll
                 for (int c0 = 0; c0 < 64; c0 += 32) {
                     uint32_t v[32];
@@ -689,15 +691,20 @@ __device__ __forceinline__ void attention_body(const TcAttnParams& P, const CUte
                             // and scaled once per tile (the scale is positive)
                             const float ra = __uint_as_float(v[e + x]), rb = __uint_as_float(v[e + x + 1]);
                             float pa = exp2f(fmaf(ra, sc2, -m_used)), pb = exp2f(fmaf(rb, sc2, -m_used));
-                            if (need_mask && ja >= vis) pa = 0.f; else tmax = fmaxf(tmax, ra);
-                            if (need_mask && ja + 1 >= vis) pb = 0.f; else tmax = fmaxf(tmax, rb);
+                            if (kMasked && ja >= vis) pa = 0.f; else tmax = fmaxf(tmax, ra);
+                            if (kMasked && ja + 1 >= vis) pb = 0.f; else tmax = fmaxf(tmax, rb);
                             const __nv_bfloat162 pr = __floats2bfloat162_rn(pa, pb);
                             pk[x >> 1] = *reinterpret_cast<const uint32_t*>(&pr);
-                            lsum += pa + pb;   // the row sum takes the unrounded terms (fp32)
+                            sum += pa + pb;   // the row sum takes the unrounded terms (fp32)
                         }
                         *reinterpret_cast<uint4*>(pdst + ((half * 64 + c0 + e) >> 3) * 2048) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
                     }
                 }
+                return sum;
+            };
+            for (int attempt = 0; attempt < 2; ++attempt) {
+                float tmax = -INFINITY;
+                lsum = need_mask ? sweep(std::true_type{}, tmax) : sweep(std::false_type{}, tmax);
                 if (attempt == 1) break;
                 const __nv_bfloat16 mine = __float2bfloat16_rn(tmax * sc2);
                 xmax[b * 256 + half * 128 + rl] = mine;
