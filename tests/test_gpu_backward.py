@@ -103,3 +103,11 @@ def test_backward_bf16_tensor_path_per_head_fill_then_partial_cache_bias():
     w = wl.Workload("bwd_tc_fill", 35, batch=2, heads=2, d=128, M=256, B=96, k=5, L=420, dtype="bf16",
                     weights_per_head=True, qkv_scale=0.0884, g_std=0.02)
     check_backward(w, bias=True)
+
+
+def test_backward_bf16_tensor_path_per_head_stacked_input():
+    # tensor-core backward: one weight set per head AND keys stacked on values as the conv input
+    # (the weight gradient's column index runs over taps and both 128-channel halves)
+    w = wl.Workload("bwd_tc_ph2d", 36, batch=2, heads=2, d=128, M=128, B=160, k=5, L=480, dtype="bf16",
+                    weights_per_head=True, qkv_scale=0.0884, g_std=0.02, c_in_mult=2)
+    check_backward(w)
