@@ -109,6 +109,10 @@ __global__ void __launch_bounds__(kThreads, 2) gemm_kernel(const __grid_constant
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem = *reinterpret_cast<volatile uint32_t*>(&tmem_slot);
+    // launched as a programmatic dependent: the set-up above overlaps the previous kernel's tail, and
+    // nothing global is touched before that kernel's results are complete and visible
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    asm volatile("griddepcontrol.wait;" ::: "memory");
 
     if (tid == 288) {
         // ---- producer
@@ -321,8 +325,21 @@ inline bool launch(const Params& P, int m_tiles, int n_tiles, int batch, cudaStr
         if (cudaFuncSetAttribute(gemm_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmem) != cudaSuccess) return false;
         attr_set = true;
     }
-    gemm_kernel<<<dim3(m_tiles, n_tiles, batch * P.splits), kThreads, kSmem, st>>>(P);
-    return cudaGetLastError() == cudaSuccess;
+    cudaLaunchConfig_t cfg{};
+    cfg.gridDim = dim3(m_tiles, n_tiles, batch * P.splits);
+    cfg.blockDim = dim3(kThreads);
+    cfg.dynamicSmemBytes = kSmem;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    if (cudaLaunchKernelEx(&cfg, gemm_kernel, P) != cudaSuccess) {
+        cudaGetLastError();
+        return false;
+    }
+    return true;
 }
 
 }  // namespace gemm
