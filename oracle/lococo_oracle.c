@@ -28,7 +28,14 @@
  *   - Eq. 7's denominator is sum_k W_ik + eps;
  *   - a compress step with a partly filled cache (c < M, c + b > M) sees only
  *     the S = c + b real entries;
- *   - the mask of Eq. 1 is the usual additive -inf mask.
+ *   - the mask of Eq. 1 is the usual additive -inf mask;
+ *   - protected slots (Section 5.2, Table 6: the compressor next to an eviction
+ *     policy that always keeps some tokens, e.g. the initial "sink" tokens):
+ *     the paper gives no formula; here rows i < protected_slots of the weight
+ *     matrix w are the unit rows e_i, so slot i keeps entry i of [cache; chunk]
+ *     unchanged (the tokens that filled those slots first), the conv still reads
+ *     every entry, and no gradient reaches the conv weights of those rows.
+ *     Cache-first order only.
  *
  * Parity status: every function below is pinned by tests/test_oracle_*.py
  * (textbook correlation, closed forms, hand-worked fixtures, one-hot gather,
@@ -50,7 +57,7 @@ typedef struct {
     int32_t k;       /* conv kernel width (odd) */
     int32_t c_in;    /* conv input channels: d or 2d */
     int32_t flags;   /* LOCOCO_ORACLE_* */
-    int32_t pad_;
+    int32_t protected_slots; /* first slots kept verbatim (Section 5.2); 0 = plain method */
     double eps;      /* added to Eq. 7's denominator */
     double scale;    /* softmax scale, 1/sqrt(d) in Eq. 1 */
 } oracle_params;
@@ -104,6 +111,16 @@ void lococo_oracle_compress(const oracle_params* P, const double* XK, const doub
     build_conv_input(P, XK, XV, S, Z);
     lococo_oracle_conv_logits(Z, S, C, G, bias, M, P->k, A);
     for (int i = 0; i < M; ++i) {
+        if (i < P->protected_slots) {
+            /* Section 5.2: w_i = e_i, the slot keeps entry i as it is */
+            if (s_out) s_out[i] = 1.0;
+            for (int j = 0; j < S && w_out; ++j) w_out[(size_t)i * S + j] = j == i ? 1.0 : 0.0;
+            for (int c = 0; c < d; ++c) {
+                Knew[(size_t)i * d + c] = XK[(size_t)i * d + c];
+                Vnew[(size_t)i * d + c] = XV[(size_t)i * d + c];
+            }
+            continue;
+        }
         double s = 0.0;
         for (int j = 0; j < S; ++j) {
             double r = A[(size_t)i * S + j];
@@ -295,6 +312,7 @@ static void compress_backward(const oracle_params* P, const double* XK, const do
         for (int j = 0; j < S; ++j) {
             const double dR = (dA[(size_t)i * S + j] - inner) / s[i];
             dA[(size_t)i * S + j] = A[(size_t)i * S + j] > 0.0 ? dR : 0.0;
+            if (i < P->protected_slots) dA[(size_t)i * S + j] = 0.0;   /* constant row: nothing flows to Eq. 6 */
         }
     }
     /* through Eq. 6 */

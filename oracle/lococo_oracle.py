@@ -36,7 +36,7 @@ def build(force: bool = False) -> Path:
 
 class _Params(ctypes.Structure):
     _fields_ = [("d", ctypes.c_int32), ("M", ctypes.c_int32), ("k", ctypes.c_int32),
-                ("c_in", ctypes.c_int32), ("flags", ctypes.c_int32), ("pad_", ctypes.c_int32),
+                ("c_in", ctypes.c_int32), ("flags", ctypes.c_int32), ("protected_slots", ctypes.c_int32),
                 ("eps", ctypes.c_double), ("scale", ctypes.c_double)]
 
 
@@ -65,10 +65,11 @@ def _p(a):
     return None if a is None else a.ctypes.data_as(ctypes.c_void_p)
 
 
-def _params(d, M, k, c_in, eps, scale, flags):
+def _params(d, M, k, c_in, eps, scale, flags, protected=0):
     if scale is None or scale == 0:
         scale = 1.0 / np.sqrt(d)
-    return _Params(d, M, k, c_in, flags, 0, float(eps), float(scale))
+    assert 0 <= protected <= M and not (protected and flags & 1)   # Section 5.2 reading: cache-first order only
+    return _Params(d, M, k, c_in, flags, int(protected), float(eps), float(scale))
 
 
 def conv_logits(Z, G, bias=None):
@@ -83,14 +84,14 @@ def conv_logits(Z, G, bias=None):
     return A
 
 
-def compress(XK, XV, G, bias=None, eps=1e-6, flags=0, want_weights=False):
+def compress(XK, XV, G, bias=None, eps=1e-6, flags=0, want_weights=False, protected=0):
     """Eq. 6 -> ReLU -> Eq. 7 -> Eq. 4, Eq. 5: XK, XV [S,d] -> new cache K, V [M,d]."""
     XK, XV, G = _f64(XK), _f64(XV), _f64(G)
     S, d = XK.shape
     M, C, k = G.shape
     assert XV.shape == (S, d) and C in (d, 2 * d) and k % 2 == 1
     b = None if bias is None else _f64(bias)
-    P = _params(d, M, k, C, eps, None, flags)
+    P = _params(d, M, k, C, eps, None, flags, protected)
     Kn, Vn = np.empty((M, d)), np.empty((M, d))
     w = np.empty((M, S)) if want_weights else None
     A = np.empty((M, S)) if want_weights else None
@@ -115,7 +116,7 @@ def attention(Q, XK, XV, c, scale=None, want_prob=False):
     return (O, lse, prob) if want_prob else (O, lse)
 
 
-def update_cache(Kc, Vc, c, Kn, Vn, G, bias=None, eps=1e-6, flags=0):
+def update_cache(Kc, Vc, c, Kn, Vn, G, bias=None, eps=1e-6, flags=0, protected=0):
     """Algorithm 2's if/else after Step 3: returns the new (Kc [M,d], Vc [M,d], c)."""
     G = _f64(G)
     M, C, k = G.shape
@@ -124,20 +125,20 @@ def update_cache(Kc, Vc, c, Kn, Vn, G, bias=None, eps=1e-6, flags=0):
     b, d = Kn.shape
     assert Kc.shape == (M, d)
     bb = None if bias is None else _f64(bias)
-    P = _params(d, M, k, C, eps, None, flags)
+    P = _params(d, M, k, C, eps, None, flags, protected)
     cc = ctypes.c_int(c)
     _load().lococo_oracle_update_cache(ctypes.byref(P), _p(Kc), _p(Vc), ctypes.byref(cc), _p(Kn), _p(Vn), b,
                                        _p(G), _p(bb))
     return Kc, Vc, cc.value
 
 
-def process_sequence(Q, K, V, G, B, bias=None, eps=1e-6, scale=None, flags=0, cache=None, want_snapshots=False):
+def process_sequence(Q, K, V, G, B, bias=None, eps=1e-6, scale=None, flags=0, cache=None, want_snapshots=False, protected=0):
     """Algorithm 2 for one unit: Q, K, V [L,d] -> O [L,d], final cache (Kc, Vc [M,d], c), lse [L]."""
     Q, K, V, G = _f64(Q), _f64(K), _f64(V), _f64(G)
     L, d = Q.shape
     M, C, k = G.shape
     bb = None if bias is None else _f64(bias)
-    P = _params(d, M, k, C, eps, scale, flags)
+    P = _params(d, M, k, C, eps, scale, flags, protected)
     if cache is None:
         Kc, Vc, c = np.zeros((M, d)), np.zeros((M, d)), 0
     else:
@@ -154,14 +155,14 @@ def process_sequence(Q, K, V, G, B, bias=None, eps=1e-6, scale=None, flags=0, ca
     return out + (sK, sV, sc) if want_snapshots else out
 
 
-def process_sequence_grad(Q, K, V, G, B, dO, dKc_final, dVc_final, bias=None, eps=1e-6, scale=None):
+def process_sequence_grad(Q, K, V, G, B, dO, dKc_final, dVc_final, bias=None, eps=1e-6, scale=None, protected=0):
     """Gradients of <dO,O> + <dKc_final,Kc_final> + <dVc_final,Vc_final> through Algorithm 2
     (empty initial cache): returns dQ, dK, dV [L,d], dG [M,C,k], dbias [M] or None."""
     Q, K, V, G = _f64(Q), _f64(K), _f64(V), _f64(G)
     L, d = Q.shape
     M, C, k = G.shape
     bb = None if bias is None else _f64(bias)
-    P = _params(d, M, k, C, eps, scale, 0)
+    P = _params(d, M, k, C, eps, scale, 0, protected)
     dO, dKf, dVf = _f64(dO), _f64(dKc_final), _f64(dVc_final)
     dQ, dK, dV = np.zeros((L, d)), np.zeros((L, d)), np.zeros((L, d))
     dG = np.zeros((M, C, k))
@@ -172,7 +173,7 @@ def process_sequence_grad(Q, K, V, G, B, dO, dKc_final, dVc_final, bias=None, ep
     return dQ, dK, dV, dG, db
 
 
-def process_batch(Q, K, V, G, B, bias=None, eps=1e-6, scale=None, flags=0):
+def process_batch(Q, K, V, G, B, bias=None, eps=1e-6, scale=None, flags=0, protected=0):
     """Algorithm 2 for [batch, heads, L, d] inputs; G [heads|1, M, C, k].  OpenMP across units.
     Returns O [batch,heads,L,d], Kc, Vc [batch,heads,M,d], c [batch,heads], lse [batch,heads,L]."""
     Q, K, V, G = _f64(Q), _f64(K), _f64(V), _f64(G)
@@ -180,7 +181,7 @@ def process_batch(Q, K, V, G, B, bias=None, eps=1e-6, scale=None, flags=0):
     Hg, M, C, k = G.shape
     assert Hg in (1, H)
     bb = None if bias is None else _f64(bias)
-    P = _params(d, M, k, C, eps, scale, flags)
+    P = _params(d, M, k, C, eps, scale, flags, protected)
     units = Bt * H
     O = np.empty((Bt, H, L, d))
     Kc, Vc = np.zeros((Bt, H, M, d)), np.zeros((Bt, H, M, d))
@@ -194,13 +195,13 @@ def process_batch(Q, K, V, G, B, bias=None, eps=1e-6, scale=None, flags=0):
     return O, Kc, Vc, c, lse
 
 
-def grad_batch(Q, K, V, G, B, dO, dKc_final, dVc_final, bias=None, eps=1e-6, scale=None):
+def grad_batch(Q, K, V, G, B, dO, dKc_final, dVc_final, bias=None, eps=1e-6, scale=None, protected=0):
     """Batched process_sequence_grad; dG is summed over the units sharing a weight set."""
     Q, K, V, G = _f64(Q), _f64(K), _f64(V), _f64(G)
     Bt, H, L, d = Q.shape
     Hg, M, C, k = G.shape
     bb = None if bias is None else _f64(bias)
-    P = _params(d, M, k, C, eps, scale, 0)
+    P = _params(d, M, k, C, eps, scale, 0, protected)
     dO, dKf, dVf = _f64(dO), _f64(dKc_final), _f64(dVc_final)
     dQ, dK, dV = np.zeros_like(Q), np.zeros_like(Q), np.zeros_like(Q)
     dG = np.zeros_like(G)
