@@ -105,6 +105,16 @@ lococo_status lococo_set_workspace(lococo_handle* handle, void* device_ptr, size
 lococo_status lococo_set_weights(lococo_handle* handle, const void* G_device, const void* bias_device,
                                  void* stream);
 
+/* Protected slots (Section 5.2, Table 6: the compressor next to an eviction policy that always
+ * keeps some tokens, such as the initial "sink" tokens).  The paper gives no formula; this
+ * library's reading: for the first `slots` cache slots the row of Eq. 7's weight matrix is the
+ * unit row e_i, so slot i keeps entry i of [cache; chunk] bit for bit (after the fill steps:
+ * token i of the sequence), the convolution still reads every entry, the other slots are
+ * compressed as before, and no gradient reaches the conv weights of those rows.
+ * 0 <= slots <= M; 0 (the default) is the plain method.  Host-side state only: it applies to
+ * every later compress step, chunk loop and backward pass of this handle. */
+lococo_status lococo_set_protected_slots(lococo_handle* handle, int32_t slots);
+
 /*
  * Algorithm 2, the branch after Step 3.  With c = cache_len:
  *   c + b <= M : fill - chunk rows are appended at cache rows c..c+b-1;

@@ -42,6 +42,7 @@ _SIGNATURES = {
     "lococo_workspace_bytes": [_P, ctypes.POINTER(ctypes.c_size_t)],
     "lococo_set_workspace": [_P, _P, ctypes.c_size_t, _P],
     "lococo_set_weights": [_P, _P, _P, _P],
+    "lococo_set_protected_slots": [_P, _I],
     "lococo_compress_step": [_P, _T, _T, _I, _T, _T, _I, _T, _T, ctypes.POINTER(_I), _P, _P],
     "lococo_chunk_attention": [_P, _T, _T, _T, _I, _T, _T, _I, _T, _P, _P],
     "lococo_saved_bytes": [_P, _I, _I, ctypes.POINTER(ctypes.c_size_t)],
@@ -158,6 +159,10 @@ class Lococo:
         if bias is not None and (tuple(bias.shape) != (sets, c.M) or bias.dtype != self.torch_dtype):
             raise ValueError("bias must be [heads|1, M] in the configured dtype")
         _check(_lib.lococo_set_weights(self._h, G.data_ptr(), _ptr(bias), _stream()), "lococo_set_weights")
+
+    def set_protected_slots(self, slots: int):
+        """Section 5.2: the first `slots` cache slots keep their entries; the others are compressed."""
+        _check(_lib.lococo_set_protected_slots(self._h, int(slots)), "lococo_set_protected_slots")
 
     def compress_step(self, K_cache, V_cache, cache_len, K_chunk, V_chunk, K_out=None, V_out=None, W_out=None):
         """Algorithm 2 Steps 4-5 (or the fill branch). Returns the new cache length."""

@@ -85,6 +85,7 @@ CompressParams make_compress_params(lococo_handle* h, View kc, View vc, int c, V
     p.g_packed = h->ws + h->off_gpack;
     p.bias = h->has_bias ? reinterpret_cast<const float*>(h->ws + h->off_bias) : nullptr;
     p.eps = cfg.norm_eps;
+    p.prot = h->prot;
     p.R = reinterpret_cast<float*>(h->ws + h->off_R);
     p.s = reinterpret_cast<float*>(h->ws + h->off_s);
     p.UK = reinterpret_cast<float*>(h->ws + h->off_UK);
@@ -284,6 +285,13 @@ lococo_status lococo_set_workspace(lococo_handle* h, void* ptr, size_t bytes, vo
     h->weights_set = false;
     if (cudaMemsetAsync(h->ws + h->off_status, 0, 256, static_cast<cudaStream_t>(stream)) != cudaSuccess)
         return LOCOCO_ERR_CUDA;
+    return LOCOCO_OK;
+}
+
+lococo_status lococo_set_protected_slots(lococo_handle* h, int32_t slots) {
+    if (!h || slots < 0 || slots > h->cfg.M) return LOCOCO_ERR_INVALID_ARG;
+    if (slots != h->prot) drop_loop_graph(h);   // a cached chunk loop carries the old count in its launches
+    h->prot = slots;
     return LOCOCO_OK;
 }
 

@@ -705,7 +705,7 @@ lococo_status lococo_process_sequence_backward(lococo_handle* h, lococo_tensor Q
         f.heads = cfg.heads; f.units = h->units; f.d = cfg.head_dim; f.M = cfg.M; f.k = cfg.k; f.c_in = cfg.c_in;
         f.S = p.S; f.weights_per_head = cfg.weights_per_head; f.g_packed = p.g_packed;
         f.bias = h->has_bias ? reinterpret_cast<const float*>(h->ws + h->off_bias) : nullptr;
-        f.eps = cfg.norm_eps; f.R = p.R; f.s = p.s;
+        f.eps = cfg.norm_eps; f.prot = h->prot; f.R = p.R; f.s = p.s;
         const int r = cfg.dtype == LOCOCO_F32 ? backward_step<float>(h, p, f, cfg.dtype, B, nullptr, st)
                                               : backward_step<__nv_bfloat16>(h, p, f, cfg.dtype, B, tb, st);
         if (r < 0) return LOCOCO_ERR_CUDA;

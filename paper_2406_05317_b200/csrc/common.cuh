@@ -59,6 +59,7 @@ struct CompressParams {
     float* W_out;          // optional [units][M][S]
     void* R16;             // optional bf16 copy of R, [units][M][R16_stride] (the backward's recompute; tensor-core path only)
     int R16_stride;        // multiple of 8
+    int prot = 0;          // protected slots (Section 5.2): rows i < prot of Eq. 7's matrix are the unit rows e_i
     void* prof;            // host only: Profiler* or nullptr
 };
 

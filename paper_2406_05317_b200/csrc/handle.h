@@ -21,6 +21,7 @@ struct Profiler {
 
 struct lococo_handle {
     lococo_config cfg{};
+    int prot = 0;   // protected slots (Section 5.2)
     int units = 0;          // batch * heads
     size_t elt = 0;         // bytes per stored element
     float scale = 0.f;      // softmax scale in effect

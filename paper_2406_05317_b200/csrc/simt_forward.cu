@@ -116,14 +116,15 @@ __global__ void __launch_bounds__(256) conv_relu_kernel(CompressParams p) {
 #pragma unroll
         for (int y = 0; y < 4; ++y) {
             const int j = j0 + tj + 16 * y;
-            if (j < p.S) R[(int64_t)i * p.S + j] = fmaxf(acc[x][y] + bi, 0.f);
+            if (j < p.S) R[(int64_t)i * p.S + j] = i < p.prot ? (j == i ? 1.f : 0.f) : fmaxf(acc[x][y] + bi, 0.f);
         }
     }
 }
 
 // ------------------------------------------------------------------ Eq. 7 denominators
 // One warp per (unit, slot) row; fixed summation order.
-__global__ void rowsum_kernel(const float* __restrict__ R, float* __restrict__ s, int rows, int S, float eps) {
+// A protected slot's row is a unit row and its denominator exactly 1 (no eps), so it keeps its entry bit for bit.
+__global__ void rowsum_kernel(const float* __restrict__ R, float* __restrict__ s, int rows, int S, float eps, int M, int prot) {
     const int row = blockIdx.x * (blockDim.x / 32) + threadIdx.x / 32;
     if (row >= rows) return;
     const int lane = threadIdx.x % 32;
@@ -132,7 +133,7 @@ __global__ void rowsum_kernel(const float* __restrict__ R, float* __restrict__ s
     for (int j = lane; j < S; j += 32) acc += r[j];
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, o);
-    if (lane == 0) s[row] = acc + eps;
+    if (lane == 0) s[row] = row % M < prot ? 1.f : acc + eps;
 }
 
 // ------------------------------------------------------------------ Eq. 4, Eq. 5 (unnormalised)
@@ -365,7 +366,7 @@ static int compress_typed(const CompressParams& p, cudaStream_t st) {
     }
     {
         const int rows = p.units * p.M;
-        if (checked([&] { rowsum_kernel<<<(rows + 7) / 8, 256, 0, st>>>(p.R, p.s, rows, p.S, p.eps); }) < 0) return -1;
+        if (checked([&] { rowsum_kernel<<<(rows + 7) / 8, 256, 0, st>>>(p.R, p.s, rows, p.S, p.eps, p.M, p.prot); }) < 0) return -1;
         ++launches;
     }
     if (p.d == 128) {
@@ -400,7 +401,7 @@ int simt_conv_rowsum(int dtype, const CompressParams& p, cudaStream_t st) {
                                        : checked([&] { conv_relu_kernel<__nv_bfloat16><<<grid, 256, smem, st>>>(p); });
     if (rc < 0) return -1;
     const int rows = p.units * p.M;
-    if (checked([&] { rowsum_kernel<<<(rows + 7) / 8, 256, 0, st>>>(p.R, p.s, rows, p.S, p.eps); }) < 0) return -1;
+    if (checked([&] { rowsum_kernel<<<(rows + 7) / 8, 256, 0, st>>>(p.R, p.s, rows, p.S, p.eps, p.M, p.prot); }) < 0) return -1;
     return 2;
 }
 

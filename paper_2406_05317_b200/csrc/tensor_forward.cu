@@ -229,6 +229,7 @@ __device__ __forceinline__ void compress_body(const TcCompressParams& P, uint8_t
         {
             const uint32_t lane_addr = tmem + ((uint32_t)((warp & 3) * 32) << 16);
             float* rstore = P.R_store ? P.R_store + ((int64_t)u * p.M + slot) * p.S : nullptr;
+            const bool keep = slot < p.prot;
             for (int c0 = eg * 32; c0 < n_tile; c0 += 96) {
                 uint32_t v[32];
                 tmem_ld32(lane_addr + c0, v);
@@ -242,6 +243,7 @@ __device__ __forceinline__ void compress_body(const TcCompressParams& P, uint8_t
                         const int ja = j0 + c0 + e + x;
                         float ra = fmaxf(__uint_as_float(v[e + x]) + bias_i, 0.f);
                         float rb = fmaxf(__uint_as_float(v[e + x + 1]) + bias_i, 0.f);
+                        if (keep) { ra = ja == slot ? 1.f : 0.f; rb = ja + 1 == slot ? 1.f : 0.f; }   // unit row (Section 5.2)
                         if (ragged && ja >= p.S) ra = 0.f;
                         if (ragged && ja + 1 >= p.S) rb = 0.f;
                         const __nv_bfloat162 pr = __floats2bfloat162_rn(ra, rb);
@@ -298,7 +300,7 @@ __device__ __forceinline__ void compress_body(const TcCompressParams& P, uint8_t
         float* sums = reinterpret_cast<float*>(ring_ptr);      // [3 groups][128 rows]; the ring is idle now
         sums[eg * kSlots + rl] = ssum;
         __syncthreads();
-        const float tot = sums[rl] + sums[kSlots + rl] + sums[2 * kSlots + rl] + p.eps;
+        const float tot = slot < p.prot ? 1.f : sums[rl] + sums[kSlots + rl] + sums[2 * kSlots + rl] + p.eps;
         const float inv = 1.f / tot;
         if (eg == 0) p.s[(int64_t)u * p.M + slot] = tot;
         const uint32_t lane_addr = tmem + ((uint32_t)((warp & 3) * 32) << 16);
@@ -391,7 +393,7 @@ __device__ __forceinline__ void finalize_tile(const TcCompressParams& P, float (
     if (ty == 0) {
         float s = 0.f;
         for (int pt = 0; pt < P.parts; ++pt) s += __ldcg(P.part_s + (base + pt) * kSlots + il0 + tx);
-        s += p.eps;
+        s = i0 + tx < p.prot ? 1.f : s + p.eps;   // a protected slot's row is e_i: denominator exactly 1
         inv_s[tx] = 1.f / s;
         if (c0 == 0) p.s[(int64_t)u * p.M + i0 + tx] = s;
     }
@@ -867,7 +869,7 @@ __device__ __forceinline__ void finalize_unit(const TcCompressParams& P, uint8_t
         if (tid < kSlots) {
             float sum = 0.f;
             for (int pt = 0; pt < P.parts; ++pt) sum += __ldcg(P.part_s + (base + pt) * kSlots + tid);
-            sum += p.eps;
+            sum = sb * kSlots + tid < p.prot ? 1.f : sum + p.eps;
             inv_s[tid] = 1.f / sum;
             p.s[(int64_t)u * p.M + sb * kSlots + tid] = sum;
         }
