@@ -331,6 +331,7 @@ def run_ours(args):
                                          f"{times[0]:.1f} s, scaled by {w.heads}/{heads_sample}"}
         out["backward"] = time_backward()
         out["layer_stack"] = time_layer_stack()
+        out["generation"] = time_generation()
     print(json.dumps(out))
     if world > 1:
         dist.destroy_process_group()
@@ -422,6 +423,45 @@ def time_layer_stack(layers=32, runs=3):
     assert all(c.device_status() == api.OK for c in ctxs)
     return {"workload": f"{layers} layers x ({WORKLOAD} shapes, conv weights shared by the heads of a layer, c_in = 2d), 4096-token prefill",
             "ms": ms, "ms_per_layer": ms / layers, "tokens_per_s_all_layers": w.batch * w.L / (ms * 1e-3)}
+
+
+def time_generation(batches=(1, 16), steps=256, runs=3):
+    """Secondary figure: the generation stage (Section 3.3: chunks of one token on a full cache, every step
+    recomputes all M slots from S = M + 1 entries), cfg2's layer shape with the weights shared by the heads,
+    `steps` token steps per call after the cache has been filled."""
+    import torch
+
+    from paper_2406_05317_b200 import api, workloads as wl
+    base = wl.CONFIGS[WORKLOAD]
+    res = []
+    for batch in batches:
+        w = base.slice(batch=batch, B=1, L=base.M + steps)
+        g = torch.Generator(device="cuda").manual_seed(7100 + batch)
+        shape = (w.batch, w.heads, w.L, w.d)
+        Q, K, V = ((torch.randn(shape, device="cuda", generator=g) * w.qkv_scale).to(torch.bfloat16) for _ in range(3))
+        O = torch.empty_like(Q)
+        ctx = api.Lococo(w.batch, w.heads, w.d, w.M, w.k, 1, dtype=torch.bfloat16, c_in=w.c_in, weights_per_head=False)
+        ctx.set_weights((torch.randn((1, w.M, w.c_in, w.k), device="cuda", generator=g) * w.g_std).to(torch.bfloat16))
+        Kc = torch.zeros(w.batch, w.heads, w.M, w.d, dtype=torch.bfloat16, device="cuda")
+        Vc = torch.zeros_like(Kc)
+        side = torch.cuda.Stream()
+        torch.cuda.synchronize()
+        ms = 0.0
+        with torch.cuda.stream(side):
+            M = w.M
+            c = ctx.process_sequence(Q[:, :, :M], K[:, :, :M], V[:, :, :M], 1, O[:, :, :M], Kc, Vc, 0)   # fill steps
+            for it in range(2 + runs):
+                a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                a.record()
+                ctx.process_sequence(Q[:, :, M:], K[:, :, M:], V[:, :, M:], 1, O[:, :, M:], Kc, Vc, c)
+                b.record()
+                b.synchronize()
+                if it >= 2:
+                    ms += a.elapsed_time(b) / runs
+        assert ctx.device_status() == api.OK
+        res.append({"batch": batch, "us_per_token_step": ms / steps * 1e3, "tokens_per_s": batch * steps / (ms * 1e-3)})
+    return {"workload": f"chunks of one token on a full cache, {base.heads} heads, d={base.d}, M={base.M}, k={base.k}, "
+                        f"shared conv weights, {steps} token steps per call", "runs": res}
 
 
 def main():
