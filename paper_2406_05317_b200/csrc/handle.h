@@ -37,6 +37,7 @@ struct lococo_handle {
     size_t off_status = 0, off_gpack = 0, off_bias = 0, off_s = 0, off_UK = 0, off_UV = 0, off_R = 0;
     size_t off_gimage = 0, off_part = 0, off_steps = 0, off_sync = 0;  // tensor-core path
     size_t off_alt_k = 0, off_alt_v = 0;   // second cache (the chunk loop alternates between the caller's and this one)
+    size_t off_merge = 0;                  // per (unit, slot block): partial sets stored in the current step
     // persistent chunk loop: step descriptors staged in pinned host memory (a small ring, one slot per call)
     static constexpr int kSeqSlots = 4;
     unsigned char* seq_host = nullptr;

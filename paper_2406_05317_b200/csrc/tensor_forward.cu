@@ -59,6 +59,9 @@ struct TcCompressParams {
                                   // normalises and writes the cache rows itself, no partials, no finalize pass
     float* R_store;               // optional [units][M][S]
     int* status;
+    int merge;                    // 1 (parts > 1, output cache != input cache): the CTA that stores the last partial set of a
+                                  // (unit, slot block) sums the sets and writes the cache rows itself, no finalize pass
+    int* merge_count;             // [units][slot blocks] partial sets stored so far; the last CTA puts the zero back
     int n_tile, tiles, parts, tiles_per_part, halves, stages, rows_pad, slot_blocks;
 };
 
@@ -82,12 +85,64 @@ __global__ void pack_image_kernel(const __nv_bfloat16* __restrict__ G, __nv_bflo
     }
 }
 
+// cache rows of slot block sb of unit u = (sum of the partial blends) / (sum of the partial row sums + eps), by ONE CTA
+// of 384 threads: the arithmetic of finalize_tile, term for term. The threads are laid out as in the compress
+// epilogues: a thread owns one slot (a warp 32 consecutive slots) and takes the eight (matrix, 32-channel chunk)
+// pieces in turn with the two other warp groups. The partial sets are channel-major, so the warp's loads of one
+// channel are 128 contiguous bytes; all loads of a piece (32 channels x parts) are in flight at once, around L1
+// (other SMs wrote the sets moments ago). The thread then holds 32 consecutive channels of its slot: 64 bytes of the
+// slot-major cache row.
+__device__ __forceinline__ void merge_partials(const TcCompressParams& P, int sb, int u) {
+    const CompressParams& p = P.base;
+    const int n = u / p.heads, h = u % p.heads;
+    const int warp = threadIdx.x >> 5;
+    const int eg = warp >> 2, rl = (warp & 3) * 32 + (threadIdx.x & 31);
+    const int slot = sb * kSlots + rl;
+    const int64_t base = ((int64_t)u * P.slot_blocks + sb) * P.part_stride;
+    float tot = 0.f;
+    for (int pt = 0; pt < P.parts; ++pt) tot += __ldcg(P.part_s + (base + pt) * kSlots + rl);
+    tot = slot < p.prot ? 1.f : tot + p.eps;   // a protected slot's row is e_i: denominator exactly 1
+    const float inv = 1.f / tot;
+    if (eg == 0) p.s[(int64_t)u * p.M + slot] = tot;
+#pragma unroll 1
+    for (int piece = eg; piece < 2 * (kD / 32); piece += 3) {
+        const int mat = piece & 1, c0 = (piece >> 1) * 32;
+        float acc[32];
+#pragma unroll
+        for (int e = 0; e < 32; ++e) acc[e] = 0.f;
+        const float* src = P.part_U + (base * 2 + mat) * (int64_t)(kSlots * kD) + c0 * kSlots + rl;
+        for (int pt0 = 0; pt0 < P.parts; pt0 += 3) {
+            float v[3][32];
+#pragma unroll
+            for (int q = 0; q < 3; ++q)
+#pragma unroll
+                for (int e = 0; e < 32; ++e)
+                    v[q][e] = pt0 + q < P.parts ? __ldcg(src + (int64_t)(pt0 + q) * (2 * kSlots * kD) + e * kSlots) : 0.f;
+#pragma unroll
+            for (int q = 0; q < 3; ++q)
+                if (pt0 + q < P.parts) {
+#pragma unroll
+                    for (int e = 0; e < 32; ++e) acc[e] += v[q][e];
+                }
+        }
+        const View& out = mat ? p.v_out : p.k_out;
+        __nv_bfloat16* orow = unit_base_mut<__nv_bfloat16>(out, n, h) + (int64_t)slot * out.st + c0;
+#pragma unroll
+        for (int e = 0; e < 32; e += 8)
+            *reinterpret_cast<uint4*>(orow + e) =
+                make_uint4(pack_bf16(acc[e] * inv, acc[e + 1] * inv), pack_bf16(acc[e + 2] * inv, acc[e + 3] * inv),
+                           pack_bf16(acc[e + 4] * inv, acc[e + 5] * inv), pack_bf16(acc[e + 6] * inv, acc[e + 7] * inv));
+    }
+}
+
 // Work of one CTA of exactly 384 threads: tiles [part*tiles_per_part, ...) of slot block sb of unit u.
 // Thread 128 issues the MMAs, thread 160 feeds the weight ring, every thread stages rows, and all
 // twelve warps share the two epilogues: warp w owns accumulator rows (TMEM lanes) 32*(w%4)..+31
 // and every third 32-column chunk, starting with chunk w/4.
 // `tmem`: base of 512 TMEM columns the CTA owns. `cache_cg`: read cache rows around L1 (set when the
 // cache was rewritten by other SMs earlier in the SAME kernel; L1 is coherent only across launches).
+// kMerge: whether the kernel is one that may be asked to merge the partial sets itself (P.merge).
+template <bool kMerge>
 __device__ __forceinline__ void compress_body(const TcCompressParams& P, uint8_t* smem, uint32_t tmem, bool cache_cg, int part,
                                               int sb, int u) {
     const CompressParams& p = P.base;
@@ -343,6 +398,25 @@ __device__ __forceinline__ void compress_body(const TcCompressParams& P, uint8_t
         }
         __syncthreads();
         if (tid < kSlots) P.part_s[pidx * kSlots + tid] = sums[tid] + sums[kSlots + tid] + sums[2 * kSlots + tid];
+        if (kMerge && P.merge) {
+            // count this partial set in; whoever stores the last one of the (unit, slot block) builds the cache rows
+            __threadfence();
+            __syncthreads();
+            volatile int* is_last = reinterpret_cast<volatile int*>(ring_ptr + 4096);
+            if (tid == 0) {
+                int* cnt = P.merge_count + (int64_t)u * P.slot_blocks + sb;
+                const int last = atomicAdd(cnt, 1) == P.parts - 1;
+                if (last) *cnt = 0;          // nobody touches the counter again before the next step
+                *is_last = last;
+            }
+            __syncthreads();
+            const bool last = *is_last != 0;
+            __syncthreads();                 // the flag's place is reused
+            if (last) {
+                __threadfence();
+                merge_partials(P, sb, u);
+            }
+        }
     }
     tc_fence_before();
     __syncthreads();
@@ -372,7 +446,7 @@ __global__ void __launch_bounds__(kThreads, 1) compress_tc_kernel(const __grid_c
     extern __shared__ __align__(128) uint8_t smem[];
     __shared__ uint32_t tmem_slot;
     const uint32_t tmem = cta_tmem_acquire(&tmem_slot);
-    compress_body(P, smem, tmem, false, blockIdx.x, blockIdx.y, blockIdx.z);
+    compress_body<false>(P, smem, tmem, false, blockIdx.x, blockIdx.y, blockIdx.z);
     cta_tmem_release(tmem);
 }
 
@@ -807,7 +881,7 @@ __device__ __forceinline__ void step_item(const TcStepParams& P, uint8_t* smem, 
     } else if (idx < P.n_attn_first + n_comp) {
         idx -= P.n_attn_first;
         const int u = idx / P.comp_per_unit, rem = idx % P.comp_per_unit;
-        compress_body(P.comp, smem, tmem, cache_cg, rem % P.comp.parts, rem / P.comp.parts, u);
+        compress_body<true>(P.comp, smem, tmem, cache_cg, rem % P.comp.parts, rem / P.comp.parts, u);
     } else {
         idx -= n_comp;
         attention_body(P.attn, P.attn.maps, false, smem, tmem, P.qtiles - 1 - idx / units, idx % units);
@@ -971,7 +1045,7 @@ __global__ void __launch_bounds__(kAttnThreads, 1) sequence_tc_kernel(const __gr
         }
         // within a unit: compress CTAs first (the longest), then the attention tiles, longest first
         // (cache rows rewritten by other SMs earlier in this same kernel are read around L1)
-        if (r < P.comp_per_unit) compress_body(P.comp, smem, tmem, n > 0, r % P.comp.parts, r / P.comp.parts, u);
+        if (r < P.comp_per_unit) compress_body<false>(P.comp, smem, tmem, n > 0, r % P.comp.parts, r / P.comp.parts, u);
         else attention_body(P.attn, Q.steps[n].attn.maps, true, smem, tmem, P.qtiles - 1 - (r - P.comp_per_unit), u);
         __syncthreads();
         if (threadIdx.x == 0) {
@@ -1072,6 +1146,8 @@ void tensor_layout_workspace(lococo_handle* h, size_t* off) {
     *off = align(*off + (size_t)h->units * c.M * kD * 2);
     h->off_alt_v = *off;
     *off = align(*off + (size_t)h->units * c.M * kD * 2);
+    h->off_merge = *off;
+    *off = align(*off + (size_t)h->units * SB * sizeof(int));   // partial sets stored per (unit, slot block)
 }
 
 int tensor_pack_weights(lococo_handle* h, const void* G, cudaStream_t st) {
@@ -1104,6 +1180,7 @@ static bool build_compress_params(lococo_handle* h, const CompressParams& p, boo
     P.part_s = P.part_U + (size_t)p.units * SB * max_parts * 2 * kSlots * kD;
     P.R_store = p.W_out ? p.R : nullptr;
     P.status = reinterpret_cast<int*>(h->ws + h->off_status);
+    P.merge_count = reinterpret_cast<int*>(h->ws + h->off_merge);
     P.n_tile = pl.n_tile; P.tiles = pl.tiles; P.parts = pl.parts; P.tiles_per_part = pl.tiles_per_part;
     P.part_stride = fused ? max_parts : pl.parts;   // fixed regions where steps with different plans share a launch
     P.halves = p.c_in / 128; P.stages = pl.stages; P.rows_pad = pl.rows_pad; P.slot_blocks = SB;
@@ -1251,7 +1328,10 @@ int tensor_chunk_step(lococo_handle* h, const AttnParams& a, const CompressParam
         attr_set = true;
     }
     // one CTA per (unit, slot block) and an output cache that is not the input: no partials, no finalize pass
-    P.comp.direct = P.comp.parts == 1 && p.W_out == nullptr && p.k_out.ptr != p.xk.cache.ptr && p.v_out.ptr != p.xv.cache.ptr;
+    const bool own_output = p.W_out == nullptr && p.k_out.ptr != p.xk.cache.ptr && p.v_out.ptr != p.xv.cache.ptr;
+    P.comp.direct = own_output && P.comp.parts == 1;
+    // several CTAs per (unit, slot block): the one that stores the last partial set sums them and writes the rows
+    P.comp.merge = own_output && P.comp.parts > 1 && p.R16 == nullptr;
     const int blocks = P.n_attn + a.units * P.comp_per_unit;
     prof_begin(p.prof, 2, st);
     // the step's CTAs read the chunk before they wait for earlier kernels: the first step of a call is therefore
@@ -1261,7 +1341,7 @@ int tensor_chunk_step(lococo_handle* h, const AttnParams& a, const CompressParam
     if (!ok) cudaGetLastError();
     prof_end(p.prof, st);
     if (!ok) return -1;
-    if (P.comp.direct) return 1;
+    if (P.comp.direct || P.comp.merge) return 1;
     const int r = finish_compress(P.comp, st);
     return r < 0 ? -1 : 1 + r;
 }
@@ -1270,7 +1350,7 @@ int tensor_chunk_step(lococo_handle* h, const AttnParams& a, const CompressParam
 // (given an output cache that is not the input).
 bool tensor_step_direct(lococo_handle* h, const CompressParams& p) {
     Plan pl;
-    return h->use_tensor && p.W_out == nullptr && make_plan(p.S, p.k, p.c_in / 128, p.units, p.M / kSlots, true, &pl) && pl.parts == 1;
+    return h->use_tensor && p.W_out == nullptr && p.R16 == nullptr && make_plan(p.S, p.k, p.c_in / 128, p.units, p.M / kSlots, true, &pl);
 }
 
 // ---- persistent chunk loop
