@@ -376,7 +376,7 @@ lococo_status run_chunk_loop(lococo_handle* h, lococo_tensor Q, lococo_tensor K,
     // the per-(unit, slot block) counts of stored partial sets start every call at zero (a step leaves them at
     // zero, but a call that gave up on a device error may not have)
     if (h->use_tensor &&
-        cudaMemsetAsync(h->ws + h->off_merge, 0, (size_t)h->units * (cfg.M / 128) * sizeof(int), st) != cudaSuccess)
+        cudaMemsetAsync(h->ws + h->off_merge, 0, (size_t)h->units * (cfg.M / 128) * 2 * sizeof(int), st) != cudaSuccess)
         return LOCOCO_ERR_CUDA;
     const int n_chunks = (L + B - 1) / B;
     const size_t snap_step = (size_t)h->units * cfg.M * cfg.head_dim * e;

@@ -61,7 +61,7 @@ struct TcCompressParams {
     int* status;
     int merge;                    // 1 (parts > 1, output cache != input cache): the CTA that stores the last partial set of a
                                   // (unit, slot block) sums the sets and writes the cache rows itself, no finalize pass
-    int* merge_count;             // [units][slot blocks] partial sets stored so far; the last CTA puts the zero back
+    int* merge_count;             // [units][slot blocks][2]: CTAs arrived at their store, partial sets stored; the last CTA puts the zeros back
     int n_tile, tiles, parts, tiles_per_part, halves, stages, rows_pad, slot_blocks;
 };
 
@@ -85,45 +85,66 @@ __global__ void pack_image_kernel(const __nv_bfloat16* __restrict__ G, __nv_bflo
     }
 }
 
-// cache rows of slot block sb of unit u = (sum of the partial blends) / (sum of the partial row sums + eps), by ONE CTA
-// of 384 threads: the arithmetic of finalize_tile, term for term. The threads are laid out as in the compress
-// epilogues: a thread owns one slot (a warp 32 consecutive slots) and takes the eight (matrix, 32-channel chunk)
-// pieces in turn with the two other warp groups. The partial sets are channel-major, so the warp's loads of one
-// channel are 128 contiguous bytes; all loads of a piece (32 channels x parts) are in flight at once, around L1
-// (other SMs wrote the sets moments ago). The thread then holds 32 consecutive channels of its slot: 64 bytes of the
-// slot-major cache row.
-__device__ __forceinline__ void merge_partials(const TcCompressParams& P, int sb, int u) {
+// cache rows of slot block sb of unit u = (sum of the partial blends) / (sum of the partial row sums + eps), by the CTA
+// (384 threads) that holds partial set `own` in its TMEM accumulators and its row sum in `own_s`; the other sets
+// come from the workspace. The arithmetic is finalize_tile's, term for term, the sets added in their order. The
+// threads are laid out as in the compress epilogues: a thread owns one slot (a warp 32 consecutive slots) and takes
+// the eight (matrix, 32-channel chunk) pieces in turn with the two other warp groups. The stored sets are
+// channel-major, so the warp's loads of one channel are 128 contiguous bytes; the loads of two sets (32 channels
+// each) are in flight at once, around L1 (other SMs wrote them moments ago). The thread then holds 32 consecutive
+// channels of its slot: 64 bytes of the slot-major cache row.
+__device__ __forceinline__ void merge_partials(const TcCompressParams& P, uint32_t tmem, int sb, int u, int own, float own_s) {
     const CompressParams& p = P.base;
     const int n = u / p.heads, h = u % p.heads;
     const int warp = threadIdx.x >> 5;
     const int eg = warp >> 2, rl = (warp & 3) * 32 + (threadIdx.x & 31);
     const int slot = sb * kSlots + rl;
     const int64_t base = ((int64_t)u * P.slot_blocks + sb) * P.part_stride;
+    const uint32_t lane_addr = tmem + ((uint32_t)((warp & 3) * 32) << 16);
     float tot = 0.f;
-    for (int pt = 0; pt < P.parts; ++pt) tot += __ldcg(P.part_s + (base + pt) * kSlots + rl);
+    for (int pt = 0; pt < P.parts; ++pt) tot += pt == own ? own_s : __ldcg(P.part_s + (base + pt) * kSlots + rl);
     tot = slot < p.prot ? 1.f : tot + p.eps;   // a protected slot's row is e_i: denominator exactly 1
     const float inv = 1.f / tot;
     if (eg == 0) p.s[(int64_t)u * p.M + slot] = tot;
 #pragma unroll 1
     for (int piece = eg; piece < 2 * (kD / 32); piece += 3) {
         const int mat = piece & 1, c0 = (piece >> 1) * 32;
+        uint32_t mine[32];
+        tmem_ld32(lane_addr + (mat ? kColUV : kColUK) + c0, mine);
+        const float* src = P.part_U + (base * 2 + mat) * (int64_t)(kSlots * kD) + c0 * kSlots + rl;
         float acc[32];
 #pragma unroll
         for (int e = 0; e < 32; ++e) acc[e] = 0.f;
-        const float* src = P.part_U + (base * 2 + mat) * (int64_t)(kSlots * kD) + c0 * kSlots + rl;
-        for (int pt0 = 0; pt0 < P.parts; pt0 += 3) {
-            float v[3][32];
+        bool first = true;
+        for (int pt = 0; pt < P.parts;) {
+            // the next two stored sets from pt on, then every set up to the second of them, in order
+            int i0 = pt;
+            if (i0 == own) ++i0;
+            int i1 = i0 + 1;
+            if (i1 == own) ++i1;
+            float v0[32], v1[32];
 #pragma unroll
-            for (int q = 0; q < 3; ++q)
+            for (int e = 0; e < 32; ++e) {
+                v0[e] = i0 < P.parts ? __ldcg(src + (int64_t)i0 * (2 * kSlots * kD) + e * kSlots) : 0.f;
+                v1[e] = i1 < P.parts ? __ldcg(src + (int64_t)i1 * (2 * kSlots * kD) + e * kSlots) : 0.f;
+            }
+            if (first) {
+                tmem_ld_wait();
+                first = false;
+            }
+            for (int x = pt; x <= i1 && x < P.parts; ++x) {
+                if (x == own) {
 #pragma unroll
-                for (int e = 0; e < 32; ++e)
-                    v[q][e] = pt0 + q < P.parts ? __ldcg(src + (int64_t)(pt0 + q) * (2 * kSlots * kD) + e * kSlots) : 0.f;
+                    for (int e = 0; e < 32; ++e) acc[e] += __uint_as_float(mine[e]);
+                } else if (x == i0) {
 #pragma unroll
-            for (int q = 0; q < 3; ++q)
-                if (pt0 + q < P.parts) {
+                    for (int e = 0; e < 32; ++e) acc[e] += v0[e];
+                } else {
 #pragma unroll
-                    for (int e = 0; e < 32; ++e) acc[e] += v[q][e];
+                    for (int e = 0; e < 32; ++e) acc[e] += v1[e];
                 }
+            }
+            pt = i1 + 1;
         }
         const View& out = mat ? p.v_out : p.k_out;
         __nv_bfloat16* orow = unit_base_mut<__nv_bfloat16>(out, n, h) + (int64_t)slot * out.st + c0;
@@ -384,38 +405,58 @@ __device__ __forceinline__ void compress_body(const TcCompressParams& P, uint8_t
         sums[eg * kSlots + rl] = ssum;
         const uint32_t lane_addr = tmem + ((uint32_t)((warp & 3) * 32) << 16);
         const int64_t pidx = ((int64_t)u * P.slot_blocks + sb) * P.part_stride + part;
-        // stored channel-major ([channel][slot]) so that a warp's 32 lanes write 128 contiguous bytes;
-        // the eight (matrix, 32-channel chunk) pieces go round the three groups
-#pragma unroll 1
-        for (int piece = eg; piece < 2 * (kD / 32); piece += 3) {
-            const int mat = piece & 1, c0 = (piece >> 1) * 32;
-            float* out = P.part_U + (pidx * 2 + mat) * (kSlots * kD) + rl;
-            uint32_t a[32];
-            tmem_ld32(lane_addr + (mat ? kColUV : kColUK) + c0, a);
-            tmem_ld_wait();
-#pragma unroll
-            for (int e = 0; e < 32; ++e) out[(c0 + e) * kSlots] = __uint_as_float(a[e]);
-        }
-        __syncthreads();
-        if (tid < kSlots) P.part_s[pidx * kSlots + tid] = sums[tid] + sums[kSlots + tid] + sums[2 * kSlots + tid];
+        // Where the step merges the sets itself (P.merge), the CTAs of a (unit, slot block) count in twice: on arrival
+        // here, and once their set is stored. The one that arrives last keeps its set where it is (TMEM), waits for
+        // the stored count of the others (CTAs that have arrived, so they are running and a few microseconds from
+        // done; the wait is bounded all the same), and builds the cache rows. It puts both counts back to zero.
+        int* counts = P.merge_count + 2 * ((int64_t)u * P.slot_blocks + sb);
+        volatile int* is_last = reinterpret_cast<volatile int*>(ring_ptr + 4096);
+        bool last = false;
         if (kMerge && P.merge) {
-            // count this partial set in; whoever stores the last one of the (unit, slot block) builds the cache rows
-            __threadfence();
+            if (tid == 0) *is_last = atomicAdd(counts, 1) == P.parts - 1;
             __syncthreads();
-            volatile int* is_last = reinterpret_cast<volatile int*>(ring_ptr + 4096);
-            if (tid == 0) {
-                int* cnt = P.merge_count + (int64_t)u * P.slot_blocks + sb;
-                const int last = atomicAdd(cnt, 1) == P.parts - 1;
-                if (last) *cnt = 0;          // nobody touches the counter again before the next step
-                *is_last = last;
+            last = *is_last != 0;
+        }
+        if (!last) {
+            // stored channel-major ([channel][slot]) so that a warp's 32 lanes write 128 contiguous bytes;
+            // the eight (matrix, 32-channel chunk) pieces go round the three groups
+#pragma unroll 1
+            for (int piece = eg; piece < 2 * (kD / 32); piece += 3) {
+                const int mat = piece & 1, c0 = (piece >> 1) * 32;
+                float* out = P.part_U + (pidx * 2 + mat) * (kSlots * kD) + rl;
+                uint32_t a[32];
+                tmem_ld32(lane_addr + (mat ? kColUV : kColUK) + c0, a);
+                tmem_ld_wait();
+#pragma unroll
+                for (int e = 0; e < 32; ++e) out[(c0 + e) * kSlots] = __uint_as_float(a[e]);
             }
             __syncthreads();
-            const bool last = *is_last != 0;
-            __syncthreads();                 // the flag's place is reused
-            if (last) {
+            if (tid < kSlots) P.part_s[pidx * kSlots + tid] = sums[tid] + sums[kSlots + tid] + sums[2 * kSlots + tid];
+            if (kMerge && P.merge) {
                 __threadfence();
-                merge_partials(P, sb, u);
+                __syncthreads();
+                if (tid == 0) atomicAdd(counts + 1, 1);
             }
+        } else {
+            if (tid == 0) {
+                int seen = 0;
+                const uint32_t limit = *failed ? 64u : (1u << 20);
+                for (uint32_t i = 0; i < limit; ++i) {
+                    asm volatile("ld.acquire.gpu.global.s32 %0, [%1];" : "=r"(seen) : "l"(counts + 1) : "memory");
+                    if (seen >= P.parts - 1) break;
+                    __nanosleep(32);
+                }
+                if (seen < P.parts - 1) {
+                    *failed = 1;
+                    atomicCAS(P.status, 0, 13);
+                }
+                counts[0] = 0;     // nobody touches the counts again before the next step
+                counts[1] = 0;
+            }
+            __syncthreads();
+            __threadfence();
+            const float own_s = sums[rl] + sums[kSlots + rl] + sums[2 * kSlots + rl];
+            merge_partials(P, tmem, sb, u, part, own_s);
         }
     }
     tc_fence_before();
@@ -1147,7 +1188,7 @@ void tensor_layout_workspace(lococo_handle* h, size_t* off) {
     h->off_alt_v = *off;
     *off = align(*off + (size_t)h->units * c.M * kD * 2);
     h->off_merge = *off;
-    *off = align(*off + (size_t)h->units * SB * sizeof(int));   // partial sets stored per (unit, slot block)
+    *off = align(*off + (size_t)h->units * SB * 2 * sizeof(int));   // per (unit, slot block): CTAs arrived, partial sets stored
 }
 
 int tensor_pack_weights(lococo_handle* h, const void* G, cudaStream_t st) {
