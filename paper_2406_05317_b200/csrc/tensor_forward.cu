@@ -821,9 +821,22 @@ __device__ __forceinline__ void attention_body(const TcAttnParams& P, const CUte
                 }
                 return sum;
             };
+            // the first tile has no reference maximum yet, so its first pass only looks for one
+            auto max_only = [&](float& tmax) {
+#pragma unroll
+                for (int c0 = 0; c0 < 64; c0 += 32) {
+                    uint32_t v[32];
+                    tmem_ld32(s_addr + c0, v);
+                    tmem_ld_wait();
+#pragma unroll
+                    for (int e = 0; e < 32; ++e)
+                        if (!need_mask || j0 + c0 + e < vis) tmax = fmaxf(tmax, __uint_as_float(v[e]));
+                }
+            };
             for (int attempt = 0; attempt < 2; ++attempt) {
                 float tmax = -INFINITY;
-                lsum = need_mask ? sweep(std::true_type{}, tmax) : sweep(std::false_type{}, tmax);
+                if (jt == 0 && attempt == 0) max_only(tmax);
+                else lsum = need_mask ? sweep(std::true_type{}, tmax) : sweep(std::false_type{}, tmax);
                 if (attempt == 1) break;
                 const __nv_bfloat16 mine = __float2bfloat16_rn(tmax * sc2);
                 xmax[b * 256 + half * 128 + rl] = mine;
