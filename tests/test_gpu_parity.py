@@ -343,3 +343,37 @@ def test_persistent_loop_equals_stepwise_launches(api):
     assert res[0][3] == res[1][3] == w.M
     assert torch.equal(res[0][0], res[1][0]) and torch.equal(res[0][1], res[1][1]) and torch.equal(res[0][2], res[1][2])
     assert res[0][4] < res[1][4]        # one persistent launch instead of two per step
+
+
+@pytest.mark.parametrize("heads,L", [(32, 1536), (4, 2048)])
+def test_merged_cache_update_has_the_bits_of_the_persistent_kernel(api, heads, L):
+    # With several compress CTAs per (unit, slot block) the chunk loop lets the last of them sum the partial
+    # blends and write the cache rows (one launch per chunk). The persistent kernel cuts the positions into the
+    # same tiles and rebuilds the cache from the same partial sets in its own way: the two must agree bit for bit.
+    # (The stand-alone entry points plan their tiles for a launch of their own, so their sums are ordered differently.)
+    w = wl.CONFIGS["cfg2"].slice(heads=heads, L=L)
+    Q, K, V = (to_device(x, w.dtype) for x in wl.make_qkv(w))
+    n_chunks = L // w.B
+
+    def fresh():
+        O = torch.empty_like(Q)
+        Kc = torch.zeros(w.batch, w.heads, w.M, w.d, dtype=Q.dtype, device="cuda")
+        return O, Kc, torch.zeros_like(Kc)
+
+    # the chunk loop (merge inside the step kernel)
+    ctx, _, _ = make_ctx(api, w, path=api.PATH_TENSOR)
+    O1, Kc1, Vc1 = fresh()
+    before = ctx.launch_count()
+    c1 = ctx.process_sequence(Q, K, V, w.B, O1, Kc1, Vc1, 0)
+    torch.cuda.synchronize()
+    assert ctx.device_status() == api.OK and c1 == w.M
+    # one launch per chunk, plus the copy back from the second cache after an odd number of steps
+    assert ctx.launch_count() - before == n_chunks + (n_chunks % 2)
+
+    # the persistent kernel
+    ctx3, _, _ = make_ctx(api, w, path=api.PATH_TENSOR_PERSISTENT)
+    O3, Kc3, Vc3 = fresh()
+    ctx3.process_sequence(Q, K, V, w.B, O3, Kc3, Vc3, 0)
+    torch.cuda.synchronize()
+    assert ctx3.device_status() == api.OK
+    assert torch.equal(O1, O3) and torch.equal(Kc1, Kc3) and torch.equal(Vc1, Vc3)
