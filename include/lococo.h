@@ -233,7 +233,9 @@ lococo_status lococo_process_sequence_backward(lococo_handle* handle, lococo_ten
                                                float* dbias, void* scratch, size_t scratch_bytes, void* stream);
 
 /* Synchronises `stream` and reads the device status word: LOCOCO_OK, or
- * LOCOCO_ERR_TIMEOUT if a bounded wait inside a kernel gave up (results invalid). */
+ * LOCOCO_ERR_TIMEOUT if a bounded wait inside a kernel gave up (results invalid).  The word
+ * stays set, and the workspace's internal counters may be left mid-step, until the workspace
+ * is handed over again with lococo_set_workspace (followed by lococo_set_weights). */
 lococo_status lococo_get_last_device_status(lococo_handle* handle, int32_t* out, void* stream);
 
 /* Number of kernels this handle has launched so far (host-side counter). */

@@ -285,6 +285,12 @@ lococo_status lococo_set_workspace(lococo_handle* h, void* ptr, size_t bytes, vo
     h->weights_set = false;
     if (cudaMemsetAsync(h->ws + h->off_status, 0, 256, static_cast<cudaStream_t>(stream)) != cudaSuccess)
         return LOCOCO_ERR_CUDA;
+    // The counts of the in-kernel merge (arrived CTAs, stored partial sets per unit and slot block) start at zero and
+    // every step puts them back to zero. Only a kernel that gave up on an expired wait can leave them otherwise; the
+    // status word then stays set as well, and both are cleared by handing the workspace over again.
+    if (h->use_tensor && cudaMemsetAsync(h->ws + h->off_merge, 0, (size_t)h->units * (h->cfg.M / 128) * 2 * sizeof(int),
+                                         static_cast<cudaStream_t>(stream)) != cudaSuccess)
+        return LOCOCO_ERR_CUDA;
     return LOCOCO_OK;
 }
 
@@ -373,11 +379,6 @@ lococo_status run_chunk_loop(lococo_handle* h, lococo_tensor Q, lococo_tensor K,
     int c = *c_inout;
     h->seq_count = 0;   // nothing is left queued from a call that failed half-way
     h->chain_open = false;
-    // the per-(unit, slot block) counts of stored partial sets start every call at zero (a step leaves them at
-    // zero, but a call that gave up on a device error may not have)
-    if (h->use_tensor &&
-        cudaMemsetAsync(h->ws + h->off_merge, 0, (size_t)h->units * (cfg.M / 128) * 2 * sizeof(int), st) != cudaSuccess)
-        return LOCOCO_ERR_CUDA;
     const int n_chunks = (L + B - 1) / B;
     const size_t snap_step = (size_t)h->units * cfg.M * cfg.head_dim * e;
     const size_t snap_all = align_up((size_t)n_chunks * snap_step, 256);
