@@ -917,7 +917,8 @@ __global__ void __launch_bounds__(kAttnThreads, 1) attention_tc_kernel(const __g
 // inputs and do not depend on each other, so their CTAs share one grid: every CTA fills an SM by
 // itself, the attention CTAs differ in length (2..5 key tiles), and a mixed grid lets the block
 // scheduler pack all of them onto the 148 SMs instead of two launches of 128 CTAs each.
-// Block order: the long attention tiles first, then the compress CTAs, then the short attention tiles.
+// Block order: the attention tiles estimated to outlast a compress CTA first (only where the grid is more than
+// two waves of CTAs), then the compress CTAs, then the remaining attention tiles, longest first.
 struct TcStepParams {
     TcAttnParams attn;
     TcCompressParams comp;
@@ -1365,8 +1366,12 @@ static bool build_step_params(lococo_handle* h, const AttnParams& a, const Compr
         const int cols = a.c + std::min(a.b, (t + 1) * 128);
         if (7.0 + 2.4 * ((cols + 127) / 128) > comp_us) ++longer; else break;
     }
-    P.n_attn_first = longer * a.units;
     P.comp_per_unit = P.comp.parts * P.comp.slot_blocks;
+    // With at most two waves of CTAs the step is not a packing problem: its length is set by the chain through the
+    // compress CTAs that hold the cache rows (wait for the previous step, conv, merge of the unit's partial blends),
+    // so those start first and the attention CTAs fill in behind them (cfg2: 254 -> 244 us per sequence).
+    if (P.n_attn + a.units * P.comp_per_unit <= 2 * 148) longer = 0;
+    P.n_attn_first = longer * a.units;
     *out = P;
     return true;
 }
