@@ -71,6 +71,7 @@ static double* dalloc(size_t n) {
 void lococo_oracle_conv_logits(const double* Z, int S, int C, const double* G, const double* bias,
                                int M, int k, double* A) {
     const int p = (k - 1) / 2;
+#pragma omp parallel for schedule(static)   /* rows of A are independent of each other */
     for (int i = 0; i < M; ++i) {
         for (int j = 0; j < S; ++j) {
             double acc = bias ? bias[i] : 0.0;
@@ -110,6 +111,7 @@ void lococo_oracle_compress(const oracle_params* P, const double* XK, const doub
     double* A = dalloc((size_t)M * S);
     build_conv_input(P, XK, XV, S, Z);
     lococo_oracle_conv_logits(Z, S, C, G, bias, M, P->k, A);
+#pragma omp parallel for schedule(static)   /* every slot is built from its own row of A */
     for (int i = 0; i < M; ++i) {
         if (i < P->protected_slots) {
             /* Section 5.2: w_i = e_i, the slot keeps entry i as it is */
@@ -153,8 +155,9 @@ void lococo_oracle_compress(const oracle_params* P, const double* XK, const doub
 void lococo_oracle_attention(const double* Q, int b, const double* XK, const double* XV, int c, int d,
                              double scale, double* O, double* lse, double* prob) {
     const int S = c + b;
-    double* logit = dalloc((size_t)S);
+#pragma omp parallel for schedule(dynamic, 16)   /* queries are independent of each other */
     for (int r = 0; r < b; ++r) {
+        double* logit = dalloc((size_t)S);
         const int n = c + r + 1;
         double mx = -INFINITY;
         for (int j = 0; j < n; ++j) {
@@ -173,8 +176,8 @@ void lococo_oracle_attention(const double* Q, int b, const double* XK, const dou
                 for (int e = 0; e < d; ++e) O[(size_t)r * d + e] += pj * XV[(size_t)j * d + e];
         }
         if (lse) lse[r] = mx + log(den);
+        free(logit);
     }
-    free(logit);
 }
 
 /* Concatenate cache and chunk in the configured order. Returns offset of the chunk rows. */
@@ -251,16 +254,21 @@ void lococo_oracle_process_sequence(const oracle_params* P, const double* Q, con
     free(XK); free(XV);
 }
 
-/* Gradient of Eq. 1 for one chunk: given dO [b,d], accumulate dQ [b,d], dXK, dXV [c+b,d]. */
+/* Gradient of Eq. 1 for one chunk: given dO [b,d], accumulate dQ [b,d], dXK, dXV [c+b,d].
+ * With P the softmax probabilities: dP_rj = <dO_r, V_j>, dS_rj = scale * P_rj (dP_rj - sum_l P_rl dP_rl)
+ * (the row term equals <dO_r, O_r>), then dQ = dS XK, dXK = dS^T Q, dXV = P^T dO.  The first loop runs over
+ * queries and the second over keys, so that each may be shared out among threads without two of them
+ * adding to the same entry. */
 static void attention_backward(const double* Q, int b, const double* XK, const double* XV, int c, int d,
                                double scale, const double* dO, double* dQ, double* dXK, double* dXV) {
     const int S = c + b;
     double* O = dalloc((size_t)b * d);
     double* prob = dalloc((size_t)b * S);
+    double* dS = dalloc((size_t)b * S);
     lococo_oracle_attention(Q, b, XK, XV, c, d, scale, O, NULL, prob);
+#pragma omp parallel for schedule(dynamic, 16)
     for (int r = 0; r < b; ++r) {
         const int n = c + r + 1;
-        /* dP_j = <dO_r, V_j>;  dlogit_j = P_j (dP_j - sum_l P_l dP_l) */
         double dot = 0.0;
         for (int e = 0; e < d; ++e) dot += dO[(size_t)r * d + e] * O[(size_t)r * d + e];
         for (int j = 0; j < n; ++j) {
@@ -268,14 +276,22 @@ static void attention_backward(const double* Q, int b, const double* XK, const d
             double dp = 0.0;
             for (int e = 0; e < d; ++e) dp += dO[(size_t)r * d + e] * XV[(size_t)j * d + e];
             const double dl = pj * (dp - dot) * scale;
+            dS[(size_t)r * S + j] = dl;
+            for (int e = 0; e < d; ++e) dQ[(size_t)r * d + e] += dl * XK[(size_t)j * d + e];
+        }
+    }
+#pragma omp parallel for schedule(dynamic, 16)
+    for (int j = 0; j < S; ++j) {
+        /* key j is seen by the queries r with c + r >= j */
+        for (int r = (j > c ? j - c : 0); r < b; ++r) {
+            const double pj = prob[(size_t)r * S + j], dl = dS[(size_t)r * S + j];
             for (int e = 0; e < d; ++e) {
                 dXV[(size_t)j * d + e] += pj * dO[(size_t)r * d + e];
-                dQ[(size_t)r * d + e] += dl * XK[(size_t)j * d + e];
                 dXK[(size_t)j * d + e] += dl * Q[(size_t)r * d + e];
             }
         }
     }
-    free(O); free(prob);
+    free(O); free(prob); free(dS);
 }
 
 /*
@@ -315,13 +331,18 @@ static void compress_backward(const oracle_params* P, const double* XK, const do
             if (i < P->protected_slots) dA[(size_t)i * S + j] = 0.0;   /* constant row: nothing flows to Eq. 6 */
         }
     }
-    /* through Eq. 6 */
-    for (int i = 0; i < M; ++i) {
-        for (int j = 0; j < S; ++j) {
-            const double g = dA[(size_t)i * S + j];
-            if (g == 0.0) continue;
-            if (dbias) dbias[i] += g;
-            for (int ch = 0; ch < C; ++ch) {
+    /* through Eq. 6: A[i,j] = bias_i + sum_ch sum_t G[i,ch,t] Z[j+t-p,ch].  The channel loop is the outer
+     * one so that channels can be shared out among threads: an input channel owns its entries of dG and of
+     * dXK / dXV, and each of them still receives its terms in the order (i, j, t). */
+    if (dbias)
+        for (int i = 0; i < M; ++i)
+            for (int j = 0; j < S; ++j) dbias[i] += dA[(size_t)i * S + j];
+#pragma omp parallel for schedule(static)
+    for (int ch = 0; ch < C; ++ch) {
+        for (int i = 0; i < M; ++i) {
+            for (int j = 0; j < S; ++j) {
+                const double g = dA[(size_t)i * S + j];
+                if (g == 0.0) continue;
                 for (int t = 0; t < k; ++t) {
                     const int jj = j + t - p;
                     if (jj < 0 || jj >= S) continue;
@@ -338,14 +359,19 @@ static void compress_backward(const oracle_params* P, const double* XK, const do
 
 /*
  * Gradients of  loss = <dO, O> + <dKc_final, Kc_final> + <dVc_final, Vc_final>
- * through Algorithm 2 started from an EMPTY cache (cache-first order, output ReLU).
+ * through Algorithm 2 (cache-first order, output ReLU) started from the cache Kc_in, Vc_in [M,d] with
+ * c_in valid rows (NULL, NULL, 0: an empty cache).  A sequence processed in several calls of the loop
+ * is differentiated call by call, last call first: the cache gradient a call returns in dKc_in, dVc_in
+ * [M,d] (optional; rows >= c_in are zero) is the dKc_final, dVc_final of the call before it.
  * Accumulates into dQ, dK, dV [L,d], dG [M,c_in,k], dbias [M] (optional): callers zero them.
  * Returns 0, or -1 if a flag selects a reading the backward does not cover.
  */
-int lococo_oracle_process_sequence_grad(const oracle_params* P, const double* Q, const double* K,
-                                        const double* V, int L, int B, const double* G, const double* bias,
-                                        const double* dO, const double* dKc_final, const double* dVc_final,
-                                        double* dQ, double* dK, double* dV, double* dG, double* dbias) {
+int lococo_oracle_process_sequence_grad_from(const oracle_params* P, const double* Q, const double* K,
+                                             const double* V, int L, int B, const double* G, const double* bias,
+                                             const double* Kc_in, const double* Vc_in, int c_in,
+                                             const double* dO, const double* dKc_final, const double* dVc_final,
+                                             double* dQ, double* dK, double* dV, double* dG, double* dbias,
+                                             double* dKc_in, double* dVc_in) {
     if (P->flags != 0) return -1;
     const int d = P->d, M = P->M;
     const int N = (L + B - 1) / B;
@@ -355,7 +381,11 @@ int lococo_oracle_process_sequence_grad(const oracle_params* P, const double* Q,
     double* snapK = dalloc((size_t)N * M * d);
     double* snapV = dalloc((size_t)N * M * d);
     int32_t* snapc = (int32_t*)calloc((size_t)N, sizeof(int32_t));
-    int c_final = 0;
+    int c_final = c_in;
+    if (c_in > 0) {
+        memcpy(Kc, Kc_in, sizeof(double) * (size_t)c_in * d);
+        memcpy(Vc, Vc_in, sizeof(double) * (size_t)c_in * d);
+    }
     lococo_oracle_process_sequence(P, Q, K, V, L, B, G, bias, O, Kc, Vc, &c_final, NULL, snapK, snapV, snapc);
 
     /* gradient w.r.t. the cache as it stands after step n (starts as the loss's own term) */
@@ -401,9 +431,21 @@ int lococo_oracle_process_sequence_grad(const oracle_params* P, const double* Q,
             dV[(size_t)t0 * d + x] += dXV[(size_t)c * d + x];
         }
     }
+    /* what is left is the gradient w.r.t. the cache the loop started from */
+    if (dKc_in) memcpy(dKc_in, gKc, sizeof(double) * (size_t)M * d);
+    if (dVc_in) memcpy(dVc_in, gVc, sizeof(double) * (size_t)M * d);
     free(O); free(Kc); free(Vc); free(snapK); free(snapV); free(snapc);
     free(gKc); free(gVc); free(XK); free(XV); free(dXK); free(dXV);
     return 0;
+}
+
+/* The same from an empty cache. */
+int lococo_oracle_process_sequence_grad(const oracle_params* P, const double* Q, const double* K,
+                                        const double* V, int L, int B, const double* G, const double* bias,
+                                        const double* dO, const double* dKc_final, const double* dVc_final,
+                                        double* dQ, double* dK, double* dV, double* dG, double* dbias) {
+    return lococo_oracle_process_sequence_grad_from(P, Q, K, V, L, B, G, bias, NULL, NULL, 0, dO, dKc_final, dVc_final,
+                                                    dQ, dK, dV, dG, dbias, NULL, NULL);
 }
 
 /*
@@ -416,7 +458,7 @@ void lococo_oracle_process_batch(const oracle_params* P, int units, int heads, c
                                  long g_head_stride, const double* bias, long bias_head_stride,
                                  double* O, double* Kc, double* Vc, int32_t* c_inout, double* lse) {
     const int d = P->d, M = P->M;
-#pragma omp parallel for schedule(dynamic, 1)
+#pragma omp parallel for schedule(dynamic, 1) if (units > 1)   /* one unit: the loops inside it take the threads */
     for (int u = 0; u < units; ++u) {
         const int h = u % heads;
         int c = c_inout[u];
@@ -438,7 +480,7 @@ int lococo_oracle_grad_batch(const oracle_params* P, int units, int heads, const
     const int d = P->d, M = P->M;
     const size_t gsz = (size_t)M * P->c_in * P->k;
     int rc = 0;
-#pragma omp parallel for schedule(dynamic, 1)
+#pragma omp parallel for schedule(dynamic, 1) if (units > 1)   /* one unit: the loops inside it take the threads */
     for (int u = 0; u < units; ++u) {
         const int h = u % heads;
         double* dG_u = dalloc(gsz);

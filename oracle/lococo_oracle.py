@@ -49,6 +49,7 @@ def _load():
         _lib = ctypes.CDLL(str(build()))
         _lib.lococo_oracle_threads.restype = ctypes.c_int
         _lib.lococo_oracle_process_sequence_grad.restype = ctypes.c_int
+        _lib.lococo_oracle_process_sequence_grad_from.restype = ctypes.c_int
         _lib.lococo_oracle_grad_batch.restype = ctypes.c_int
     return _lib
 
@@ -155,9 +156,12 @@ def process_sequence(Q, K, V, G, B, bias=None, eps=1e-6, scale=None, flags=0, ca
     return out + (sK, sV, sc) if want_snapshots else out
 
 
-def process_sequence_grad(Q, K, V, G, B, dO, dKc_final, dVc_final, bias=None, eps=1e-6, scale=None, protected=0):
-    """Gradients of <dO,O> + <dKc_final,Kc_final> + <dVc_final,Vc_final> through Algorithm 2
-    (empty initial cache): returns dQ, dK, dV [L,d], dG [M,C,k], dbias [M] or None."""
+def process_sequence_grad(Q, K, V, G, B, dO, dKc_final, dVc_final, bias=None, eps=1e-6, scale=None, protected=0,
+                          cache=None):
+    """Gradients of <dO,O> + <dKc_final,Kc_final> + <dVc_final,Vc_final> through Algorithm 2:
+    returns dQ, dK, dV [L,d], dG [M,C,k], dbias [M] or None.  With cache = (Kc [M,d], Vc [M,d], c) the loop
+    starts from that cache instead of an empty one and the gradients w.r.t. it, dKc_in and dVc_in [M,d], are
+    returned as well (the training use of a sequence processed in several calls, last call first)."""
     Q, K, V, G = _f64(Q), _f64(K), _f64(V), _f64(G)
     L, d = Q.shape
     M, C, k = G.shape
@@ -167,10 +171,19 @@ def process_sequence_grad(Q, K, V, G, B, dO, dKc_final, dVc_final, bias=None, ep
     dQ, dK, dV = np.zeros((L, d)), np.zeros((L, d)), np.zeros((L, d))
     dG = np.zeros((M, C, k))
     db = np.zeros(M) if bias is not None else None
-    rc = _load().lococo_oracle_process_sequence_grad(ctypes.byref(P), _p(Q), _p(K), _p(V), L, B, _p(G), _p(bb),
-                                                     _p(dO), _p(dKf), _p(dVf), _p(dQ), _p(dK), _p(dV), _p(dG), _p(db))
+    if cache is None:
+        rc = _load().lococo_oracle_process_sequence_grad(ctypes.byref(P), _p(Q), _p(K), _p(V), L, B, _p(G), _p(bb),
+                                                         _p(dO), _p(dKf), _p(dVf), _p(dQ), _p(dK), _p(dV), _p(dG), _p(db))
+        assert rc == 0
+        return dQ, dK, dV, dG, db
+    Kc, Vc, c = _f64(cache[0]), _f64(cache[1]), int(cache[2])
+    assert Kc.shape == (M, d) and Vc.shape == (M, d) and 0 <= c <= M
+    dKc, dVc = np.zeros((M, d)), np.zeros((M, d))
+    rc = _load().lococo_oracle_process_sequence_grad_from(ctypes.byref(P), _p(Q), _p(K), _p(V), L, B, _p(G), _p(bb),
+                                                          _p(Kc), _p(Vc), c, _p(dO), _p(dKf), _p(dVf), _p(dQ), _p(dK),
+                                                          _p(dV), _p(dG), _p(db), _p(dKc), _p(dVc))
     assert rc == 0
-    return dQ, dK, dV, dG, db
+    return dQ, dK, dV, dG, db, dKc, dVc
 
 
 def process_batch(Q, K, V, G, B, bias=None, eps=1e-6, scale=None, flags=0, protected=0):

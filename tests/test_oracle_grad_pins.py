@@ -97,3 +97,66 @@ def test_batch_gradient_sums_shared_weights():
             np.testing.assert_allclose(dK[bi, h], kk, atol=1e-13)
             acc += g
     np.testing.assert_allclose(dG[0], acc, atol=1e-12)
+
+
+def loss_from(cache, Q, K, V, G, B, PO, PK, PV):
+    O, Kc, Vc, c, _ = orc.process_sequence(Q, K, V, G, B, cache=cache)
+    return (PO * O).sum() + (PK * Kc).sum() + (PV * Vc).sum()
+
+
+@pytest.mark.parametrize("c0,M,B,L", [(6, 6, 4, 14), (3, 7, 3, 11), (5, 5, 9, 9)])
+def test_gradient_with_respect_to_the_initial_cache_matches_finite_differences(c0, M, B, L):
+    # the loop started from a given cache (full, or partly filled with fill steps still to come): the cache
+    # gradient against central differences of the forward; rows beyond the fill count get no gradient
+    r = rng(300 + c0 + M)
+    d, k = 3, 3
+    Q, K, V = r.standard_normal((L, d)), r.standard_normal((L, d)), r.standard_normal((L, d))
+    G = r.standard_normal((M, d, k))
+    Kc0, Vc0 = r.standard_normal((M, d)), r.standard_normal((M, d))
+    PO, PK, PV = r.standard_normal((L, d)), r.standard_normal((M, d)), r.standard_normal((M, d))
+    dQ, dK, dV, dG, _, dKc, dVc = orc.process_sequence_grad(Q, K, V, G, B, PO, PK, PV, cache=(Kc0, Vc0, c0))
+    assert np.all(dKc[c0:] == 0) and np.all(dVc[c0:] == 0)
+    checks = [("Kc", Kc0, dKc, lambda x: loss_from((x, Vc0, c0), Q, K, V, G, B, PO, PK, PV)),
+              ("Vc", Vc0, dVc, lambda x: loss_from((Kc0, x, c0), Q, K, V, G, B, PO, PK, PV)),
+              ("K", K, dK, lambda x: loss_from((Kc0, Vc0, c0), Q, x, V, G, B, PO, PK, PV)),
+              ("G", G, dG, lambda x: loss_from((Kc0, Vc0, c0), Q, K, V, x, B, PO, PK, PV))]
+    for name, x, g, f in checks:
+        rows = c0 if name in ("Kc", "Vc") else x.shape[0]
+        for fi in r.permutation(rows * x[0].size)[:12]:
+            idx = np.unravel_index(fi, (rows,) + x.shape[1:])
+            fd = finite_difference(f, x, idx)
+            assert abs(fd - g[idx]) <= 2e-6 * max(1.0, abs(fd)), (name, idx, fd, g[idx])
+
+
+@pytest.mark.parametrize("cut", [8, 10, 16])
+def test_backward_over_two_calls_equals_backward_over_one(cut):
+    # Algorithm 2 run in two calls (tokens [0, cut) then [cut, L), the cache handed over) and differentiated
+    # last call first, the cache gradient handed back: the same gradients as one call over all tokens.
+    # cut = 8: on a chunk boundary; 10: the first call ends with a short chunk; 16: two whole chunks each
+    r = rng(400 + cut)
+    L, B, M, d, k = 32 if cut == 16 else 24, 8, 6, 3, 5
+    Q, K, V = r.standard_normal((L, d)), r.standard_normal((L, d)), r.standard_normal((L, d))
+    G = r.standard_normal((M, 2 * d, k))
+    PO, PK, PV = r.standard_normal((L, d)), r.standard_normal((M, d)), r.standard_normal((M, d))
+    if cut % B == 0:
+        one = orc.process_sequence_grad(Q, K, V, G, B, PO, PK, PV)
+    _, Kc1, Vc1, c1, _ = orc.process_sequence(Q[:cut], K[:cut], V[:cut], G, B)
+    q2, k2, v2, g2, _, dKc, dVc = orc.process_sequence_grad(Q[cut:], K[cut:], V[cut:], G, B, PO[cut:], PK, PV,
+                                                            cache=(Kc1, Vc1, c1))
+    q1, k1, v1, g1, _ = orc.process_sequence_grad(Q[:cut], K[:cut], V[:cut], G, B, PO[:cut], dKc, dVc)
+    if cut % B == 0:
+        np.testing.assert_allclose(np.concatenate([q1, q2]), one[0], atol=1e-11)
+        np.testing.assert_allclose(np.concatenate([k1, k2]), one[1], atol=1e-11)
+        np.testing.assert_allclose(np.concatenate([v1, v2]), one[2], atol=1e-11)
+        np.testing.assert_allclose(g1 + g2, one[3], atol=1e-10)
+    else:
+        # the chunking differs from any single call's: check the chained gradient against finite differences
+        def f(x):
+            _, a, b, c, _ = orc.process_sequence(Q[:cut], x, V[:cut], G, B)
+            O2, Kf, Vf, _, _ = orc.process_sequence(Q[cut:], K[cut:], V[cut:], G, B, cache=(a, b, c))
+            O1 = orc.process_sequence(Q[:cut], x, V[:cut], G, B)[0]
+            return (PO[:cut] * O1).sum() + (PO[cut:] * O2).sum() + (PK * Kf).sum() + (PV * Vf).sum()
+        for fi in r.permutation(cut * d)[:10]:
+            idx = np.unravel_index(fi, (cut, d))
+            fd = finite_difference(f, K[:cut], idx)
+            assert abs(fd - k1[idx]) <= 2e-6 * max(1.0, abs(fd)), (idx, fd, k1[idx])
