@@ -24,10 +24,32 @@ if str(ROOT) not in sys.path:
 METRIC = "chunk-step tokens/sec per layer (32 heads)"
 UNIT = "tokens/s"
 WORKLOAD = "cfg2"
-# dram__bytes_read.sum + dram__bytes_write.sum of one chunk_step_tc_kernel launch at this workload, from an ncu
-# capture of the committed kernel (steady-state step): 36.9 MB read + 0.5 MB written; None while the kernel is
-# newer than the last capture
-STEP_KERNEL_DRAM_BYTES = 37.4e6
+WORKLOAD_TEXT = ("cfg2: Llama-2-7B-shaped layer, 32 heads, d=128, M=128, B=512, k=21, L=4096, batch 1 per GPU, "
+                 "per-head conv weights, c_in=d")
+# The ncu summary of the dominant kernel ends with one machine-readable line: the DRAM bytes of one launch
+# (dram__bytes_read.sum + dram__bytes_write.sum) and a digest of the kernel sources at the time of the capture.
+STEP_KERNEL_PROFILE = ROOT / "profiles" / "chunk_step_tc_kernel_cfg2.md"
+STEP_KERNEL_SOURCES = ("tensor_forward.cu", "tc_common.cuh", "common.cuh")
+
+
+def kernel_sources_digest():
+    import hashlib
+    h = hashlib.sha256()
+    for name in STEP_KERNEL_SOURCES:
+        h.update((ROOT / "paper_2406_05317_b200" / "csrc" / name).read_bytes())
+    return h.hexdigest()[:16]
+
+
+def step_kernel_traffic():
+    """DRAM bytes per launch from the committed capture, or None when the kernel sources have changed since."""
+    try:
+        for line in STEP_KERNEL_PROFILE.read_text().splitlines():
+            if line.startswith("traffic_table:"):
+                t = json.loads(line[len("traffic_table:"):])
+                return float(t["dram_bytes_per_launch"]) if t["sources_sha256_16"] == kernel_sources_digest() else None
+    except Exception:
+        pass
+    return None
 
 
 # ------------------------------------------------------------------ algorithmic work
@@ -149,25 +171,22 @@ def run_reference(args):
     from paper_2406_05317_b200 import workloads as wl
     w = wl.CONFIGS[WORKLOAD]
     threads = orc.threads()
-    heads_sample = max(1, min(w.heads, threads))
-    ws = w.slice(heads=heads_sample)
-    Q, K, V = wl.make_qkv(ws)
-    G, _ = wl.make_weights(ws)
+    # a step is the whole workload (all 32 heads, all 8 chunks): a few seconds of CPU work, nothing is scaled
+    Q, K, V = wl.make_qkv(w)
+    G, _ = wl.make_weights(w)
     for _ in range(args.warmup):
-        orc.process_batch(Q, K, V, G, ws.B)
+        orc.process_batch(Q, K, V, G, w.B)
     t = time.perf_counter()
     for _ in range(args.steps):
-        orc.process_batch(Q, K, V, G, ws.B)
-    dt = (time.perf_counter() - t) / args.steps
-    layer_ms = dt * 1e3 * (w.heads / heads_sample)
+        orc.process_batch(Q, K, V, G, w.B)
+    layer_ms = (time.perf_counter() - t) / args.steps * 1e3
     value = w.batch * w.L / (layer_ms / 1e3)
-    sample = f"{heads_sample} of {w.heads} heads, all {w.n_chunks} chunks, scaled by {w.heads}/{heads_sample}"
+    sample = f"{w.heads} of {w.heads} heads, all {w.n_chunks} chunks (the whole workload), {layer_ms / 1e3:.1f} s per step"
     print(json.dumps({
         "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
         "steps": args.steps, "warmup": args.warmup, "ms_per_step": layer_ms, "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-        "config": {"workload": f"{WORKLOAD}: Llama-2-7B-shaped layer, 32 heads, d=128, M=128, B=512, k=21, L=4096, "
-                               "batch 1, per-head conv weights"},
+        "config": {"workload": WORKLOAD_TEXT},
         "cpu_baseline": {"value": value, "unit": UNIT, "cores": threads, "kind": "oracle", "sample": sample},
         "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
     }))
@@ -303,8 +322,7 @@ def run_ours(args):
         "metric": METRIC, "value": total_tokens / (total_ms * 1e-3), "unit": UNIT, "n_gpus": world,
         "steps": args.steps, "warmup": args.warmup, "ms_per_step": total_ms / args.steps,
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
-        "config": {"workload": f"{WORKLOAD}: Llama-2-7B-shaped layer, 32 heads, d=128, M=128, B=512, k=21, L=4096, "
-                               "batch 1 per GPU, per-head conv weights, c_in=d",
+        "config": {"workload": WORKLOAD_TEXT,
                    "l2": "256 MB flush between timed steps", "chunks_per_step": w.n_chunks,
                    "parallelism": f"sequences x{world} (no collective)"},
         "clocks": clocks,
@@ -316,7 +334,7 @@ def run_ours(args):
         "roofline": {"bound": "tensor", "kernel": kernel, "flops_per_launch": flops_per_launch,
                      "achieved": achieved, "peak": peaks["bf16_tflops"], "unit": "TFLOP/s",
                      "frac": (achieved / peaks["bf16_tflops"]) if achieved else None,
-                     "traffic": STEP_KERNEL_DRAM_BYTES if (step_n and not seq_n) else None,
+                     "traffic": step_kernel_traffic() if (step_n and not seq_n) else None,
                      "peak_source": peaks["source"] + " burst", "launches": dom_n,
                      "us_per_launch": dom_per_launch_ms * 1e3, "us_per_launch_isolated": isolated_per_launch_ms * 1e3,
                      "duration": "timed region / launches of this kernel (its launches overlap their neighbours)"},
@@ -329,12 +347,131 @@ def run_ours(args):
         out["cpu_baseline"] = {"value": value, "unit": UNIT, "cores": threads, "kind": "oracle",
                                "sample": f"{heads_sample} of {w.heads} heads, all {w.n_chunks} chunks, "
                                          f"{times[0]:.1f} s, scaled by {w.heads}/{heads_sample}"}
+        out["eager"] = time_eager(ctx, w, Q, K, V, flush)
+        out["configs"] = {name: time_config(name) for name in ("cfg3", "cfg4")}
         out["backward"] = time_backward()
         out["layer_stack"] = time_layer_stack()
         out["generation"] = time_generation()
+        out["sweep"] = time_sweep(full=args.sweep)
     print(json.dumps(out))
     if world > 1:
         dist.destroy_process_group()
+
+
+def time_eager(ctx, w, Q, K, V, flush, runs=10):
+    """The headline workload without the CUDA-graph replay: every call gets output and cache tensors that
+    differ from the previous call's, so the library launches the chunk loop kernel by kernel each time."""
+    import torch
+    sets = [(torch.empty_like(Q), torch.zeros(w.batch, w.heads, w.M, w.d, dtype=Q.dtype, device="cuda"),
+             torch.zeros(w.batch, w.heads, w.M, w.d, dtype=Q.dtype, device="cuda")) for _ in range(2)]
+    ms = 0.0
+    for it in range(3 + runs):
+        O, Kc, Vc = sets[it % 2]
+        flush.fill_(1)
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record()
+        ctx.process_sequence(Q, K, V, w.B, O, Kc, Vc, 0)
+        b.record()
+        b.synchronize()
+        if it >= 3:
+            ms += a.elapsed_time(b) / runs
+    return {"what": "same workload, no CUDA-graph replay (buffers change from call to call)", "ms_per_step": ms,
+            "tokens_per_s": w.batch * w.L / (ms * 1e-3)}
+
+
+def time_config(name, runs=5):
+    """Whole lococo_process_sequence at another configuration: seeded inputs of the workload recipe, resident on
+    the device, no cache snapshots, repeated identical calls on a side stream (CUDA-graph replay from the third),
+    256 MB L2 flush between calls; roofline fraction as for the headline workload."""
+    import torch
+
+    from paper_2406_05317_b200 import api, workloads as wl
+    w = wl.CONFIGS[name]
+    tdt = torch.bfloat16
+    ctx = api.Lococo(w.batch, w.heads, w.d, w.M, w.k, w.B, dtype=tdt, c_in=w.c_in, weights_per_head=w.weights_per_head)
+    G, _ = wl.make_weights(w)
+    ctx.set_weights(torch.from_numpy(G).cuda().to(tdt))
+    Q = torch.empty(w.batch, w.heads, w.L, w.d, dtype=tdt, device="cuda")
+    K, V, O = torch.empty_like(Q), torch.empty_like(Q), torch.empty_like(Q)
+    for n in range(w.batch):                       # sequence by sequence: the host never holds the whole batch
+        for dst, x in zip((Q, K, V), wl.make_sequence(w, n)):
+            dst[n].copy_(torch.from_numpy(x).to(tdt))
+    Kc = torch.zeros(w.batch, w.heads, w.M, w.d, dtype=tdt, device="cuda")
+    Vc = torch.zeros_like(Kc)
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")
+    side = torch.cuda.Stream()
+    torch.cuda.synchronize()
+    ms = 0.0
+    launches0 = 0
+    with torch.cuda.stream(side):
+        for it in range(3 + runs):
+            if it == 3:
+                launches0 = ctx.launch_count()
+            flush.fill_(1)
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record()
+            ctx.process_sequence(Q, K, V, w.B, O, Kc, Vc, 0)
+            b.record()
+            b.synchronize()
+            if it >= 3:
+                ms += a.elapsed_time(b) / runs
+    assert ctx.device_status() == api.OK
+    launches = (ctx.launch_count() - launches0) // runs
+    conv_f, blend_f, attn_f = sequence_flops(w)
+    units = w.batch * w.heads
+    flops = units * (conv_f + blend_f + attn_f)
+    sets = w.heads if w.weights_per_head else 1
+    nbytes = 4.0 * units * w.L * w.d * 2 + units * 2 * w.M * w.d * 2 + sets * w.M * w.c_in * w.k * 2
+    peaks = measured_peaks()
+    roof_ms = max(flops / (peaks["bf16_tflops"] * 1e12), nbytes / (peaks["hbm_gbs"] * 1e9)) * 1e3
+    return {"workload": f"{name}: batch {w.batch}, {w.heads} heads, d={w.d}, M={w.M}, B={w.B}, k={w.k}, L={w.L}, "
+                        f"{'per-head' if w.weights_per_head else 'shared'} conv weights, c_in=d, seeded recipe",
+            "ms_per_step": ms, "tokens_per_s": w.batch * w.L / (ms * 1e-3), "gpu_launches": launches,
+            "flops_per_step": flops, "bytes_per_step": nbytes, "achieved_tflops": flops / (ms * 1e-3) / 1e12,
+            "roofline_ms": roof_ms, "frac": roof_ms / ms, "bound": "tensor", "peak_source": peaks["source"] + " burst"}
+
+
+def time_sweep(full=False, runs=3):
+    """Kernel width and cache size (the paper's ablations over k and M, as a performance curve): one layer of 32
+    heads, chunks of 512 tokens, weights shared by the heads, 4096 tokens per call; time per chunk step and
+    TFLOP/s on algorithmic flops. Default: the corners k in {3, 21, 61} x M in {128, 512}; --sweep: the whole grid."""
+    import torch
+
+    from paper_2406_05317_b200 import api, workloads as wl
+    base = wl.CONFIGS[WORKLOAD]
+    ks = (3, 9, 21, 41, 61) if full else (3, 21, 61)
+    Ms = (128, 256, 512, 1024) if full else (128, 512)
+    g = torch.Generator(device="cuda").manual_seed(7300)
+    shape = (base.batch, base.heads, base.L, base.d)
+    Q, K, V = ((torch.randn(shape, device="cuda", generator=g) * base.qkv_scale).to(torch.bfloat16) for _ in range(3))
+    O = torch.empty_like(Q)
+    rows = []
+    side = torch.cuda.Stream()
+    for M in Ms:
+        for k in ks:
+            w = base.slice(M=M, k=k, weights_per_head=False)
+            ctx = api.Lococo(w.batch, w.heads, w.d, M, k, w.B, dtype=torch.bfloat16, c_in=w.c_in, weights_per_head=False)
+            ctx.set_weights((torch.randn((1, M, w.c_in, k), device="cuda", generator=g) * w.g_std).to(torch.bfloat16))
+            Kc = torch.zeros(w.batch, w.heads, M, w.d, dtype=torch.bfloat16, device="cuda")
+            Vc = torch.zeros_like(Kc)
+            torch.cuda.synchronize()
+            ms = 0.0
+            with torch.cuda.stream(side):
+                for it in range(3 + runs):
+                    a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                    a.record()
+                    ctx.process_sequence(Q, K, V, w.B, O, Kc, Vc, 0)
+                    b.record()
+                    b.synchronize()
+                    if it >= 3:
+                        ms += a.elapsed_time(b) / runs
+            assert ctx.device_status() == api.OK
+            conv_f, blend_f, attn_f = sequence_flops(w)
+            flops = w.batch * w.heads * (conv_f + blend_f + attn_f)
+            rows.append({"M": M, "k": k, "us_per_chunk_step": ms / w.n_chunks * 1e3,
+                         "tflops": flops / (ms * 1e-3) / 1e12})
+    return {"workload": f"{base.heads} heads, d={base.d}, B={base.B}, L={base.L}, shared conv weights, c_in=d; "
+                        "whole lococo_process_sequence divided by its chunks", "rows": rows}
 
 
 def time_backward(name="cfg5", runs=2):
@@ -348,12 +485,10 @@ def time_backward(name="cfg5", runs=2):
                      weights_per_head=w.weights_per_head)
     G, _ = wl.make_weights(w)
     ctx.set_weights(torch.from_numpy(G).cuda().to(torch.bfloat16))
-    g = torch.Generator(device="cuda").manual_seed(5000)
-    shape = (w.batch, w.heads, w.L, w.d)
-    rnd = lambda sh, s=1.0: (torch.randn(sh, device="cuda", generator=g) * s).to(torch.bfloat16)
-    Q, K, V, PO = rnd(shape, w.qkv_scale), rnd(shape, w.qkv_scale), rnd(shape, w.qkv_scale), rnd(shape)
+    dev = lambda x: torch.from_numpy(x).cuda().to(torch.bfloat16)
+    Q, K, V = (dev(x) for x in wl.make_qkv(w))                     # the seeded recipe (heavy-tailed keys)
+    PO, PK, PV = (dev(x) for x in wl.make_loss_projections(w))
     cshape = (w.batch, w.heads, w.M, w.d)
-    PK, PV = rnd(cshape), rnd(cshape)
     O, gQ, gK, gV = (torch.empty_like(Q) for _ in range(4))
     Kc, Vc = torch.zeros(cshape, dtype=torch.bfloat16, device="cuda"), torch.zeros(cshape, dtype=torch.bfloat16, device="cuda")
     gG = torch.zeros(G.shape, dtype=torch.float32, device="cuda")
@@ -470,6 +605,7 @@ def main():
     ap.add_argument("--steps", type=int, default=20)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--sweep", action="store_true", help="time the whole kernel-width x cache-size grid, not its corners")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
     if args.impl == "reference":

@@ -51,9 +51,15 @@ typedef enum { LOCOCO_F32 = 0, LOCOCO_BF16 = 1 } lococo_dtype;
 
 /* Which kernels serve a call. AUTO: tensor-core (tcgen05) kernels where the shape and
  * dtype allow, CUDA-core kernels otherwise. TENSOR_PERSISTENT: the tensor-core kernels, with
- * the compress steps of lococo_process_sequence (Algorithm 2, loop) run by ONE cooperative
- * launch whose CTAs stay resident and meet at a device-wide barrier between the steps,
- * instead of one launch per chunk; results are identical bit for bit. */
+ * all consecutive compress steps of a lococo_process_sequence call (Algorithm 2, loop) run by ONE
+ * ordinary launch of one CTA per SM instead of one launch per chunk. Its CTAs pull (step, unit,
+ * piece) work items from a single list in step order; an item of step n waits (bounded) until the
+ * step counter of ITS unit says that the cache of step n-1 is complete, and the CTA that finishes
+ * the last item of a (step, unit) pair rebuilds that unit's cache and advances the counter. There
+ * is no device-wide barrier and no need for all CTAs to be resident at once: an item only waits
+ * for items earlier in the list, which a running CTA has already taken. Results are identical bit
+ * for bit to the per-chunk launches. This path is a tested variant, not the default: the per-chunk
+ * launches, overlapped as programmatic dependents, are faster at every measured shape. */
 typedef enum {
     LOCOCO_PATH_AUTO = 0,
     LOCOCO_PATH_SIMT = 1,
@@ -149,7 +155,10 @@ lococo_status lococo_compress_step(lococo_handle* handle, lococo_tensor K_cache,
  * cfg describes the problem as for lococo_create (max_chunk, path and softmax_scale are
  * ignored); G [heads|1, M, c_in, k] and bias (or NULL) are device pointers in cfg->dtype and
  * are re-packed on every call.  The tensors are those of lococo_compress_step; the outputs may
- * alias the cache inputs.  Only a real compress step is accepted (cache_len + b > M): the fill
+ * be the cache inputs themselves (same base pointer and strides: an update in place).  As in
+ * lococo_compress_step only equal base pointers are recognised: an output that overlaps another
+ * tensor at an offset is not detected and gives undefined results.
+ * Only a real compress step is accepted (cache_len + b > M): the fill
  * branch needs no scratch, use lococo_compress_step for it.
  * Errors: LOCOCO_ERR_WORKSPACE when the scratch this problem needs, about
  *   4*batch*heads*M*(cache_len+b) + 8*batch*heads*M*d + sizeof(G) bytes,
@@ -216,21 +225,27 @@ lococo_status lococo_process_sequence_host(lococo_handle* handle, const void* Q_
 
 /*
  * Gradients of  loss = <dO, O> + <dK_cache_final, K_cache_final> + <dV_cache_final, V_cache_final>
- * through lococo_process_sequence started from an empty cache (the training use of
- * Algorithm 2; Section 3.2.1: the conv parameters are trained end to end).
- * Q, K, V, O: the forward's tensors; saved: what that forward wrote.
+ * through one lococo_process_sequence call (the training use of Algorithm 2; Section 3.2.1: the
+ * conv parameters are trained end to end).
+ * Q, K, V, O: the forward's tensors; cache_len_in: the cache fill count that forward started from
+ * (0: an empty cache); saved: what that forward wrote (it holds the cache before every step).
  * dQ, dK, dV (configured dtype) are overwritten; dG (fp32 [heads|1, M, c_in, k]) and
  * dbias (fp32 [heads|1, M], optional) are accumulated (+=), summed over the units that
  * share a weight set.  dK_cache_final/dV_cache_final may have ptr == NULL (zero).
+ * dK_cache_in/dV_cache_in ([batch, heads, M, d], configured dtype, ptr == NULL: not wanted) receive
+ * the gradient w.r.t. the cache the forward started from (rows at and beyond cache_len_in: zeros).
+ * A sequence processed in several forward calls is differentiated call by call, last call first,
+ * each call's dK_cache_in/dV_cache_in being the dK_cache_final/dV_cache_final of the call before it.
  * scratch: device memory of lococo_backward_scratch_bytes.
  */
 lococo_status lococo_backward_scratch_bytes(const lococo_handle* handle, int32_t L, int32_t B, size_t* out);
 lococo_status lococo_process_sequence_backward(lococo_handle* handle, lococo_tensor Q, lococo_tensor K,
                                                lococo_tensor V, lococo_tensor O, int32_t L, int32_t B,
-                                               const void* saved, lococo_tensor dO,
+                                               int32_t cache_len_in, const void* saved, lococo_tensor dO,
                                                lococo_tensor dK_cache_final, lococo_tensor dV_cache_final,
                                                lococo_tensor dQ, lococo_tensor dK, lococo_tensor dV, float* dG,
-                                               float* dbias, void* scratch, size_t scratch_bytes, void* stream);
+                                               float* dbias, lococo_tensor dK_cache_in, lococo_tensor dV_cache_in,
+                                               void* scratch, size_t scratch_bytes, void* stream);
 
 /* Synchronises `stream` and reads the device status word: LOCOCO_OK, or
  * LOCOCO_ERR_TIMEOUT if a bounded wait inside a kernel gave up (results invalid).  The word

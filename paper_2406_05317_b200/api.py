@@ -50,8 +50,8 @@ _SIGNATURES = {
     "lococo_host_staging_bytes": [_P, _I, ctypes.POINTER(ctypes.c_size_t)],
     "lococo_process_sequence_host": [_P, _P, _P, _P, _I, _I, _P, _P, _P, ctypes.POINTER(_I), _P, ctypes.c_size_t, _P],
     "lococo_backward_scratch_bytes": [_P, _I, _I, ctypes.POINTER(ctypes.c_size_t)],
-    "lococo_process_sequence_backward": [_P, _T, _T, _T, _T, _I, _I, _P, _T, _T, _T, _T, _T, _T, _P, _P, _P,
-                                         ctypes.c_size_t, _P],
+    "lococo_process_sequence_backward": [_P, _T, _T, _T, _T, _I, _I, _I, _P, _T, _T, _T, _T, _T, _T, _P, _P, _T, _T,
+                                         _P, ctypes.c_size_t, _P],
     "lococo_get_last_device_status": [_P, ctypes.POINTER(_I), _P],
     "lococo_launch_count": [_P, ctypes.POINTER(ctypes.c_int64)],
     "lococo_compress_step_static": [ctypes.POINTER(Config), _P, _P, _T, _T, _I, _T, _T, _I, _T, _T, _P],
@@ -218,12 +218,13 @@ class Lococo:
         return n.value
 
     def process_sequence_backward(self, Q, K, V, O, B, saved, dO, dK_cache_final, dV_cache_final, dQ, dK, dV, dG,
-                                  dbias, scratch):
+                                  dbias, scratch, cache_len_in=0, dK_cache_in=None, dV_cache_in=None):
+        """Gradients through one process_sequence call that started from `cache_len_in` cache rows."""
         _check(_lib.lococo_process_sequence_backward(
-            self._h, _view(Q), _view(K), _view(V), _view(O), Q.shape[2], B, _ptr(saved), _view(dO),
+            self._h, _view(Q), _view(K), _view(V), _view(O), Q.shape[2], B, cache_len_in, _ptr(saved), _view(dO),
             _view(dK_cache_final), _view(dV_cache_final), _view(dQ), _view(dK), _view(dV), _ptr(dG), _ptr(dbias),
-            scratch.data_ptr(), scratch.numel() * scratch.element_size(), _stream()),
-            "lococo_process_sequence_backward")
+            _view(dK_cache_in), _view(dV_cache_in), scratch.data_ptr(), scratch.numel() * scratch.element_size(),
+            _stream()), "lococo_process_sequence_backward")
 
     def device_status(self) -> int:
         out = _I()

@@ -58,6 +58,25 @@ def build(force: bool = False, verbose: bool = False) -> Path:
     return LIB
 
 
+PROBE_SRC = PKG.parent / "tests" / "cuda" / "wait_probe.cu"
+PROBE_LIB = PKG.parent / "tests" / "cuda" / "libwait_probe.so"
+
+
+def build_test_probe(force: bool = False) -> Path:
+    """Compile the test-only library (a kernel whose bounded wait is made to run out) next to its source.
+    It is not part of liblococo.so and exports nothing the header declares."""
+    deps = [PROBE_SRC, CSRC / "tc_common.cuh"]
+    if not force and PROBE_LIB.exists() and all(p.stat().st_mtime <= PROBE_LIB.stat().st_mtime for p in deps):
+        return PROBE_LIB
+    nvcc = os.environ.get("NVCC", "/usr/local/cuda/bin/nvcc")
+    tmp = PROBE_LIB.with_suffix(f".{os.getpid()}.tmp")
+    subprocess.check_call([nvcc, *ARCH, "-lineinfo", "-O3", "-std=c++17", "-Xcompiler", "-fPIC", "-shared", "-I", str(CSRC),
+                           "-o", str(tmp), str(PROBE_SRC)])
+    os.replace(tmp, PROBE_LIB)
+    return PROBE_LIB
+
+
 if __name__ == "__main__":
     build(force="--force" in sys.argv, verbose="-v" in sys.argv)
+    build_test_probe(force="--force" in sys.argv)
     print(LIB)

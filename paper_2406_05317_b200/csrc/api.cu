@@ -475,7 +475,9 @@ lococo_status lococo_process_sequence(lococo_handle* h, lococo_tensor Q, lococo_
     static_assert(sizeof(key) <= sizeof(lg.key), "key buffer too small");
     cudaStreamCaptureStatus cap = cudaStreamCaptureStatusNone;
     // (the legacy default stream cannot be captured: callers on it always get the eager loop)
-    const bool graph_ok = !lg.disabled && !h->prof.on && h->use_tensor && st != nullptr && st != cudaStreamLegacy &&
+    // (nor is the persistent loop captured: its step descriptors reach the device by a copy from a small ring of pinned
+    // host slots that later eager calls reuse, so a replay would read whatever the ring holds by then)
+    const bool graph_ok = !lg.disabled && !h->prof.on && h->use_tensor && !h->persistent_loop && st != nullptr && st != cudaStreamLegacy &&
                           st != cudaStreamPerThread && cudaStreamIsCapturing(st, &cap) == cudaSuccess && cap == cudaStreamCaptureStatusNone;
     const bool same = graph_ok && lg.key_len == sizeof(key) && std::memcmp(lg.key, &key, sizeof(key)) == 0;
     if (same && lg.exec) {
@@ -538,9 +540,10 @@ lococo_status lococo_host_staging_bytes(const lococo_handle* h, int32_t L, size_
 lococo_status lococo_process_sequence_host(lococo_handle* h, const void* Qh, const void* Kh, const void* Vh, int32_t L,
                                            int32_t B, void* Oh, void* Kc_h, void* Vc_h, int32_t* final_len,
                                            void* staging, size_t staging_bytes, void* stream) {
+    if (!h || !Qh || !Kh || !Vh || !Oh || !staging || L < 1) return LOCOCO_ERR_INVALID_ARG;
+    if (B < 1 || B > h->cfg.max_chunk) return LOCOCO_ERR_INVALID_ARG;   // the scratch is sized for chunks of at most max_chunk
     lococo_status s = ready(h);
     if (s) return s;
-    if (!Qh || !Kh || !Vh || !Oh || !staging || L < 1) return LOCOCO_ERR_INVALID_ARG;
     if (reinterpret_cast<uintptr_t>(staging) & 255u) return LOCOCO_ERR_INVALID_ARG;
     size_t need = 0;
     lococo_host_staging_bytes(h, L, &need);

@@ -497,6 +497,19 @@ __global__ void bwd_init_g_kernel(View gk_in, View gv_in, float* gK, float* gV, 
     }
 }
 
+// The gradient w.r.t. the cache the loop started from, out of the fp32 accumulators (all M rows; rows beyond the
+// initial fill count hold zeros).
+template <typename T>
+__global__ void bwd_store_g_kernel(const float* gK, const float* gV, View gk_out, View gv_out, int heads, int M, int d) {
+    const int u = blockIdx.y, n = u / heads, h = u % heads;
+    const int total = M * d;
+    for (int x = blockIdx.x * blockDim.x + threadIdx.x; x < total; x += gridDim.x * blockDim.x) {
+        const int row = x / d, ch = x % d;
+        if (gk_out.ptr) unit_base_mut<T>(gk_out, n, h)[(int64_t)row * gk_out.st + ch] = from_f32<T>(gK[(int64_t)u * total + x]);
+        if (gv_out.ptr) unit_base_mut<T>(gv_out, n, h)[(int64_t)row * gv_out.st + ch] = from_f32<T>(gV[(int64_t)u * total + x]);
+    }
+}
+
 bool launched() { return cudaGetLastError() == cudaSuccess; }
 
 // All kernels of one reversed step. Returns the number of launches or -1.
@@ -570,6 +583,12 @@ int init_g(View gk, View gv, float* gK, float* gV, int heads, int units, int M, 
     return launched() ? 1 : -1;
 }
 
+template <typename T>
+int store_g(const float* gK, const float* gV, View gk, View gv, int heads, int units, int M, int d, cudaStream_t st) {
+    bwd_store_g_kernel<T><<<dim3((M * d + 255) / 256, units), 256, 0, st>>>(gK, gV, gk, gv, heads, M, d);
+    return launched() ? 1 : -1;
+}
+
 }  // namespace
 }  // namespace lococo
 
@@ -624,14 +643,16 @@ lococo_status lococo_backward_scratch_bytes(const lococo_handle* h, int32_t L, i
 }
 
 lococo_status lococo_process_sequence_backward(lococo_handle* h, lococo_tensor Q, lococo_tensor K, lococo_tensor V,
-                                               lococo_tensor O, int32_t L, int32_t B, const void* saved, lococo_tensor dO,
-                                               lococo_tensor dKc_final, lococo_tensor dVc_final, lococo_tensor dQ,
-                                               lococo_tensor dK, lococo_tensor dV, float* dG, float* dbias, void* scratch,
+                                               lococo_tensor O, int32_t L, int32_t B, int32_t cache_len_in, const void* saved,
+                                               lococo_tensor dO, lococo_tensor dKc_final, lococo_tensor dVc_final,
+                                               lococo_tensor dQ, lococo_tensor dK, lococo_tensor dV, float* dG, float* dbias,
+                                               lococo_tensor dKc_in, lococo_tensor dVc_in, void* scratch,
                                                size_t scratch_bytes, void* stream) {
     if (!h) return LOCOCO_ERR_INVALID_ARG;
     if (!h->ws || !h->weights_set) return LOCOCO_ERR_WORKSPACE;
     const lococo_config& cfg = h->cfg;
     if (L < 1 || B < 1 || B > cfg.max_chunk || !saved || !dG || !scratch) return LOCOCO_ERR_INVALID_ARG;
+    if (cache_len_in < 0 || cache_len_in > cfg.M) return LOCOCO_ERR_INVALID_ARG;
     if ((reinterpret_cast<uintptr_t>(saved) & 255u) || (reinterpret_cast<uintptr_t>(scratch) & 255u) ||
         (reinterpret_cast<uintptr_t>(dG) & 15u))
         return LOCOCO_ERR_INVALID_ARG;
@@ -640,6 +661,7 @@ lococo_status lococo_process_sequence_backward(lococo_handle* h, lococo_tensor Q
         !bview_ok(dK, e) || !bview_ok(dV, e))
         return LOCOCO_ERR_INVALID_ARG;
     if ((dKc_final.ptr && !bview_ok(dKc_final, e)) || (dVc_final.ptr && !bview_ok(dVc_final, e))) return LOCOCO_ERR_INVALID_ARG;
+    if ((dKc_in.ptr && !bview_ok(dKc_in, e)) || (dVc_in.ptr && !bview_ok(dVc_in, e))) return LOCOCO_ERR_INVALID_ARG;
     if (dbias && !h->has_bias) return LOCOCO_ERR_INVALID_ARG;
     const Scratch sl = scratch_layout(h, B);
     if (scratch_bytes < sl.total) return LOCOCO_ERR_WORKSPACE;
@@ -667,10 +689,10 @@ lococo_status lococo_process_sequence_backward(lococo_handle* h, lococo_tensor Q
     if (launched_n < 0) return LOCOCO_ERR_CUDA;
     h->launches += launched_n;
 
-    // cache fill count before every step of the forward (empty cache at the start)
+    // cache fill count before every step of the forward
     int c_before[4096];
     if (n_chunks > 4096) return LOCOCO_ERR_UNSUPPORTED_SHAPE;
-    for (int n = 0, c = 0; n < n_chunks; ++n) {
+    for (int n = 0, c = cache_len_in; n < n_chunks; ++n) {
         const int b = std::min(B, L - n * B);
         c_before[n] = c;
         c = c + b <= cfg.M ? c + b : cfg.M;
@@ -708,6 +730,15 @@ lococo_status lococo_process_sequence_backward(lococo_handle* h, lococo_tensor Q
         f.eps = cfg.norm_eps; f.prot = h->prot; f.R = p.R; f.s = p.s;
         const int r = cfg.dtype == LOCOCO_F32 ? backward_step<float>(h, p, f, cfg.dtype, B, nullptr, st)
                                               : backward_step<__nv_bfloat16>(h, p, f, cfg.dtype, B, tb, st);
+        if (r < 0) return LOCOCO_ERR_CUDA;
+        h->launches += r;
+    }
+    // what the accumulators hold now is the gradient w.r.t. the cache the forward started from
+    if (dKc_in.ptr || dVc_in.ptr) {
+        const int r = cfg.dtype == LOCOCO_F32
+                          ? store_g<float>(gK, gV, bdev(dKc_in, 0, e), bdev(dVc_in, 0, e), cfg.heads, h->units, cfg.M, cfg.head_dim, st)
+                          : store_g<__nv_bfloat16>(gK, gV, bdev(dKc_in, 0, e), bdev(dVc_in, 0, e), cfg.heads, h->units, cfg.M,
+                                                   cfg.head_dim, st);
         if (r < 0) return LOCOCO_ERR_CUDA;
         h->launches += r;
     }

@@ -29,7 +29,7 @@ struct lococo_handle {
     // true once a kernel of this library has been launched in the current call: only then may the next one be
     // launched as a programmatic dependent (its early, pre-wait reads must not race with a foreign kernel)
     bool chain_open = false;
-    bool persistent_loop = false;   // chunk loop as one cooperative launch (LOCOCO_PATH_TENSOR_PERSISTENT)
+    bool persistent_loop = false;   // consecutive compress steps as one persistent launch (LOCOCO_PATH_TENSOR_PERSISTENT)
     bool weights_set = false;
     bool has_bias = false;
     char* ws = nullptr;     // caller-owned device workspace
@@ -75,7 +75,7 @@ bool tensor_step_direct(lococo_handle* h, const CompressParams& p);
 bool tensor_attention_supported(const lococo_handle* h, const AttnParams& p);
 int tensor_attention(lococo_handle* h, const AttnParams& p, cudaStream_t st);
 int tensor_chunk_step(lococo_handle* h, const AttnParams& a, const CompressParams& p, cudaStream_t st);
-// Persistent chunk loop: queue consecutive compress steps, then run them all in one cooperative launch.
+// Persistent chunk loop: queue consecutive compress steps, then run them all in one launch of one CTA per SM.
 bool tensor_sequence_add(lococo_handle* h, const AttnParams& a, const CompressParams& p, cudaStream_t st);
 int tensor_sequence_launch(lococo_handle* h, cudaStream_t st, void* prof);
 void tensor_sequence_release(lococo_handle* h);

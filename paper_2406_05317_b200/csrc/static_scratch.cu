@@ -1,6 +1,8 @@
 // lococo_compress_step_static: the compress step for callers that cannot allocate device
 // memory. Its scratch lives in a fixed array inside the library image instead of a
 // caller-provided workspace.
+#include <atomic>
+
 #include "common.cuh"
 
 namespace {
@@ -12,18 +14,19 @@ constexpr size_t kStaticScratchBytes = 8u << 20;  // 8 MiB, resident on every GP
 static __device__ __align__(256) unsigned char g_static_scratch[kStaticScratchBytes];
 
 constexpr int kMaxDevices = 64;
-unsigned char* g_scratch_addr[kMaxDevices] = {};
+std::atomic<unsigned char*> g_scratch_addr[kMaxDevices];
 
-// Device address of the array on the current device; looked up once per device.
+// Device address of the array on the current device; looked up once per device. Host threads that make
+// their first call at the same time each run the query and store the same address.
 unsigned char* scratch_for_current_device() {
     int dev = -1;
     if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return nullptr;
-    if (!g_scratch_addr[dev]) {
-        unsigned char* ptr = nullptr;
+    unsigned char* ptr = g_scratch_addr[dev].load(std::memory_order_acquire);
+    if (!ptr) {
         if (cudaGetSymbolAddress(reinterpret_cast<void**>(&ptr), g_static_scratch) != cudaSuccess) return nullptr;
-        g_scratch_addr[dev] = ptr;
+        g_scratch_addr[dev].store(ptr, std::memory_order_release);
     }
-    return g_scratch_addr[dev];
+    return ptr;
 }
 
 size_t align256(size_t x) { return (x + 255) / 256 * 256; }

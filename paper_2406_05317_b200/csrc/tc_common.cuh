@@ -40,8 +40,9 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
 // and in *failed (shared, makes later waits give up quickly), and returns false.
 // The caller carries on, so the kernel always terminates and frees its TMEM.
 constexpr uint32_t kWaitLimit = 1u << 22;
-static __device__ __noinline__ bool mbar_wait_slow(uint32_t bar, uint32_t parity, int* status, volatile int* failed, int code) {
-    const uint32_t limit = *failed ? 64u : kWaitLimit;
+static __device__ __noinline__ bool mbar_wait_slow(uint32_t bar, uint32_t parity, int* status, volatile int* failed, int code,
+                                                    uint32_t max_polls = kWaitLimit) {
+    const uint32_t limit = *failed ? 64u : max_polls;
     for (uint32_t i = 0; i < limit; ++i) {
         if (mbar_try_wait(bar, parity)) return true;
     }

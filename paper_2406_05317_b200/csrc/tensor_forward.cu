@@ -11,8 +11,10 @@
 //      rounding, and the result is written back to shared memory as the A operand of
 //   4. Eq. 4 / Eq. 5: U_K += R * X_K and U_V += R * X_V, which read the SAME staged tiles,
 //      now contracted over positions (MN-major B operand);
-// and the division by the row sum is applied after all tiles are summed (it commutes
-// with the blend), by finalize_parts_kernel.
+// and the division by the row sum is applied after all tiles are summed (it commutes with the blend):
+// by the CTA itself where it saw every position of its slots, by the CTA of a (unit, slot block) that
+// arrives last at its store where the chunk loop lets the step merge its partial sets, and by
+// finalize_parts_kernel after a stand-alone compress step.
 #include <cuda.h>   // tensor map types only: the encoder is looked up at run time
 
 #include <algorithm>
@@ -544,7 +546,9 @@ __global__ void __launch_bounds__(256) finalize_parts_kernel(TcCompressParams P)
 // ------------------------------------------------------------------ Eq. 1, chunk form
 // One CTA = 128 queries of one unit, pipelined over 128-key tiles of [cache; chunk] with three
 // kinds of warps that only meet at mbarriers:
-//   loaders (2 warps)   stage Q once and the K/V tiles, double-buffered, with cp.async;
+//   loaders (3 warps)   one lane drives the tensor copy engine: Q once, then the K/V tiles, double-buffered;
+//                       the warps copy by hand (cp.async) only the tile that straddles the end of a
+//                       partly filled cache, or an operand whose strides the driver would not encode;
 //   MMA issuer (1 lane) S_t = Q K_t^T into one of two TMEM buffers, then O += P_{t-1} V_{t-1},
 //                       so the next tile's logits are computed while this tile's softmax runs;
 //   softmax (8 warps)   two threads per query row (64 columns each): row maximum, P = exp2(s - m)
@@ -1262,6 +1266,19 @@ static cudaError_t launch_overlapped(void (*kernel)(Param), dim3 grid, dim3 bloc
     return cudaLaunchKernelEx(&cfg, kernel, arg);
 }
 
+
+// The dynamic shared-memory limit of a kernel is a per-device attribute: it is set on the first launch on each device.
+template <typename Kernel>
+static bool smem_limit_set(Kernel kernel, int bytes, bool (&done)[64]) {
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return false;
+    if (!done[dev]) {
+        if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes) != cudaSuccess) return false;
+        done[dev] = true;
+    }
+    return true;
+}
+
 // finalize (+ optional mixing-weight output) after the compress CTAs of either launch form
 static int finish_compress(const TcCompressParams& P, cudaStream_t st) {
     const CompressParams& p = P.base;
@@ -1283,12 +1300,8 @@ static int finish_compress(const TcCompressParams& P, cudaStream_t st) {
 int tensor_compress(lococo_handle* h, const CompressParams& p, cudaStream_t st) {
     TcCompressParams P;
     if (!build_compress_params(h, p, false, &P)) return -1;
-    static bool attr_set = false;
-    if (!attr_set) {
-        if (cudaFuncSetAttribute(compress_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxSmem) != cudaSuccess)
-            return -1;
-        attr_set = true;
-    }
+    static bool attr_set[64] = {};
+    if (!smem_limit_set(compress_tc_kernel, kMaxSmem, attr_set)) return -1;
     dim3 grid(P.parts, P.slot_blocks, p.units);
     prof_begin(p.prof, 0, st);
     // the full 227 KB keeps one CTA per SM, so a CTA always finds its 512 TMEM columns free
@@ -1380,12 +1393,8 @@ static bool build_step_params(lococo_handle* h, const AttnParams& a, const Compr
 int tensor_chunk_step(lococo_handle* h, const AttnParams& a, const CompressParams& p, cudaStream_t st) {
     TcStepParams P;
     if (!build_step_params(h, a, p, &P)) return -1;
-    static bool attr_set = false;
-    if (!attr_set) {
-        if (cudaFuncSetAttribute(chunk_step_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxSmem) != cudaSuccess)
-            return -1;
-        attr_set = true;
-    }
+    static bool attr_set[64] = {};
+    if (!smem_limit_set(chunk_step_tc_kernel, kMaxSmem, attr_set)) return -1;
     // one CTA per (unit, slot block) and an output cache that is not the input: no partials, no finalize pass
     const bool own_output = p.W_out == nullptr && p.k_out.ptr != p.xk.cache.ptr && p.v_out.ptr != p.xv.cache.ptr;
     P.comp.direct = own_output && P.comp.parts == 1;
@@ -1505,12 +1514,8 @@ bool tensor_attention_supported(const lococo_handle* h, const AttnParams& p) {
 }
 
 int tensor_attention(lococo_handle* h, const AttnParams& p, cudaStream_t st) {
-    static bool attr_set = false;
-    if (!attr_set) {
-        if (cudaFuncSetAttribute(attention_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kAttnSmem) != cudaSuccess)
-            return -1;
-        attr_set = true;
-    }
+    static bool attr_set[64] = {};
+    if (!smem_limit_set(attention_tc_kernel, (int)kAttnSmem, attr_set)) return -1;
     TcAttnParams P{};
     P.base = p;
     P.status = reinterpret_cast<int*>(h->ws + h->off_status);

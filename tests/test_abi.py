@@ -82,6 +82,22 @@ def test_calls_without_workspace_or_weights_are_refused(api):
     lib.lococo_destroy(h)
 
 
+def test_host_entry_point_checks_the_chunk_size_before_anything_else(api):
+    # a chunk size of 0 would divide by zero on the host, one above max_chunk would overrun the scratch
+    st, h = make(api)
+    lib = api.raw()
+    buf = ctypes.c_void_p(4096)
+    n = ctypes.c_int32()
+    for B in (0, -3, 17):
+        assert lib.lococo_process_sequence_host(h, buf, buf, buf, 64, B, buf, None, None, ctypes.byref(n), buf,
+                                                1 << 30, None) == api.ERR_INVALID_ARG, B
+    # a valid chunk size gets as far as the missing workspace
+    assert lib.lococo_process_sequence_host(h, buf, buf, buf, 64, 16, buf, None, None, ctypes.byref(n), buf,
+                                            1 << 30, None) == api.ERR_WORKSPACE
+    T = api.Tensor(ctypes.c_void_p(4096), 1024, 1024, 64)
+    lib.lococo_destroy(h)
+
+
 def test_status_strings(api):
     seen = {api.status_string(s) for s in range(6)}
     assert len(seen) == 6 and "ok" in seen

@@ -2,6 +2,8 @@
 times (tensor-core path, side stream, repeated calls so that the CUDA-graph replay is what runs).
 Where the oracle cannot finish the whole problem in seconds it checks whole (sequence, head) units
 taken out of the full run, sampled cache slots, and properties that hold at any size."""
+import time
+
 import numpy as np
 import pytest
 import torch
@@ -70,7 +72,7 @@ def test_cfg3_full_size_units_against_the_oracle():
     assert bool(torch.isfinite(O.float()).all())
 
 
-def test_cfg4_full_size_sampled_slots_and_cross_path():
+def test_cfg4_full_size_against_the_oracle():
     # fine-tuning shape at full size: 32 heads, M=512, B=4096, 32768 tokens (8 compress steps).
     from oracle import lococo_oracle as orc
     from paper_2406_05317_b200 import api
@@ -101,9 +103,33 @@ def test_cfg4_full_size_sampled_slots_and_cross_path():
         Or, _ = orc.attention(Q[0, h, :640], K[0, h, :640], V[0, h, :640], 0)
         assert_close(to_host(O1[0, h]), Or, "bf16", f"cfg4 head {h} first queries")
         assert_close(to_host(O[0, h, :640]), Or, "bf16", f"cfg4 head {h} first queries (full run)")
-    # (3) the whole 8-step recurrence: tensor-core path against the CUDA-core path (itself checked
-    #     against the oracle on the shortened cfg4 slice), same bar as against the oracle
+    # (3) the whole 8-step recurrence (Algorithm 2 at M = 512, B = 4096, heavy-tailed keys) against the
+    #     oracle: two whole heads taken out of the full run, every output element
+    t0 = time.time()
+    for h in (0, 19):
+        Or, Kr, Vr, cr, _ = orc.process_sequence(Q[0, h], K[0, h], V[0, h], G[0], w.B)
+        assert cr == w.M
+        assert_close(to_host(O[0, h]), Or, "bf16", f"cfg4 head {h} O, all 8 chunks")
+        assert_close(to_host(Kc[0, h]), Kr, "bf16", f"cfg4 head {h} final K cache")
+        assert_close(to_host(Vc[0, h]), Vr, "bf16", f"cfg4 head {h} final V cache")
+    print(f"cfg4: oracle, 2 heads x 8 chunks: {time.time() - t0:.1f} s on {orc.threads()} threads")
+    # (4) the other heads: tensor-core path against the CUDA-core path, same bar
     O2, Kc2, Vc2, _ = run_full(api, w, repeats=1, path=api.PATH_SIMT)
     assert_close(to_host(O[0, :4]), to_host(O2[0, :4]), "bf16", "cfg4 O, tensor vs CUDA-core path")
     assert_close(to_host(Kc), to_host(Kc2), "bf16", "cfg4 K cache, tensor vs CUDA-core path")
     assert_close(to_host(Vc), to_host(Vc2), "bf16", "cfg4 V cache, tensor vs CUDA-core path")
+
+
+def test_cfg5_full_shape_one_head_gradients_against_the_oracle():
+    # the fine-tuning step at its real shape (M = 512, B = 4096, 32768 tokens, 8 compress steps, heavy-tailed
+    # keys) on the one-head slice: dQ, dK, dV and the conv-weight gradient through all 8 steps against the
+    # float64 oracle's, every element
+    from oracle import lococo_oracle as orc
+    from paper_2406_05317_b200 import api
+    from tests.test_gpu_backward import run_backward, check_gradients
+    w = wl.CONFIGS["cfg5"].slice(heads=1)
+    got, (Q, K, V, G, bvec, PO, PK, PV) = run_backward(api, w)
+    t0 = time.time()
+    rQ, rK, rV, rG, _ = orc.grad_batch(Q, K, V, G, w.B, PO, PK, PV)
+    print(f"cfg5: oracle gradients, 1 head x 8 chunks: {time.time() - t0:.1f} s on {orc.threads()} threads")
+    check_gradients(w, got, dict(dQ=rQ, dK=rK, dV=rV, dG=rG))

@@ -325,7 +325,7 @@ def test_repeated_identical_calls_replay_the_same_loop(api):
 
 
 def test_persistent_loop_equals_stepwise_launches(api):
-    # PATH_TENSOR_PERSISTENT runs the compress steps of a call inside one cooperative kernel; the
+    # PATH_TENSOR_PERSISTENT runs the compress steps of a call inside one persistent kernel; the
     # default tensor-core path launches every step: same CTA bodies, same bits, fewer launches
     w = wl.CONFIGS["cfg3"].slice(batch=2, heads=4, L=1024)     # 2 fill steps, then 14 compress steps
     Q, K, V = (to_device(x, w.dtype) for x in wl.make_qkv(w))
@@ -343,6 +343,46 @@ def test_persistent_loop_equals_stepwise_launches(api):
     assert res[0][3] == res[1][3] == w.M
     assert torch.equal(res[0][0], res[1][0]) and torch.equal(res[0][1], res[1][1]) and torch.equal(res[0][2], res[1][2])
     assert res[0][4] < res[1][4]        # one persistent launch instead of two per step
+
+
+def test_persistent_loop_repeated_calls_survive_other_calls_on_the_handle(api):
+    # The persistent kernel's step descriptors travel through a small ring of pinned host slots. Identical
+    # calls repeated on a side stream (where the per-chunk path would replay a CUDA graph), with a host-buffer
+    # call of more chunks than the ring has slots in between, must keep giving the same bits.
+    w = wl.CONFIGS["cfg2"].slice(heads=2, L=3072)      # 6 chunks
+    Qh, Kh, Vh = wl.make_qkv(w)
+    Q, K, V = (to_device(x, w.dtype) for x in (Qh, Kh, Vh))
+    ctx, _, _ = make_ctx(api, w, path=api.PATH_TENSOR_PERSISTENT)
+    side = torch.cuda.Stream()
+
+    def call():
+        O = torch.empty_like(Q)
+        Kc = torch.zeros(w.batch, w.heads, w.M, w.d, dtype=Q.dtype, device="cuda")
+        Vc = torch.zeros_like(Kc)
+        return O, Kc, Vc
+
+    O, Kc, Vc = call()
+    outs = []
+    torch.cuda.synchronize()
+    for rep in range(5):
+        if rep == 3:
+            pin = lambda x: torch.from_numpy(x).to(torch.bfloat16).pin_memory()
+            hO = torch.empty(Q.shape, dtype=torch.bfloat16).pin_memory()
+            staging = torch.empty(ctx.host_staging_bytes(w.L) + 256, dtype=torch.uint8, device="cuda")
+            off = (-staging.data_ptr()) % 256
+            with torch.cuda.stream(side):
+                ctx.process_sequence_host(pin(Qh), pin(Kh), pin(Vh), w.B, hO, staging[off:])
+            host_O = hO.clone()
+        Kc.zero_(); Vc.zero_()
+        torch.cuda.synchronize()
+        with torch.cuda.stream(side):
+            assert ctx.process_sequence(Q, K, V, w.B, O, Kc, Vc, 0) == w.M
+        torch.cuda.synchronize()
+        outs.append((O.clone(), Kc.clone(), Vc.clone()))
+    assert ctx.device_status() == api.OK
+    for o, k, v in outs[1:]:
+        assert torch.equal(o, outs[0][0]) and torch.equal(k, outs[0][1]) and torch.equal(v, outs[0][2])
+    assert torch.equal(host_O, outs[0][0].cpu())
 
 
 @pytest.mark.parametrize("heads,L", [(32, 1536), (4, 2048)])
