@@ -65,6 +65,8 @@ struct TcCompressParams {
                                   // (unit, slot block) sums the sets and writes the cache rows itself, no finalize pass
     int* merge_count;             // [units][slot blocks][2]: CTAs arrived at their store, partial sets stored; the last CTA puts the zeros back
     int n_tile, tiles, parts, tiles_per_part, halves, stages, rows_pad, slot_blocks;
+    int pair;                     // 1: generation-stage form, one CTA per TWO units that share a weight set (compress_pair_body)
+    int pairs;                    // CTAs of that form
 };
 
 // G [sets][M][C][k] -> per (set, slot block, tap, 128-channel half) a 32 KB image of the
@@ -465,6 +467,348 @@ __device__ __forceinline__ void compress_body(const TcCompressParams& P, uint8_t
     __syncthreads();
     if (tid == 128) {
         for (int s = 0; s < 2 * NS + 2; ++s) mbar_inval(bar_full + 8 * s);
+    }
+}
+
+// ------------------------------------------------------------------ generation stage (Section 3.3: segments of one token)
+// With chunks of one (or a few) tokens S = c + b is barely larger than M: a compress step per unit is a single
+// short position tile, and a CTA per unit streams the whole weight image (k stages of 32 KB) from L2 for about
+// 130 positions, so with more units than SMs the step runs at what L2 delivers and not at the tensor pipe's rate.
+// Here one CTA takes TWO units that use the same weight set: every weight stage feeds the MMAs of both (twice the
+// MMA time per stage, half the weight traffic per unit). Conditions (checked on the host): M = 128, a full cache
+// (c = M), c_in = d, one position tile (n_tile = S rounded up to 16), an output cache that is not the input cache.
+//   TMEM: unit x owns columns 256x..256x+255: the conv accumulator D first (n_tile columns), and once D has been
+//   turned into R in shared memory the two blend accumulators U_K, U_V (128 columns each) take its place.
+//   Shared memory: [one region: the weight ring (4 stages) while the conv runs; afterwards R of both units and
+//   the two value tiles of the cache rows, which only the blends need and which the tensor copy engine brings in
+//   (128-byte swizzle, as the attention kernel's value tiles) while the accumulators are read out; at the end the
+//   staging buffers of the cache write] [key tiles x2: rows -pad .. max(S+pad, n_tile)-1, un-swizzled].
+//   The value blend runs on the tensor cores over the cache rows; the few chunk rows (positions c .. S-1) are added
+//   on the CUDA cores from the same bf16 R (fp32 products and sums, as the MMA's).
+// Units of pair `pair`: with one weight set for all heads, units 2*pair and 2*pair+1; with a set per head, the same
+// head of sequences 2*i and 2*i+1 (pair = i*heads + head). The second unit may be missing (odd count).
+__device__ __forceinline__ void pair_units(const CompressParams& p, int pair, int& u0, int& u1) {
+    if (p.weights_per_head) {
+        const int h = pair % p.heads, i = pair / p.heads, batch = p.units / p.heads;
+        u0 = 2 * i * p.heads + h;
+        u1 = 2 * i + 1 < batch ? u0 + p.heads : -1;
+    } else {
+        u0 = 2 * pair;
+        u1 = u0 + 1 < p.units ? u0 + 1 : -1;
+    }
+}
+
+constexpr int kPairStages = 4;
+constexpr uint32_t kPairVTile = 32768;            // 128 cache rows x 128 channels, two 64-channel halves of 16 KB (128-byte swizzle)
+constexpr uint32_t kPairOutRow = 272;             // bytes per row of a staged output tile: 256 + 16, so that 16-byte accesses of 8 rows miss each other's banks
+constexpr uint32_t kPairOutTile = kSlots * kPairOutRow;
+
+// Eight MMAs of one K loop (128 channels in steps of 16) from ONE instruction block: descriptors advance by fixed steps,
+// the first MMA overwrites the accumulator when `acc_first` is 0. Keeps the issuing thread's instruction count per MMA
+// below the MMA's own duration at small N.
+__device__ __forceinline__ void umma_ss_k8(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t astep, uint32_t bstep,
+                                           uint32_t idesc, uint32_t acc_first) {
+    asm volatile(
+        "{\n\t.reg .pred p0, p1;\n\t.reg .b64 a, b, sa, sb;\n\t"
+        "setp.ne.b32 p0, %6, 0;\n\tsetp.eq.b32 p1, 0, 0;\n\t"
+        "cvt.u64.u32 sa, %4;\n\tcvt.u64.u32 sb, %5;\n\t"
+        "mov.b64 a, %1;\n\tmov.b64 b, %2;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], a, b, %3, p0;\n\t"
+        "add.u64 a, a, sa;\n\tadd.u64 b, b, sb;\n\ttcgen05.mma.cta_group::1.kind::f16 [%0], a, b, %3, p1;\n\t"
+        "add.u64 a, a, sa;\n\tadd.u64 b, b, sb;\n\ttcgen05.mma.cta_group::1.kind::f16 [%0], a, b, %3, p1;\n\t"
+        "add.u64 a, a, sa;\n\tadd.u64 b, b, sb;\n\ttcgen05.mma.cta_group::1.kind::f16 [%0], a, b, %3, p1;\n\t"
+        "add.u64 a, a, sa;\n\tadd.u64 b, b, sb;\n\ttcgen05.mma.cta_group::1.kind::f16 [%0], a, b, %3, p1;\n\t"
+        "add.u64 a, a, sa;\n\tadd.u64 b, b, sb;\n\ttcgen05.mma.cta_group::1.kind::f16 [%0], a, b, %3, p1;\n\t"
+        "add.u64 a, a, sa;\n\tadd.u64 b, b, sb;\n\ttcgen05.mma.cta_group::1.kind::f16 [%0], a, b, %3, p1;\n\t"
+        "add.u64 a, a, sa;\n\tadd.u64 b, b, sb;\n\ttcgen05.mma.cta_group::1.kind::f16 [%0], a, b, %3, p1;\n\t}" ::"r"(d_tmem),
+        "l"(adesc), "l"(bdesc), "r"(idesc), "r"(astep), "r"(bstep), "r"(acc_first)
+        : "memory");
+}
+
+struct PairLayout {
+    uint32_t rows_k, lbo_k, r_bytes, x_bytes, total;
+};
+__host__ __device__ inline PairLayout pair_layout(int S, int n_tile, int k) {
+    const int pad = (k - 1) / 2;
+    PairLayout L;
+    // rows the conv reads for valid columns (S + k - 1) and rows the key blend reads (pad + n_tile), odd so that the 16
+    // channel groups of a row fall into different banks
+    L.rows_k = (uint32_t)(((S + k - 1 > pad + n_tile) ? S + k - 1 : pad + n_tile) | 1);
+    L.lbo_k = L.rows_k * 16u;
+    L.r_bytes = (uint32_t)(n_tile / 8) * 2048u;
+    uint32_t x = kPairStages * (uint32_t)kStageBytes;
+    if (x < 2u * L.r_bytes + 2u * kPairVTile) x = 2u * L.r_bytes + 2u * kPairVTile;
+    if (x < 4u * kPairOutTile) x = 4u * kPairOutTile;
+    L.x_bytes = x;
+    L.total = 1024u + x + 2u * 16u * L.lbo_k + (2 * kPairStages + 3) * 8u + 16u + 2u * 3u * kSlots * 4u;
+    return L;
+}
+
+// `vmap`: tensor map of the value cache ([batch, heads, c rows, 128] in boxes of 128 rows x 64 channels), in kernel
+// parameter space.
+__device__ __forceinline__ void compress_pair_body(const TcCompressParams& P, const CUtensorMap* vmap, uint8_t* smem_raw,
+                                                   uint32_t tmem, int pair) {
+    const CompressParams& p = P.base;
+    const int tid = threadIdx.x, warp = tid >> 5;
+    const int eg = warp >> 2;                          // epilogue group: which column chunks
+    const int rl = (warp & 3) * 32 + (tid & 31);       // accumulator row = slot
+    const int n_tile = P.n_tile, pad = (p.k - 1) / 2;
+    const PairLayout L = pair_layout(p.S, n_tile, p.k);
+    const uint32_t lbo_k = L.lbo_k, r_bytes = L.r_bytes;
+    int units[2];
+    pair_units(p, pair, units[0], units[1]);
+    const int nu = units[1] >= 0 ? 2 : 1;
+
+    // the swizzle of the value tiles is a function of the shared-memory address: the region starts on a 1024-byte boundary
+    uint8_t* x_ptr = smem_raw + ((1024u - (smem_u32(smem_raw) & 1023u)) & 1023u);
+    uint8_t* zk_ptr = x_ptr + L.x_bytes;
+    uint64_t* bars = reinterpret_cast<uint64_t*>(zk_ptr + 2 * 16 * lbo_k);
+    volatile int* failed = reinterpret_cast<volatile int*>(bars + 2 * kPairStages + 3);
+    float* sums = reinterpret_cast<float*>(const_cast<int*>(failed) + 4);          // [2 units][3 groups][128 rows]
+    const uint32_t ring = smem_u32(x_ptr), zk = smem_u32(zk_ptr);
+    const uint32_t vt = ring + 2 * r_bytes;                                         // value tiles, after R of both units
+    const uint32_t bar_full = smem_u32(bars), bar_empty = bar_full + 8 * kPairStages;
+    const uint32_t bar_acc = bar_empty + 8 * kPairStages, bar_blend = bar_acc + 8, bar_v = bar_blend + 8;
+
+    if (tid == 128) {
+        for (int s = 0; s < kPairStages; ++s) {
+            mbar_init(bar_full + 8 * s, 1);
+            mbar_init(bar_empty + 8 * s, 1);
+        }
+        mbar_init(bar_acc, 1);
+        mbar_init(bar_blend, 1);
+        mbar_init(bar_v, 1);
+        *failed = 0;
+        fence_barrier_init();
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+
+    const int h0 = units[0] % p.heads;
+    const int set = p.weights_per_head ? h0 : 0;
+    const __nv_bfloat16* gimg = P.gimage + (int64_t)set * p.k * (kStageBytes / 2);   // one slot block, one channel half
+    const uint32_t idesc_conv = instr_desc_bf16(n_tile, false, false);
+    const uint32_t idesc_blend = instr_desc_bf16(kD, false, true);
+    const int slot = rl;
+    float bias_i = 0.f;
+    if (p.bias) bias_i = p.bias[(p.weights_per_head ? h0 * p.M : 0) + slot];
+    const int total = p.k;
+
+    auto load_stage = [&](int it) {
+        const uint32_t s = it % kPairStages;
+        if (it >= kPairStages) mbar_wait(bar_empty + 8 * s, ((it / kPairStages) - 1) & 1, P.status, failed, 31);
+        mbar_expect_tx(bar_full + 8 * s, kStageBytes);
+        bulk_load(ring + s * kStageBytes, gimg + (int64_t)it * (kStageBytes / 2), kStageBytes, bar_full + 8 * s);
+    };
+    if (tid == 160) {
+        for (int i = 0; i < min(kPairStages, total); ++i) load_stage(i);
+    }
+    // ---- 1. stage the key rows: the tile of unit x holds positions -pad .. rows_k-pad-1 (zeros outside [0,S)).
+    // Each thread owns one 8-channel group and every 24th row. `rows_of`: 1 only rows outside the cache (chunk rows and
+    // zeros), 2 only cache rows.
+    auto stage_keys = [&](int x, int rows_of) {
+        const int u = units[x], n = u / p.heads, h = u % p.heads;
+        const int q = tid & 15;
+        const __nv_bfloat16* cbase = unit_base<__nv_bfloat16>(p.xk.cache, n, h) + q * 8;
+        const __nv_bfloat16* kbase = unit_base<__nv_bfloat16>(p.xk.chunk, n, h) + q * 8;
+        const uint32_t d0 = zk + x * 16 * lbo_k + q * lbo_k;
+        for (int r = tid >> 4; r < (int)L.rows_k; r += kThreads / 16) {
+            const int j = r - pad;
+            const bool valid = j >= 0 && j < p.S;
+            const bool in_cache = valid && j < p.xk.c;
+            if ((rows_of == 1 && in_cache) || (rows_of == 2 && !in_cache)) continue;
+            const __nv_bfloat16* src = !valid ? kbase : (in_cache ? cbase + (int64_t)j * p.xk.cache.st : kbase + (int64_t)(j - p.xk.c) * p.xk.chunk.st);
+            cp_async16(d0 + r * 16, src, valid ? 16u : 0u);
+        }
+    };
+    for (int x = 0; x < nu; ++x) stage_keys(x, 1);
+    wait_for_earlier_kernels();          // the cache rows are the previous step's result
+    for (int x = 0; x < nu; ++x) stage_keys(x, 2);
+    cp_async_wait_all();
+    fence_proxy_async();
+    __syncthreads();
+
+    // ---- 2. Eq. 6: every weight stage (one tap) feeds both units' accumulators
+    if (tid == 160) {
+        for (int it = kPairStages; it < total; ++it) load_stage(it);
+    } else if (tid == 128) {
+        const uint64_t a0 = smem_desc(ring, 2048, 128);
+        const uint64_t b0 = smem_desc(zk, lbo_k, 128), b1 = smem_desc(zk + 16 * lbo_k, lbo_k, 128);
+        const uint32_t bstep = (2 * lbo_k) >> 4;
+        uint32_t st = 0, ph = 0;
+        for (int it = 0; it < total; ++it) {
+            mbar_wait(bar_full + 8 * st, ph, P.status, failed, 32);
+            tc_fence_after();
+            const uint64_t ad = a0 + st * (uint32_t)(kStageBytes >> 4);
+            umma_ss_k8(tmem, ad, b0 + it, 256u, bstep, idesc_conv, it != 0);              // tap t = row offset t (16 bytes per row)
+            if (nu == 2) umma_ss_k8(tmem + 256, ad, b1 + it, 256u, bstep, idesc_conv, it != 0);
+            umma_commit(bar_empty + 8 * st);
+            if (++st == (uint32_t)kPairStages) { st = 0; ph ^= 1; }
+        }
+        umma_commit(bar_acc);
+    }
+    mbar_wait(bar_acc, 0, P.status, failed, 33);
+    tc_fence_after();
+    // the ring is idle now: the value tiles of the cache rows (needed by the blends only) are requested here, through
+    // the tensor copy engine, and arrive while the accumulators are read out
+    if (tid == 160) {
+        mbar_expect_tx(bar_v, (uint32_t)nu * kPairVTile);
+        for (int x = 0; x < nu; ++x) {
+            const int u = units[x], n = u / p.heads, h = u % p.heads;
+            tma_load_4d(vt + x * kPairVTile, vmap, 0, 0, h, n, bar_v);
+            tma_load_4d(vt + x * kPairVTile + kPairVTile / 2, vmap, 64, 0, h, n, bar_v);
+        }
+    }
+
+    // ---- 3. accumulators -> bias, ReLU, row sums (Eq. 7), bf16 -> A operands of the blends (over the idle ring)
+    const uint32_t lane_addr = tmem + ((uint32_t)((warp & 3) * 32) << 16);
+    const bool keep = slot < p.prot;
+#pragma unroll 1                                  // (one copy of the code for both units: code that runs once costs its own fetch)
+    for (int x = 0; x < nu; ++x) {
+        {
+            float ssum = 0.f;
+            for (int c0 = eg * 32; c0 < n_tile; c0 += 96) {
+                uint32_t v[32];
+                tmem_ld32(lane_addr + x * 256 + c0, v);
+                tmem_ld_wait();
+#pragma unroll
+                for (int e = 0; e < 32; e += 8) {
+                    if (c0 + e >= n_tile) break;          // n_tile is a multiple of 16, not of 32
+                    uint32_t pk[4];
+#pragma unroll
+                    for (int y = 0; y < 8; y += 2) {
+                        const int ja = c0 + e + y;
+                        float ra = fmaxf(__uint_as_float(v[e + y]) + bias_i, 0.f);
+                        float rb = fmaxf(__uint_as_float(v[e + y + 1]) + bias_i, 0.f);
+                        if (keep) { ra = ja == slot ? 1.f : 0.f; rb = ja + 1 == slot ? 1.f : 0.f; }   // unit row (Section 5.2)
+                        if (ja >= p.S) ra = 0.f;
+                        if (ja + 1 >= p.S) rb = 0.f;
+                        const __nv_bfloat162 pr = __floats2bfloat162_rn(ra, rb);
+                        pk[y >> 1] = *reinterpret_cast<const uint32_t*>(&pr);
+                        ssum += __low2float(pr) + __high2float(pr);
+                    }
+                    *reinterpret_cast<uint4*>(x_ptr + x * r_bytes + ((c0 + e) >> 3) * 2048 + rl * 16) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
+                }
+            }
+            sums[(x * 3 + eg) * kSlots + rl] = ssum;
+        }
+    }
+    fence_proxy_async();
+    tc_fence_before();
+    __syncthreads();
+
+    // ---- 4. Eq. 4, Eq. 5 (unnormalised) into the columns the conv accumulators occupied: keys over all positions
+    // from the staged key tiles, values over the cache rows from the swizzled tiles
+    if (tid == 128) {
+        tc_fence_after();
+        for (int x = 0; x < nu; ++x) {
+            uint64_t ad = smem_desc(ring + x * r_bytes, 2048, 128);
+            uint64_t bk = smem_desc(zk + x * 16 * lbo_k + (uint32_t)pad * 16, 128, lbo_k);
+            for (int kk = 0; kk < n_tile / 16; ++kk) {
+                umma_ss(tmem + x * 256, ad, bk, idesc_blend, kk != 0);
+                ad += (2 * 2048) >> 4;      // 16 positions = two 8-position groups of R
+                bk += (16 * 16) >> 4;       // 16 rows of the key tile
+            }
+        }
+        mbar_wait(bar_v, 0, P.status, failed, 35);
+        tc_fence_after();
+        for (int x = 0; x < nu; ++x) {
+            const uint64_t ad = smem_desc(ring + x * r_bytes, 2048, 128);
+            const uint64_t bv = smem_desc_sw128(vt + x * kPairVTile, kPairVTile / 2, 1024);
+            // 16 cache rows = two 8-row groups of 1024 bytes per step
+            umma_ss_k8(tmem + x * 256 + 128, ad, bv, 256u, 128u, idesc_blend, 0);
+        }
+        umma_commit(bar_blend);
+    }
+    mbar_wait(bar_blend, 0, P.status, failed, 34);
+    tc_fence_after();
+
+    // ---- 5. Eq. 7 after Eq. 4-5: add the chunk rows' share of the value blend, divide by the row sum, and write the
+    // cache rows. A thread owns a slot; the rows are staged in shared memory so that the stores to the cache are
+    // whole 256-byte rows (a warp storing 32 rows' pieces directly pays for 32 separate segments per instruction).
+    const int n_tail = p.S - p.xk.c;                     // chunk rows: positions c .. S-1 (<= 16 of them)
+    float rtail[2][16];
+#pragma unroll
+    for (int x = 0; x < 2; ++x) {
+        const uint8_t* rrow = x_ptr + x * r_bytes + rl * 16;
+#pragma unroll
+        for (int g = 0; g < 2; ++g) {
+            uint4 w4 = make_uint4(0u, 0u, 0u, 0u);
+            if (x < nu && p.xk.c + 8 * g < n_tile) w4 = *reinterpret_cast<const uint4*>(rrow + ((p.xk.c >> 3) + g) * 2048);
+            const __nv_bfloat162* h2 = reinterpret_cast<const __nv_bfloat162*>(&w4);
+#pragma unroll
+            for (int y = 0; y < 4; ++y) {
+                const float2 f = __bfloat1622float2(h2[y]);
+                rtail[x][8 * g + 2 * y] = f.x;
+                rtail[x][8 * g + 2 * y + 1] = f.y;
+            }
+        }
+    }
+    __syncthreads();                                      // R has been read: its space now stages the output rows
+#pragma unroll 1
+    for (int x = 0; x < nu; ++x) {
+        const int u = units[x], n = u / p.heads, h = u % p.heads;
+        const float tot = slot < p.prot ? 1.f : sums[(x * 3) * kSlots + rl] + sums[(x * 3 + 1) * kSlots + rl] + sums[(x * 3 + 2) * kSlots + rl] + p.eps;
+        const float inv = 1.f / tot;
+        if (eg == 0) p.s[(int64_t)u * p.M + slot] = tot;
+        const __nv_bfloat16* vn = unit_base<__nv_bfloat16>(p.xv.chunk, n, h);
+#pragma unroll 1
+        for (int piece = eg; piece < 2 * (kD / 32); piece += 3) {
+            const int mat = piece & 1, c0 = (piece >> 1) * 32;
+            uint32_t a[32];
+            tmem_ld32(lane_addr + x * 256 + mat * 128 + c0, a);
+            tmem_ld_wait();
+            float acc[32];
+#pragma unroll
+            for (int e = 0; e < 32; ++e) acc[e] = __uint_as_float(a[e]);
+            if (mat == 1) {
+#pragma unroll
+                for (int y = 0; y < 16; ++y) {
+                    if (y >= n_tail) break;
+                    const float w = x == 0 ? rtail[0][y] : rtail[1][y];
+                    const uint4* row = reinterpret_cast<const uint4*>(vn + (int64_t)y * p.xv.chunk.st + c0);   // the same 64 bytes for the whole warp
+#pragma unroll
+                    for (int g = 0; g < 4; ++g) {
+                        const uint4 v4 = row[g];
+                        const __nv_bfloat162* h2 = reinterpret_cast<const __nv_bfloat162*>(&v4);
+#pragma unroll
+                        for (int e = 0; e < 4; ++e) {
+                            const float2 f = __bfloat1622float2(h2[e]);
+                            acc[8 * g + 2 * e] = fmaf(w, f.x, acc[8 * g + 2 * e]);
+                            acc[8 * g + 2 * e + 1] = fmaf(w, f.y, acc[8 * g + 2 * e + 1]);
+                        }
+                    }
+                }
+            }
+            uint8_t* orow = x_ptr + (x * 2 + mat) * kPairOutTile + rl * kPairOutRow + c0 * 2;
+#pragma unroll
+            for (int e = 0; e < 32; e += 8)
+                *reinterpret_cast<uint4*>(orow + e * 2) =
+                    make_uint4(pack_bf16(acc[e] * inv, acc[e + 1] * inv), pack_bf16(acc[e + 2] * inv, acc[e + 3] * inv),
+                               pack_bf16(acc[e + 4] * inv, acc[e + 5] * inv), pack_bf16(acc[e + 6] * inv, acc[e + 7] * inv));
+        }
+    }
+    __syncthreads();
+#pragma unroll 1
+    for (int x = 0; x < nu; ++x) {
+        const int u = units[x], n = u / p.heads, h = u % p.heads;
+#pragma unroll 1
+        for (int mat = 0; mat < 2; ++mat) {
+            const View& out = mat ? p.v_out : p.k_out;
+            __nv_bfloat16* obase = unit_base_mut<__nv_bfloat16>(out, n, h);
+            const uint8_t* tile = x_ptr + (x * 2 + mat) * kPairOutTile;
+            for (int idx = tid; idx < kSlots * 16; idx += kThreads) {
+                const int row = idx >> 4, piece16 = idx & 15;
+                *reinterpret_cast<uint4*>(obase + (int64_t)row * out.st + piece16 * 8) =
+                    *reinterpret_cast<const uint4*>(tile + row * kPairOutRow + piece16 * 16);
+            }
+        }
+    }
+    tc_fence_before();
+    __syncthreads();
+    if (tid == 128) {
+        for (int s = 0; s < 2 * kPairStages + 3; ++s) mbar_inval(bar_full + 8 * s);
     }
 }
 
@@ -916,6 +1260,113 @@ __global__ void __launch_bounds__(kAttnThreads, 1) attention_tc_kernel(const __g
     cta_tmem_release(tmem);
 }
 
+// Eq. 1 for a chunk of ONE query (the generation stage) on the CUDA cores: a 128-row MMA tile would hold one live row.
+// The step is a chain of memory latencies and every CTA runs this code exactly once, so it is written for few
+// round trips and few instructions (short rolled loops: straight-line code that runs once costs its own fetch):
+// the work of a unit is spread over four warps, a quarter of the keys each; a warp brings its key and value rows
+// into shared memory with one burst of 16-byte async copies, then scores and accumulates from there. A lane owns
+// four channels; the four warps' (maximum, sum, output) triples meet in shared memory.
+constexpr int kDecodeWarpsPerUnit = 4;
+constexpr int kDecodeUnitsPerCta = kThreads / 32 / kDecodeWarpsPerUnit;
+constexpr int kDecodeRows = 33;                                        // keys per warp
+constexpr int kDecodeMaxKeys = kDecodeRows * kDecodeWarpsPerUnit;      // 132: a cache of 128 slots and the query's own key
+
+__device__ __forceinline__ void decode_attention_body(const TcAttnParams& P, uint8_t* smem, int first_unit) {
+    const AttnParams& p = P.base;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int u = first_unit + warp / kDecodeWarpsPerUnit, part = warp % kDecodeWarpsPerUnit;
+    const bool live = u < p.units;
+    const int n = live ? u / p.heads : 0, h = live ? u % p.heads : 0;
+    const int S = p.c + 1;
+    const int per = (S + kDecodeWarpsPerUnit - 1) / kDecodeWarpsPerUnit;
+    const int j_begin = part * per, j_end = live ? min(S, j_begin + per) : j_begin;   // this warp's keys
+    const int nk = j_end - j_begin;
+    uint8_t* rows = smem + warp * (2 * kDecodeRows * 256);            // [keys: nk rows][values: nk rows at kDecodeRows], 256 bytes each
+    const uint32_t rows_a = smem_u32(rows);
+    float* xch = reinterpret_cast<float*>(smem + (kThreads / 32) * (2 * kDecodeRows * 256));
+    auto f4 = [](uint2 x, float (&o)[4]) {
+        const float2 a = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&x.x));
+        const float2 b = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&x.y));
+        o[0] = a.x; o[1] = a.y; o[2] = b.x; o[3] = b.y;
+    };
+    float q[4];
+    f4(live ? *reinterpret_cast<const uint2*>(unit_base<__nv_bfloat16>(p.q, n, h) + 4 * lane) : make_uint2(0u, 0u), q);
+    wait_for_earlier_kernels();          // the cache rows are the previous step's result
+    {
+        // 16 lanes per row, two rows per instruction; rows of the cache, then (the last key) the chunk's row
+        const __nv_bfloat16* kc = unit_base<__nv_bfloat16>(p.xk.cache, n, h) + 8 * (lane & 15);
+        const __nv_bfloat16* vc = unit_base<__nv_bfloat16>(p.xv.cache, n, h) + 8 * (lane & 15);
+        const __nv_bfloat16* kn = unit_base<__nv_bfloat16>(p.xk.chunk, n, h) + 8 * (lane & 15);
+        const __nv_bfloat16* vn = unit_base<__nv_bfloat16>(p.xv.chunk, n, h) + 8 * (lane & 15);
+#pragma unroll 1
+        for (int r = lane >> 4; r < nk; r += 2) {
+            const int j = j_begin + r;
+            const uint32_t dst = rows_a + r * 256 + (lane & 15) * 16;
+            cp_async16(dst, j < p.c ? kc + (int64_t)j * p.xk.cache.st : kn, 16u);
+            cp_async16(dst + kDecodeRows * 256, j < p.c ? vc + (int64_t)j * p.xv.cache.st : vn, 16u);
+        }
+        cp_async_wait_all();
+        __syncwarp();
+    }
+    const float sc2 = p.scale * 1.4426950408889634f;
+    // scores: lane l keeps the score of keys l and 32 + l of this warp
+    float s0 = -INFINITY, s1 = -INFINITY;
+#pragma unroll 1
+    for (int r = 0; r < nk; ++r) {
+        float kf[4];
+        f4(*reinterpret_cast<const uint2*>(rows + r * 256 + lane * 8), kf);
+        float d = fmaf(q[0], kf[0], fmaf(q[1], kf[1], fmaf(q[2], kf[2], q[3] * kf[3])));
+#pragma unroll
+        for (int o = 16; o; o >>= 1) d += __shfl_xor_sync(0xffffffffu, d, o);
+        d *= sc2;
+        if ((r & 31) == lane) { if (r < 32) s0 = d; else s1 = d; }
+    }
+    float m_w = fmaxf(s0, s1);
+#pragma unroll
+    for (int o = 16; o; o >>= 1) m_w = fmaxf(m_w, __shfl_xor_sync(0xffffffffu, m_w, o));
+    const float p0 = lane < nk ? exp2f(s0 - m_w) : 0.f, p1 = 32 + lane < nk ? exp2f(s1 - m_w) : 0.f;
+    float l_w = p0 + p1;
+#pragma unroll
+    for (int o = 16; o; o >>= 1) l_w += __shfl_xor_sync(0xffffffffu, l_w, o);
+    float o4[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll 1
+    for (int r = 0; r < nk; ++r) {
+        const float pj = __shfl_sync(0xffffffffu, r < 32 ? p0 : p1, r & 31);
+        float vf[4];
+        f4(*reinterpret_cast<const uint2*>(rows + (kDecodeRows + r) * 256 + lane * 8), vf);
+#pragma unroll
+        for (int e = 0; e < 4; ++e) o4[e] = fmaf(pj, vf[e], o4[e]);
+    }
+    // the four warps of a unit meet: [warp][maximum, sum, -, -, 128 outputs]
+    constexpr int kRec = 4 + kD;
+    float* mine = xch + warp * kRec;
+    if (lane == 0) { mine[0] = nk > 0 ? m_w : -INFINITY; mine[1] = l_w; }
+    *reinterpret_cast<float4*>(mine + 4 + 4 * lane) = make_float4(o4[0], o4[1], o4[2], o4[3]);
+    __syncthreads();
+    if (live && part == 0) {
+        const float* base = xch + (warp / kDecodeWarpsPerUnit) * kDecodeWarpsPerUnit * kRec;
+        float m_all = -INFINITY;
+#pragma unroll
+        for (int w = 0; w < kDecodeWarpsPerUnit; ++w) m_all = fmaxf(m_all, base[w * kRec]);
+        float l_all = 0.f, o[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+        for (int w = 0; w < kDecodeWarpsPerUnit; ++w) {
+            const float* src = base + w * kRec;
+            const float mw = src[0];
+            const float f = mw == -INFINITY ? 0.f : exp2f(mw - m_all);
+            l_all += src[1] * f;
+            const float4 ow = *reinterpret_cast<const float4*>(src + 4 + 4 * lane);
+            o[0] = fmaf(ow.x, f, o[0]); o[1] = fmaf(ow.y, f, o[1]); o[2] = fmaf(ow.z, f, o[2]); o[3] = fmaf(ow.w, f, o[3]);
+        }
+        const float inv = 1.f / l_all;
+        uint2 out;
+        out.x = pack_bf16(o[0] * inv, o[1] * inv);
+        out.y = pack_bf16(o[2] * inv, o[3] * inv);
+        reinterpret_cast<uint2*>(unit_base_mut<__nv_bfloat16>(p.o, n, h))[lane] = out;
+        if (p.lse && lane == 0) p.lse[(int64_t)u * p.lse_stride] = (m_all + log2f(l_all)) * 0.6931471805599453f;
+    }
+}
+
 // ------------------------------------------------------------------ one chunk step, one launch
 // Step 3 (attention with the OLD cache) and Steps 4-5 (the new cache) of Algorithm 2 read the same
 // inputs and do not depend on each other, so their CTAs share one grid: every CTA fills an SM by
@@ -927,6 +1378,7 @@ struct TcStepParams {
     TcAttnParams attn;
     TcCompressParams comp;
     int qtiles, n_attn_first, n_attn, comp_per_unit;   // comp_per_unit = parts * slot_blocks
+    int decode;                                        // 1: chunks of one query, attention by decode_attention_body (a warp per unit)
     // position in the item list of a persistent launch (sequence_tc_kernel)
     int items_per_unit, item_end, finished_target;     // finished_target: items of a unit up to and including this step
 };
@@ -934,16 +1386,21 @@ struct TcStepParams {
 // Work item `idx` of one chunk step, in the order above.
 __device__ __forceinline__ void step_item(const TcStepParams& P, uint8_t* smem, uint32_t tmem, bool cache_cg, int idx) {
     const int units = P.attn.base.units;
-    const int n_comp = units * P.comp_per_unit;
+    const int n_comp = P.comp.pair ? P.comp.pairs : units * P.comp_per_unit;
     if (idx < P.n_attn_first) {
         attention_body(P.attn, P.attn.maps, false, smem, tmem, P.qtiles - 1 - idx / units, idx % units);
     } else if (idx < P.n_attn_first + n_comp) {
         idx -= P.n_attn_first;
-        const int u = idx / P.comp_per_unit, rem = idx % P.comp_per_unit;
-        compress_body<true>(P.comp, smem, tmem, cache_cg, rem % P.comp.parts, rem / P.comp.parts, u);
+        if (P.comp.pair) {
+            compress_pair_body(P.comp, &P.attn.maps[kMapVCache], smem, tmem, idx);
+        } else {
+            const int u = idx / P.comp_per_unit, rem = idx % P.comp_per_unit;
+            compress_body<true>(P.comp, smem, tmem, cache_cg, rem % P.comp.parts, rem / P.comp.parts, u);
+        }
     } else {
         idx -= n_comp;
-        attention_body(P.attn, P.attn.maps, false, smem, tmem, P.qtiles - 1 - idx / units, idx % units);
+        if (P.decode) decode_attention_body(P.attn, smem, (idx - P.n_attn_first) * kDecodeUnitsPerCta);
+        else attention_body(P.attn, P.attn.maps, false, smem, tmem, P.qtiles - 1 - idx / units, idx % units);
     }
 }
 
@@ -1400,7 +1857,26 @@ int tensor_chunk_step(lococo_handle* h, const AttnParams& a, const CompressParam
     P.comp.direct = own_output && P.comp.parts == 1;
     // several CTAs per (unit, slot block): the one that stores the last partial set sums them and writes the rows
     P.comp.merge = own_output && P.comp.parts > 1 && p.R16 == nullptr;
-    const int blocks = P.n_attn + a.units * P.comp_per_unit;
+    // generation stage: chunks so short that a unit's positions are one small tile. Two units per compress CTA share
+    // every weight stage, and a chunk of one query is attended to by a warp instead of a 128-row MMA tile.
+    const int n_tile16 = (p.S + 15) / 16 * 16;
+    if (own_output && p.R16 == nullptr && p.M == kSlots && p.xk.c == kSlots && p.c_in == kD && p.units > 148 && n_tile16 <= 144 &&
+        pair_layout(p.S, n_tile16, p.k).total <= (uint32_t)kMaxSmem && ((P.attn.tma_mask >> kMapVCache) & 1) &&
+        (!p.weights_per_head || p.units / p.heads >= 2)) {
+        P.comp.pair = 1;
+        P.comp.direct = 1;
+        P.comp.merge = 0;
+        P.comp.n_tile = n_tile16;
+        P.comp.tiles = P.comp.parts = P.comp.tiles_per_part = 1;
+        P.comp.pairs = p.weights_per_head ? p.heads * ((p.units / p.heads + 1) / 2) : (p.units + 1) / 2;
+    }
+    int n_attn_ctas = P.n_attn;
+    if (a.b == 1 && a.c + 1 <= kDecodeMaxKeys) {
+        P.decode = 1;
+        P.n_attn_first = 0;
+        n_attn_ctas = (a.units + kDecodeUnitsPerCta - 1) / kDecodeUnitsPerCta;
+    }
+    const int blocks = n_attn_ctas + (P.comp.pair ? P.comp.pairs : a.units * P.comp_per_unit);
     prof_begin(p.prof, 2, st);
     // the step's CTAs read the chunk before they wait for earlier kernels: the first step of a call is therefore
     // launched in plain stream order, after whatever the caller ran before (it may have produced Q, K, V)

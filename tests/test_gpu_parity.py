@@ -113,6 +113,64 @@ def test_generation_mode_chunk_of_one_token(api, orc, path):
     check_sequence(api, orc, w, path)
 
 
+@pytest.mark.parametrize("batch,heads,B,per_head,c_mult,L", [
+    (16, 32, 1, False, 1, 136),     # the generation stage at batch 16: 512 units, 256 two-unit CTAs, 8 steps
+    (5, 32, 1, True, 1, 134),       # a set per head, odd batch: the last pair of every head has one unit
+    (5, 31, 1, False, 1, 134),      # odd number of units with shared weights
+    (5, 32, 4, False, 1, 144),      # chunks of 4 tokens: two-unit compress CTAs, tensor-core attention
+    (5, 32, 16, True, 1, 176),      # chunks of 16: S = 144, the widest tile of the two-unit form
+    (2, 2, 1, False, 1, 140),       # fewer units than SMs: one unit per compress CTA, warp-per-unit attention
+    (5, 32, 1, False, 2, 132),      # keys stacked on values: the one-unit form, warp-per-unit attention
+])
+def test_generation_stage_two_units_per_cta(api, orc, batch, heads, B, per_head, c_mult, L):
+    # Section 3.3: in the generation stage the segment length is 1. Short chunks on a full cache of M = 128 slots run
+    # the compress step with two units per CTA (shared weight stages) and, for one query, attention with a warp per unit.
+    # With random weights and token-by-token steps the slots soon resemble one another and whole rows of logits sit
+    # close to zero, where Eq. 7 is discontinuous (a row with no positive logit is a zero slot, a row with one tiny
+    # positive logit is that token): a positive bias keeps the rows away from that edge, so that the comparison
+    # measures the arithmetic and not the conditioning of the input.
+    w = wl.Workload(f"gen{batch}x{heads}b{B}", 14, batch=batch, heads=heads, d=128, M=128, B=B, k=21, L=L, dtype="bf16",
+                    weights_per_head=per_head, qkv_scale=0.0884, g_std=0.02, c_in_mult=c_mult)
+    G, _ = wl.make_weights(w)
+    bvec = wl.round_to_bf16(np.full((heads if per_head else 1, w.M), 0.05, dtype=np.float32))
+    ctx = api.Lococo(w.batch, w.heads, w.d, w.M, w.k, w.B, dtype=torch.bfloat16, c_in=w.c_in, weights_per_head=per_head)
+    ctx.set_weights(to_device(G, "bf16"), to_device(bvec, "bf16"))
+    Qh, Kh, Vh = wl.make_qkv(w)
+    Q, K, V = (to_device(x, "bf16") for x in (Qh, Kh, Vh))
+    O = torch.empty_like(Q)
+    Kc = torch.zeros(w.batch, w.heads, w.M, w.d, dtype=Q.dtype, device="cuda")
+    Vc = torch.zeros_like(Kc)
+    assert ctx.process_sequence(Q, K, V, w.B, O, Kc, Vc, 0) == w.M
+    torch.cuda.synchronize()
+    assert ctx.device_status() == api.OK
+    Or, Kr, Vr, cr, _ = orc.process_batch(Qh, Kh, Vh, G, w.B, bias=bvec)
+    assert_close(to_host(O), Or, "bf16", f"{w.name} O")
+    assert_close(to_host(Kc), Kr, "bf16", f"{w.name} K cache")
+    assert_close(to_host(Vc), Vr, "bf16", f"{w.name} V cache")
+
+
+def test_generation_stage_bit_identical_across_unit_pairings(api):
+    # a unit's result must not depend on which unit shares its CTA: the same six sequences in another order
+    # (units are paired with their neighbours in the batch)
+    w = wl.Workload("gen_pairs", 15, batch=6, heads=32, d=128, M=128, B=1, k=21, L=134, dtype="bf16",
+                    weights_per_head=False, qkv_scale=0.0884, g_std=0.02)
+    Q, K, V = (to_device(x, w.dtype) for x in wl.make_qkv(w))
+    ctx, _, _ = make_ctx(api, w)
+    outs = []
+    for order in ([0, 1, 2, 3, 4, 5], [3, 0, 5, 1, 4, 2]):
+        q, k, v = (x[order].contiguous() for x in (Q, K, V))
+        O = torch.empty_like(q)
+        Kc = torch.zeros(w.batch, w.heads, w.M, w.d, dtype=q.dtype, device="cuda")
+        Vc = torch.zeros_like(Kc)
+        assert ctx.process_sequence(q, k, v, w.B, O, Kc, Vc, 0) == w.M
+        torch.cuda.synchronize()
+        back = torch.argsort(torch.tensor(order))
+        outs.append((O[back], Kc[back], Vc[back]))
+    assert ctx.device_status() == api.OK
+    for a, b in zip(*outs):
+        assert torch.equal(a, b)
+
+
 @pytest.mark.parametrize("dtype", ["f32", "bf16"])
 def test_ragged_everything(api, orc, dtype):
     # sizes that are multiples of nothing: M=40, B=37, L=301 (last chunk short), k=7,
