@@ -560,7 +560,7 @@ def time_layer_stack(layers=32, runs=3):
             "ms": ms, "ms_per_layer": ms / layers, "tokens_per_s_all_layers": w.batch * w.L / (ms * 1e-3)}
 
 
-def time_generation(batches=(1, 16), steps=256, runs=3):
+def time_generation(batches=(1, 16, 64), steps=256, runs=3):
     """Secondary figure: the generation stage (Section 3.3: chunks of one token on a full cache, every step
     recomputes all M slots from S = M + 1 entries), cfg2's layer shape with the weights shared by the heads,
     `steps` token steps per call after the cache has been filled."""
@@ -594,7 +594,9 @@ def time_generation(batches=(1, 16), steps=256, runs=3):
                 if it >= 2:
                     ms += a.elapsed_time(b) / runs
         assert ctx.device_status() == api.OK
-        res.append({"batch": batch, "us_per_token_step": ms / steps * 1e3, "tokens_per_s": batch * steps / (ms * 1e-3)})
+        step_flops = batch * w.heads * (conv_flops(w.M + 1, w.M, w.c_in, w.k) + blend_flops(w.M + 1, w.M, w.d) + attn_flops(1, w.M, w.d))
+        res.append({"batch": batch, "us_per_token_step": ms / steps * 1e3, "tokens_per_s": batch * steps / (ms * 1e-3),
+                    "tflops": step_flops / (ms / steps * 1e-3) / 1e12})
     return {"workload": f"chunks of one token on a full cache, {base.heads} heads, d={base.d}, M={base.M}, k={base.k}, "
                         f"shared conv weights, {steps} token steps per call", "runs": res}
 

@@ -221,6 +221,7 @@ __device__ __forceinline__ void compress_body(const TcCompressParams& P, uint8_t
     const int tile_begin = part * P.tiles_per_part;
     const int tile_end = min(P.tiles, tile_begin + P.tiles_per_part);
     int tile_it = 0;
+#pragma unroll 1
     for (int tile = tile_begin; tile < tile_end; ++tile, ++tile_it) {
         const int j0 = tile * n_tile;
         // The weight producer (one thread of warp 5) runs ahead of everything else: a tile's
@@ -283,6 +284,7 @@ __device__ __forceinline__ void compress_body(const TcCompressParams& P, uint8_t
             const uint32_t bstep = (2 * lbo_z) >> 4;
             // stage index and phase, tap and channel half are tracked incrementally: no division here
             uint32_t st = g % NS, ph = (g / NS) & 1, tap = 0, half = 0;
+#pragma unroll 1
             for (int it = 0; it < total; ++it) {
                 mbar_wait(bar_full + 8 * st, ph, P.status, failed, 2);
                 tc_fence_after();
@@ -310,6 +312,7 @@ __device__ __forceinline__ void compress_body(const TcCompressParams& P, uint8_t
             const uint32_t lane_addr = tmem + ((uint32_t)((warp & 3) * 32) << 16);
             float* rstore = P.R_store ? P.R_store + ((int64_t)u * p.M + slot) * p.S : nullptr;
             const bool keep = slot < p.prot;
+#pragma unroll 1
             for (int c0 = eg * 32; c0 < n_tile; c0 += 96) {
                 uint32_t v[32];
                 tmem_ld32(lane_addr + c0, v);
@@ -346,6 +349,7 @@ __device__ __forceinline__ void compress_body(const TcCompressParams& P, uint8_t
         // ---- 4. Eq. 4, Eq. 5 (unnormalised): U_K += R X_K, U_V += R X_V from the staged tiles
         if (tid == 128) {
             tc_fence_after();
+#pragma unroll 1
             for (int kk = 0; kk < n_tile / 16; ++kk) {
                 const uint64_t ad = smem_desc(ring + kk * 2 * 2048, 2048, 128);
                 const uint32_t row0 = (uint32_t)(pad + kk * 16) * 16;
@@ -1059,21 +1063,18 @@ __device__ __forceinline__ void attention_body(const TcAttnParams& P, const CUte
             copy_rows(qs, safe + (int64_t)r0 * p.q.st, p.q.st, p.b - r0);
             announce_copied(q_full);
         }
-        load_kv(0, 0, 0);
-        load_kv(0, 0, 1);
-        if (ntiles > 1) {
-            load_kv(1, 1, 0);
-            load_kv(1, 1, 1);
-        }
-        // Tile t (>= 2) goes into the buffers of tile t-2: its keys as soon as S(t-2) has read the key
-        // buffer, its values as soon as PV(t-2) has read the value buffer. A tile is announced (or left
-        // to the engine to announce) before this warp waits for the next buffer.
-        for (int t = 2; t < ntiles; ++t) {
+        // Tiles 0 and 1 go straight into the two buffers. Tile t (>= 2) goes into the buffers of tile t-2: its keys as
+        // soon as S(t-2) has read the key buffer, its values as soon as PV(t-2) has read the value buffer. A tile is
+        // announced (or left to the engine to announce) before this warp waits for the next buffer. (One call site
+        // for all tiles: the loader's code is inlined where it is called, and there is a lot of it.)
+#pragma unroll 1
+        for (int t = 0; t < ntiles; ++t) {
             const int b = t & 1, ph = ((t - 2) >> 1) & 1;
-            mbar_wait(s_full(b), ph, P.status, failed, 4);
-            load_kv(t, b, 0);
-            mbar_wait(pv_done(b), ph, P.status, failed, 5);
-            load_kv(t, b, 1);
+#pragma unroll 1
+            for (int which = 0; which < 2; ++which) {
+                if (t >= 2) mbar_wait(which ? pv_done(b) : s_full(b), ph, P.status, failed, 4 + which);
+                load_kv(t, b, which);
+            }
         }
         if (cache_tiles == 0) wait_for_earlier_kernels();   // keeps the chain of waits unbroken
     } else if (tid == kMma) {
@@ -1095,6 +1096,7 @@ __device__ __forceinline__ void attention_body(const TcAttnParams& P, const CUte
             umma_commit(pv_done(b));
         };
         mbar_wait(q_full, 0, P.status, failed, 7);
+#pragma unroll 1
         for (int jt = 0; jt < ntiles; ++jt) {
             const int b = jt & 1;
             mbar_wait(k_full(b), (jt >> 1) & 1, P.status, failed, 7);
@@ -1121,6 +1123,7 @@ __device__ __forceinline__ void attention_body(const TcAttnParams& P, const CUte
         // the two threads of a row exchange their maxima rounded to bf16, one slot per tile parity:
         // both then derive the same reference maximum, which only has to be near the true one
         __nv_bfloat16* xmax = reinterpret_cast<__nv_bfloat16*>(xchg);   // [2 parities][2 halves][128 rows]
+#pragma unroll 1
         for (int jt = 0; jt < ntiles; ++jt) {
             const int b = jt & 1;
             mbar_wait(s_full(b), (jt >> 1) & 1, P.status, failed, 9);
@@ -1181,6 +1184,7 @@ __device__ __forceinline__ void attention_body(const TcAttnParams& P, const CUte
                         if (!need_mask || j0 + c0 + e < vis) tmax = fmaxf(tmax, __uint_as_float(v[e]));
                 }
             };
+#pragma unroll 1
             for (int attempt = 0; attempt < 2; ++attempt) {
                 float tmax = -INFINITY;
                 if (jt == 0 && attempt == 0) max_only(tmax);
@@ -1383,13 +1387,13 @@ struct TcStepParams {
     int items_per_unit, item_end, finished_target;     // finished_target: items of a unit up to and including this step
 };
 
-// Work item `idx` of one chunk step, in the order above.
+// Work item `idx` of one chunk step, in the order above. (Each body appears once: the kernel's code is several times the
+// size of an SM's instruction cache as it is, and code that has to be fetched is time the CTA spends waiting.)
 __device__ __forceinline__ void step_item(const TcStepParams& P, uint8_t* smem, uint32_t tmem, bool cache_cg, int idx) {
     const int units = P.attn.base.units;
     const int n_comp = P.comp.pair ? P.comp.pairs : units * P.comp_per_unit;
-    if (idx < P.n_attn_first) {
-        attention_body(P.attn, P.attn.maps, false, smem, tmem, P.qtiles - 1 - idx / units, idx % units);
-    } else if (idx < P.n_attn_first + n_comp) {
+    const bool is_comp = idx >= P.n_attn_first && idx < P.n_attn_first + n_comp;
+    if (is_comp) {
         idx -= P.n_attn_first;
         if (P.comp.pair) {
             compress_pair_body(P.comp, &P.attn.maps[kMapVCache], smem, tmem, idx);
@@ -1398,8 +1402,8 @@ __device__ __forceinline__ void step_item(const TcStepParams& P, uint8_t* smem, 
             compress_body<true>(P.comp, smem, tmem, cache_cg, rem % P.comp.parts, rem / P.comp.parts, u);
         }
     } else {
-        idx -= n_comp;
-        if (P.decode) decode_attention_body(P.attn, smem, (idx - P.n_attn_first) * kDecodeUnitsPerCta);
+        if (idx >= P.n_attn_first) idx -= n_comp;       // the attention items after the compress CTAs continue the first ones' numbering
+        if (P.decode) decode_attention_body(P.attn, smem, idx * kDecodeUnitsPerCta);
         else attention_body(P.attn, P.attn.maps, false, smem, tmem, P.qtiles - 1 - idx / units, idx % units);
     }
 }
