@@ -198,6 +198,239 @@ gemm::Params base_params(lococo_handle* h) {
     return P;
 }
 
+
+// ------------------------------------------------------------------ Eq. 1 reversed, keys' side, fused
+// One CTA owns a tile of 128 keys of one unit and walks over the tiles of 64 queries that can see it. Per query tile:
+//   S^T = X_K Q^T and dP^T = X_V dO^T           (keys on the TMEM lanes, queries on the columns)
+//   P^T = exp(scale S^T - lse), dS^T = scale P^T (dP^T - delta), under the causal mask, in registers (P in fp32);
+//         both go to shared memory in bf16 as MMA A operands, dS^T also to global memory for dQ = dS X_K
+//   dX_V += P^T dO, dX_K += dS^T Q                accumulated in TMEM over all query tiles, added to memory at the end
+// so P never reaches memory and dS is written once. Three roles meet at mbarriers: one lane drives the tensor copy
+// engine (keys and values once, then Q / dO tiles through two stages), one lane issues the MMAs (the score products of
+// tile t+1 are queued behind the gradient products of tile t), eight warps turn scores into P^T and dS^T.
+// TMEM: S^T x2 (64 columns each), dP^T x2, dX_V, dX_K (128 each) = 512 columns.
+namespace fused {
+
+using namespace tc;
+
+constexpr int kThreads = 320;
+constexpr uint32_t kKvTile = 32768;       // 128 rows x 128 channels: two 64-channel halves of 16 KB (128-byte swizzle)
+constexpr uint32_t kQTile = 16384;        // 64 rows x 128 channels: two halves of 8 KB
+constexpr uint32_t kPTile = 16384;        // 128 keys x 64 queries, bf16: [8-query group][128 rows][8 queries]
+constexpr uint32_t kSmem = 2 * kKvTile + 2 * 2 * kQTile + 2 * 2 * kPTile + 2 * 128 * 4 + 256 + 1024;
+
+struct alignas(64) Params {
+    CUtensorMap map_x;            // packed [unit][pad + position][K 128 | V 128], boxes of 128 rows x 64 channels
+    CUtensorMap map_q, map_do;    // [batch, heads, tokens, 128] views, boxes of 64 rows x 64 channels
+    const float* lse;             // log-sum-exp of the forward, first query of the block; lse_z: unit stride
+    const float* delta;           // <dO, O> per query, first query of the block
+    int64_t lse_z, delta_z;
+    __nv_bfloat16* ds_t;          // dS^T [unit][key][query of the block], row stride ds_row, unit stride ds_z
+    int64_t ds_z;
+    int ds_row;
+    float* dXK;                   // [unit][S][128] fp32, += ; dXV likewise
+    float* dXV;
+    int heads, S, c, pad;
+    int q0, qb, b;                // first query of the block, queries in the block, chunk length
+    float scale, scale2;          // softmax scale, and scale * log2 e
+    int* status;
+};
+
+__global__ void __launch_bounds__(kThreads, 1) attn_bwd_kv_kernel(const __grid_constant__ Params P) {
+    extern __shared__ __align__(128) uint8_t smem_raw[];
+    __shared__ uint32_t tmem_slot;
+    uint8_t* smem = smem_raw + ((1024u - (smem_u32(smem_raw) & 1023u)) & 1023u);
+    uint8_t* k_ptr = smem;
+    uint8_t* v_ptr = k_ptr + kKvTile;
+    uint8_t* qd_ptr = v_ptr + kKvTile;                 // stage x: [Q | dO]
+    uint8_t* p_ptr = qd_ptr + 2 * 2 * kQTile;          // buffer x: [P^T | dS^T]
+    float* vec = reinterpret_cast<float*>(p_ptr + 2 * 2 * kPTile);   // buffer x: [64 lse * log2 e | 64 delta]
+    uint64_t* bars = reinterpret_cast<uint64_t*>(vec + 2 * 128);
+    volatile int* failed = reinterpret_cast<volatile int*>(bars + 12);
+    const uint32_t ks = smem_u32(k_ptr), vs = smem_u32(v_ptr), qds = smem_u32(qd_ptr), ps = smem_u32(p_ptr);
+    const uint32_t bar0 = smem_u32(bars);
+    auto qd_full = [&](int x) { return bar0 + 8 * x; };          // loader -> MMA: Q, dO tile staged
+    auto s_full = [&](int x) { return bar0 + 16 + 8 * x; };      // MMA -> warps: S^T, dP^T in TMEM
+    auto s_free = [&](int x) { return bar0 + 32 + 8 * x; };      // warps -> MMA: S^T, dP^T read
+    auto p_full = [&](int x) { return bar0 + 48 + 8 * x; };      // warps -> MMA: P^T, dS^T written
+    auto g_done = [&](int x) { return bar0 + 64 + 8 * x; };      // MMA -> loader, warps: gradient products done
+    const uint32_t kv_full = bar0 + 80, acc_done = bar0 + 88;
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int jt = blockIdx.x, u = blockIdx.y;
+    const int n = u / P.heads, h = u % P.heads;
+    const int j0 = jt * 128;
+
+    if (tid == 256) {
+        for (int x = 0; x < 2; ++x) {
+            mbar_init(qd_full(x), 1);
+            mbar_init(s_full(x), 1);
+            mbar_init(s_free(x), 256);
+            mbar_init(p_full(x), 256);
+            mbar_init(g_done(x), 1);
+        }
+        mbar_init(kv_full, 1);
+        mbar_init(acc_done, 1);
+        *failed = 0;
+        fence_barrier_init();
+    }
+    if (warp == 0) {
+        tmem_alloc(smem_u32(&tmem_slot), 512);
+        tmem_relinquish();
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem = *reinterpret_cast<volatile uint32_t*>(&tmem_slot);
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+
+    // query tiles (64 rows) of the block that see a key of this tile; whole pairs of tiles, because dQ = dS X_K works in
+    // tiles of 128 queries and reads what is written here, zeros included
+    const int T = (P.qb + 63) / 64;
+    const int first = 2 * (max(0, j0 - P.c - P.q0) / 128);
+    const bool any = first < T && j0 < P.S;
+
+    if (tid == 288 && any) {
+        // ---------------- loader
+        mbar_expect_tx(kv_full, 2 * kKvTile);
+        for (int x = 0; x < 4; ++x)      // K channels 0-63, 64-127, V channels 0-63, 64-127
+            tma_load_4d(ks + x * (kKvTile / 2), &P.map_x, 64 * x, P.pad + j0, u, 0, kv_full);
+#pragma unroll 1
+        for (int t = first; t < T; ++t) {
+            const int x = (t - first) & 1, use = (t - first) >> 1;
+            if (use >= 1) mbar_wait(g_done(x), (use - 1) & 1, P.status, failed, 40);
+            mbar_expect_tx(qd_full(x), 2 * kQTile);
+            const uint32_t dst = qds + x * 2 * kQTile;
+            const int row = P.q0 + 64 * t;
+            tma_load_4d(dst, &P.map_q, 0, row, h, n, qd_full(x));
+            tma_load_4d(dst + kQTile / 2, &P.map_q, 64, row, h, n, qd_full(x));
+            tma_load_4d(dst + kQTile, &P.map_do, 0, row, h, n, qd_full(x));
+            tma_load_4d(dst + kQTile + kQTile / 2, &P.map_do, 64, row, h, n, qd_full(x));
+        }
+    } else if (tid == 256 && any) {
+        // ---------------- MMA issuer
+        const uint32_t idesc_s = instr_desc_bf16(64, false, false);
+        const uint32_t idesc_g = instr_desc_bf16(128, false, true);
+        const uint64_t ka = smem_desc_sw128(ks, 16, 1024), va = smem_desc_sw128(vs, 16, 1024);
+        auto kstep = [](int kk, uint32_t half_bytes) { return (uint64_t)(((kk >> 2) * half_bytes + (kk & 3) * 32u) >> 4); };
+        auto issue_grad = [&](int t) {
+            const int x = (t - first) & 1, use = (t - first) >> 1;
+            mbar_wait(p_full(x), use & 1, P.status, failed, 41);
+            tc_fence_after();
+            const uint32_t q_addr = qds + x * 2 * kQTile, pt = ps + x * 2 * kPTile;
+            const uint64_t pa = smem_desc(pt, 2048, 128), da = smem_desc(pt + kPTile, 2048, 128);
+            const uint64_t qb_mn = smem_desc_sw128(q_addr, kQTile / 2, 1024), dob_mn = smem_desc_sw128(q_addr + kQTile, kQTile / 2, 1024);
+#pragma unroll
+            for (int kk = 0; kk < 4; ++kk) {       // 16 queries per step: two 8-query groups of the A operand, two 8-row groups of the B operand
+                umma_ss(tmem + 256, pa + kk * 256u, dob_mn + kk * 128u, idesc_g, (t != first || kk != 0));
+                umma_ss(tmem + 384, da + kk * 256u, qb_mn + kk * 128u, idesc_g, (t != first || kk != 0));
+            }
+            umma_commit(g_done(x));
+        };
+        mbar_wait(kv_full, 0, P.status, failed, 42);
+#pragma unroll 1
+        for (int t = first; t < T; ++t) {
+            const int x = (t - first) & 1, use = (t - first) >> 1;
+            mbar_wait(qd_full(x), use & 1, P.status, failed, 43);
+            if (use >= 1) mbar_wait(s_free(x), (use - 1) & 1, P.status, failed, 44);
+            tc_fence_after();
+            const uint32_t q_addr = qds + x * 2 * kQTile;
+            const uint64_t qk = smem_desc_sw128(q_addr, 16, 1024), dok = smem_desc_sw128(q_addr + kQTile, 16, 1024);
+#pragma unroll
+            for (int kk = 0; kk < 8; ++kk) umma_ss(tmem + x * 64, ka + kstep(kk, kKvTile / 2), qk + kstep(kk, kQTile / 2), idesc_s, kk != 0);
+#pragma unroll
+            for (int kk = 0; kk < 8; ++kk) umma_ss(tmem + 128 + x * 64, va + kstep(kk, kKvTile / 2), dok + kstep(kk, kQTile / 2), idesc_s, kk != 0);
+            umma_commit(s_full(x));
+            if (t > first) issue_grad(t - 1);
+        }
+        issue_grad(T - 1);
+        umma_commit(acc_done);
+    }
+    if (warp < 8 && any) {
+        // ---------------- P^T and dS^T: a thread owns one key (TMEM lane) and 32 of the tile's 64 queries
+        const int rl = (warp & 3) * 32 + lane, half = warp >> 2;
+        const int j = j0 + rl;
+        const uint32_t lane_base = tmem + ((uint32_t)((warp & 3) * 32) << 16);
+        __nv_bfloat16* ds_row = P.ds_t + (int64_t)u * P.ds_z + (int64_t)j * P.ds_row;
+#pragma unroll 1
+        for (int t = first; t < T; ++t) {
+            const int x = (t - first) & 1, use = (t - first) >> 1;
+            float* vb = vec + x * 128;
+            if (tid < 128) {
+                const int q = 64 * t + (tid & 63);                   // query within the block
+                const bool ok = q < P.qb;
+                vb[tid] = tid < 64 ? (ok ? P.lse[(int64_t)u * P.lse_z + q] * 1.4426950408889634f : 0.f)
+                                   : (ok ? P.delta[(int64_t)u * P.delta_z + q] : 0.f);
+            }
+            asm volatile("bar.sync 1, 256;" ::: "memory");
+            mbar_wait(s_full(x), use & 1, P.status, failed, 45);
+            tc_fence_after();
+            uint32_t sv[32], dv[32];
+            tmem_ld32(lane_base + x * 64 + half * 32, sv);
+            tmem_ld32(lane_base + 128 + x * 64 + half * 32, dv);
+            tmem_ld_wait();
+            tc_fence_before();
+            mbar_arrive(s_free(x));
+            if (use >= 1) mbar_wait(g_done(x), (use - 1) & 1, P.status, failed, 46);      // the P^T, dS^T buffer is free again
+            const int qc0 = 64 * t + half * 32;                      // first of this thread's queries, within the block
+            // key j is seen by query r of the chunk when j < c + r + 1
+            const int lim = j - P.c - P.q0;                          // visible: query (within the block) >= lim
+            uint8_t* pdst = p_ptr + x * 2 * kPTile + rl * 16;
+#pragma unroll
+            for (int e = 0; e < 32; e += 8) {
+                uint32_t pk[4], dk[4];
+#pragma unroll
+                for (int y = 0; y < 8; y += 2) {
+                    const int qa = qc0 + e + y;
+                    const bool on0 = j < P.S && qa < P.qb && qa >= lim, on1 = j < P.S && qa + 1 < P.qb && qa + 1 >= lim;
+                    const float p0 = on0 ? exp2f(__uint_as_float(sv[e + y]) * P.scale2 - vb[half * 32 + e + y]) : 0.f;
+                    const float p1 = on1 ? exp2f(__uint_as_float(sv[e + y + 1]) * P.scale2 - vb[half * 32 + e + y + 1]) : 0.f;
+                    const float d0 = p0 * (__uint_as_float(dv[e + y]) - vb[64 + half * 32 + e + y]) * P.scale;
+                    const float d1 = p1 * (__uint_as_float(dv[e + y + 1]) - vb[64 + half * 32 + e + y + 1]) * P.scale;
+                    pk[y >> 1] = pack_bf16(p0, p1);
+                    dk[y >> 1] = pack_bf16(on0 ? d0 : 0.f, on1 ? d1 : 0.f);
+                }
+                const uint32_t g = (uint32_t)((half * 32 + e) >> 3) * 2048u;
+                *reinterpret_cast<uint4*>(pdst + g) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
+                *reinterpret_cast<uint4*>(pdst + kPTile + g) = make_uint4(dk[0], dk[1], dk[2], dk[3]);
+                if (j < P.S) *reinterpret_cast<uint4*>(ds_row + qc0 + e) = make_uint4(dk[0], dk[1], dk[2], dk[3]);
+            }
+            fence_proxy_async();
+            mbar_arrive(p_full(x));
+        }
+        // ---------------- the accumulated key and value gradients of this tile
+        mbar_wait(acc_done, 0, P.status, failed, 47);
+        tc_fence_after();
+        {
+            const bool row_live = j < P.S;
+            float* ok = P.dXK + ((int64_t)u * P.S + (row_live ? j : 0)) * kD + half * 64;
+            float* ov = P.dXV + ((int64_t)u * P.S + (row_live ? j : 0)) * kD + half * 64;
+#pragma unroll 1
+            for (int piece = 0; piece < 4; ++piece) {
+                const int mat = piece >> 1, c0 = (piece & 1) * 32;
+                uint32_t a[32];
+                tmem_ld32(lane_base + (mat ? 384 : 256) + half * 64 + c0, a);     // (the whole warp, whatever its rows)
+                tmem_ld_wait();
+                if (row_live) {
+                    float4* dst = reinterpret_cast<float4*>((mat ? ok : ov) + c0);
+#pragma unroll
+                    for (int e = 0; e < 8; ++e) {
+                        float4 cur = dst[e];
+                        cur.x += __uint_as_float(a[4 * e]); cur.y += __uint_as_float(a[4 * e + 1]);
+                        cur.z += __uint_as_float(a[4 * e + 2]); cur.w += __uint_as_float(a[4 * e + 3]);
+                        dst[e] = cur;
+                    }
+                }
+            }
+        }
+    }
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 0) tmem_dealloc(tmem, 512);
+}
+
+}  // namespace fused
+
 }  // namespace
 
 bool tensor_backward_supported(const lococo_handle* h) {
@@ -341,60 +574,62 @@ int tensor_backward_attention(lococo_handle* h, const BwdStep& p, int B, char* s
     const int U = p.units, H = p.heads, batch = U / H, S = p.S, pad = (p.k - 1) / 2;
     __nv_bfloat16* xpad = reinterpret_cast<__nv_bfloat16*>(sc + L.xpad);
     __nv_bfloat16* pb = reinterpret_cast<__nv_bfloat16*>(sc + L.pb);
-    __nv_bfloat16* dsb = reinterpret_cast<__nv_bfloat16*>(sc + L.dsb);
     const Tensor4 t_xpad{xpad, {256, (uint64_t)L.Sp2, (uint64_t)U, 1}, {512, (uint64_t)L.Sp2 * 512, (uint64_t)U * L.Sp2 * 512}};
     const Tensor4 t_q = of_view(p.q, p.b, H, batch), t_do = of_view(p.d_o, p.b, H, batch);
     const int s_tiles = (S + 127) / 128;
     int n = 0;
-    for (int q0 = 0; q0 < p.b; q0 += L.QB) {
-        const int qb = std::min(L.QB, p.b - q0), q_tiles = (qb + 127) / 128;
+    // blocks of queries: the buffer of dS^T (the former P and dS buffers together) holds 2 * QB queries
+    const int QBf = 2 * L.QB;
+    if (L.dsb <= L.pb || L.total - L.pb < (size_t)U * QBf * L.Sp * 2) return -1;   // the two regions follow each other
+    __nv_bfloat16* dst_t = pb;                               // [unit][key][query of the block]
+    static bool attr_set[64] = {};
+    {
+        int dev = -1;
+        if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return -1;
+        if (!attr_set[dev]) {
+            if (cudaFuncSetAttribute(fused::attn_bwd_kv_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, fused::kSmem) != cudaSuccess) return -1;
+            attr_set[dev] = true;
+        }
+    }
+    for (int q0 = 0; q0 < p.b; q0 += QBf) {
+        const int qb = std::min(QBf, p.b - q0), q_tiles = (qb + 127) / 128;
         const int Sv = std::min(S, p.c + q0 + qb);          // keys any query of the block can see
         const int sv_tiles = (Sv + 127) / 128;
-        // P = exp(scale Q X_K^T - lse) and dS = scale P (dO X_V^T - delta): ONE launch computes both products
-        // of a tile into two accumulators and applies the softmax and its gradient to them, under the causal
-        // mask; only bf16 P and dS reach memory
-        {
-            gemm::Params G = base_params(h);
-            if (!operand(G.A, t_q, false) || !operand(G.B, t_xpad, false) || !operand(G.A2, t_do, false) || !operand(G.B2, t_xpad, false))
+        {   // keys' side, fused: dX_V += P^T dO, dX_K += dS^T Q, and dS^T for the queries' side
+            fused::Params F{};
+            gemm::Operand ox, oq, od;
+            if (!operand(ox, t_xpad, false) || !operand(oq, t_q, true) || !operand(od, t_do, true)) return -1;
+            F.map_x = ox.map; F.map_q = oq.map; F.map_do = od.map;
+            F.lse = p.lse + q0; F.lse_z = p.lse_stride;
+            F.delta = p.delta + q0; F.delta_z = p.b;
+            F.ds_t = dst_t; F.ds_z = (int64_t)L.Sp * QBf; F.ds_row = QBf;
+            F.dXK = p.dXK; F.dXV = p.dXV;
+            F.heads = H; F.S = S; F.c = p.c; F.pad = pad;
+            F.q0 = q0; F.qb = qb; F.b = p.b;
+            F.scale = p.scale; F.scale2 = p.scale * 1.4426950408889634f;
+            F.status = reinterpret_cast<int*>(h->ws + h->off_status);
+            cudaLaunchConfig_t cfg{};
+            cfg.gridDim = dim3(sv_tiles, U);
+            cfg.blockDim = dim3(fused::kThreads);
+            cfg.dynamicSmemBytes = fused::kSmem;
+            cfg.stream = st;
+            cudaLaunchAttribute attr[1];
+            attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+            attr[0].val.programmaticStreamSerializationAllowed = 1;
+            cfg.attrs = attr;
+            cfg.numAttrs = 1;
+            if (cudaLaunchKernelEx(&cfg, fused::attn_bwd_kv_kernel, F) != cudaSuccess) {
+                cudaGetLastError();
                 return -1;
-            G.z_inner = H;
-            for (int which = 0; which < 2; ++which) {
-                gemm::Operand& A = which ? G.A2 : G.A;
-                gemm::Operand& Bo = which ? G.B2 : G.B;
-                A.c[0].si = 64; A.c[1].c0 = q0; A.c[1].tm = 128; A.c[2].zi = 1; A.c[3].zo = 1;
-                Bo.c[0].c0 = which * kD; Bo.c[0].si = 64; Bo.c[1].c0 = pad; Bo.c[1].tni = 128; Bo.c[2].zi = 1; Bo.c[2].zo = H;
             }
-            G.steps = 2;
-            G.out = pb; G.out2 = dsb;
-            G.out_zi = (int64_t)L.QB * L.Sp; G.out_zo = (int64_t)H * L.QB * L.Sp; G.out_m = L.Sp;
-            G.M = qb; G.N = Sv;
-            G.causal_tiles = 1; G.causal_c = p.c + q0;
-            G.mode = gemm::kPairBF16; G.alpha = p.scale; G.scale2 = p.scale * 1.4426950408889634f;
-            G.rowvec = p.lse + q0; G.rowvec_z = p.lse_stride;
-            G.rowvec2 = p.delta + q0; G.rowvec2_z = p.b;
-            if (!gemm::launch(G, q_tiles, sv_tiles, U, st)) return -1;
             ++n;
         }
-        const Tensor4 t_pb{pb, {(uint64_t)Sv, (uint64_t)qb, (uint64_t)U, 1}, {(uint64_t)L.Sp * 2, (uint64_t)L.QB * L.Sp * 2, (uint64_t)U * L.QB * L.Sp * 2}};
-        const Tensor4 t_dsb{dsb, {(uint64_t)Sv, (uint64_t)qb, (uint64_t)U, 1}, {(uint64_t)L.Sp * 2, (uint64_t)L.QB * L.Sp * 2, (uint64_t)U * L.QB * L.Sp * 2}};
-        for (int which = 0; which < 2; ++which) {           // dX_V += P^T dO, dX_K += dS^T Q
+        {   // queries' side: dQ = dS X_K, with dS read as stored (keys along rows)
             gemm::Params G = base_params(h);
-            if (!operand(G.A, which ? t_dsb : t_pb, true) || !operand(G.B, which ? t_q : t_do, true)) return -1;
+            const Tensor4 t_dst{dst_t, {(uint64_t)qb, (uint64_t)Sv, (uint64_t)U, 1}, {(uint64_t)QBf * 2, (uint64_t)L.Sp * QBf * 2, (uint64_t)U * L.Sp * QBf * 2}};
+            if (!operand(G.A, t_dst, true) || !operand(G.B, t_xpad, true)) return -1;
             G.z_inner = H;
             G.A.c[0].tm = 128; G.A.c[1].si = 64; G.A.c[2].zi = 1; G.A.c[2].zo = H;
-            G.B.c[0].tni = 128; G.B.c[1].c0 = q0; G.B.c[1].si = 64; G.B.c[2].zi = 1; G.B.c[3].zo = 1;
-            G.steps = (qb + 63) / 64;
-            G.k_lo_on = 1; G.k_lo_c0 = -(p.c + q0);          // query rows that cannot see this key tile contribute nothing
-            G.out = which ? p.dXK : p.dXV; G.out_zi = (int64_t)S * kD; G.out_zo = (int64_t)H * S * kD; G.out_m = kD;
-            G.M = Sv; G.N = kD; G.mode = gemm::kAddF32;
-            if (!gemm::launch(G, sv_tiles, 1, U, st)) return -1;
-            ++n;
-        }
-        {   // dQ = dS X_K
-            gemm::Params G = base_params(h);
-            if (!operand(G.A, t_dsb, false) || !operand(G.B, t_xpad, true)) return -1;
-            G.z_inner = H;
-            G.A.c[0].si = 64; G.A.c[1].tm = 128; G.A.c[2].zi = 1; G.A.c[2].zo = H;
             G.B.c[0].tni = 128; G.B.c[1].c0 = pad; G.B.c[1].si = 64; G.B.c[2].zi = 1; G.B.c[2].zo = H;
             G.steps = (Sv + 63) / 64;
             G.k_hi_on = 1; G.k_hi_c0 = p.c + q0 + 128;       // keys beyond the last query of the tile are masked
