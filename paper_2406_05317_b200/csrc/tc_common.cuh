@@ -166,6 +166,43 @@ __device__ __forceinline__ void umma_ss(uint32_t d_tmem, uint64_t adesc, uint64_
         "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate)
         : "memory");
 }
+// Eight MMAs of one K loop (128 elements in steps of 16) from ONE instruction block: descriptors advance by fixed steps,
+// the first MMA overwrites the accumulator when `acc_first` is 0. Keeps the issuing thread's instruction count per MMA
+// below the MMA's own duration at small N.
+__device__ __forceinline__ void umma_ss_k8(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t astep, uint32_t bstep,
+                                           uint32_t idesc, uint32_t acc_first) {
+    asm volatile(
+        "{\n\t.reg .pred p0, p1;\n\t.reg .b64 a, b, sa, sb;\n\t"
+        "setp.ne.b32 p0, %6, 0;\n\tsetp.eq.b32 p1, 0, 0;\n\t"
+        "cvt.u64.u32 sa, %4;\n\tcvt.u64.u32 sb, %5;\n\t"
+        "mov.b64 a, %1;\n\tmov.b64 b, %2;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], a, b, %3, p0;\n\t"
+        "add.u64 a, a, sa;\n\tadd.u64 b, b, sb;\n\ttcgen05.mma.cta_group::1.kind::f16 [%0], a, b, %3, p1;\n\t"
+        "add.u64 a, a, sa;\n\tadd.u64 b, b, sb;\n\ttcgen05.mma.cta_group::1.kind::f16 [%0], a, b, %3, p1;\n\t"
+        "add.u64 a, a, sa;\n\tadd.u64 b, b, sb;\n\ttcgen05.mma.cta_group::1.kind::f16 [%0], a, b, %3, p1;\n\t"
+        "add.u64 a, a, sa;\n\tadd.u64 b, b, sb;\n\ttcgen05.mma.cta_group::1.kind::f16 [%0], a, b, %3, p1;\n\t"
+        "add.u64 a, a, sa;\n\tadd.u64 b, b, sb;\n\ttcgen05.mma.cta_group::1.kind::f16 [%0], a, b, %3, p1;\n\t"
+        "add.u64 a, a, sa;\n\tadd.u64 b, b, sb;\n\ttcgen05.mma.cta_group::1.kind::f16 [%0], a, b, %3, p1;\n\t"
+        "add.u64 a, a, sa;\n\tadd.u64 b, b, sb;\n\ttcgen05.mma.cta_group::1.kind::f16 [%0], a, b, %3, p1;\n\t}" ::"r"(d_tmem),
+        "l"(adesc), "l"(bdesc), "r"(idesc), "r"(astep), "r"(bstep), "r"(acc_first)
+        : "memory");
+}
+
+// The same for a K loop of four steps (64 elements).
+__device__ __forceinline__ void umma_ss_k4(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t astep, uint32_t bstep,
+                                           uint32_t idesc, uint32_t acc_first) {
+    asm volatile(
+        "{\n\t.reg .pred p0, p1;\n\t.reg .b64 a, b, sa, sb;\n\t"
+        "setp.ne.b32 p0, %6, 0;\n\tsetp.eq.b32 p1, 0, 0;\n\t"
+        "cvt.u64.u32 sa, %4;\n\tcvt.u64.u32 sb, %5;\n\t"
+        "mov.b64 a, %1;\n\tmov.b64 b, %2;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], a, b, %3, p0;\n\t"
+        "add.u64 a, a, sa;\n\tadd.u64 b, b, sb;\n\ttcgen05.mma.cta_group::1.kind::f16 [%0], a, b, %3, p1;\n\t"
+        "add.u64 a, a, sa;\n\tadd.u64 b, b, sb;\n\ttcgen05.mma.cta_group::1.kind::f16 [%0], a, b, %3, p1;\n\t"
+        "add.u64 a, a, sa;\n\tadd.u64 b, b, sb;\n\ttcgen05.mma.cta_group::1.kind::f16 [%0], a, b, %3, p1;\n\t}" ::"r"(d_tmem),
+        "l"(adesc), "l"(bdesc), "r"(idesc), "r"(astep), "r"(bstep), "r"(acc_first)
+        : "memory");
+}
 // The mbarrier receives one arrival when all MMAs issued so far by this thread have completed.
 __device__ __forceinline__ void umma_commit(uint32_t bar) {
     asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");

@@ -207,17 +207,23 @@ gemm::Params base_params(lococo_handle* h) {
 //   dX_V += P^T dO, dX_K += dS^T Q                accumulated in TMEM over all query tiles, added to memory at the end
 // so P never reaches memory and dS is written once. Three roles meet at mbarriers: one lane drives the tensor copy
 // engine (keys and values once, then Q / dO tiles through two stages), one lane issues the MMAs (the score products of
-// tile t+1 are queued behind the gradient products of tile t), eight warps turn scores into P^T and dS^T.
+// tile t+1 are queued behind the gradient products of tile t), sixteen warps turn scores into P^T and dS^T (that
+// part is bound by instruction issue: about a microsecond per tile with eight warps).
 // TMEM: S^T x2 (64 columns each), dP^T x2, dX_V, dX_K (128 each) = 512 columns.
 namespace fused {
 
 using namespace tc;
 
-constexpr int kThreads = 320;
+constexpr int kEpiWarps = 16;             // four warps per TMEM lane quarter, 16 of a tile's 64 queries each
+constexpr int kEpiThreads = 32 * kEpiWarps;
+constexpr int kMmaThread = kEpiThreads, kLoadThread = kEpiThreads + 32;
+constexpr int kThreads = kEpiThreads + 64;
 constexpr uint32_t kKvTile = 32768;       // 128 rows x 128 channels: two 64-channel halves of 16 KB (128-byte swizzle)
 constexpr uint32_t kQTile = 16384;        // 64 rows x 128 channels: two halves of 8 KB
 constexpr uint32_t kPTile = 16384;        // 128 keys x 64 queries, bf16: [8-query group][128 rows][8 queries]
-constexpr uint32_t kSmem = 2 * kKvTile + 2 * 2 * kQTile + 2 * 2 * kPTile + 2 * 128 * 4 + 256 + 1024;
+constexpr int kQStages = 3;              // Q / dO stages: a stage is held from its score products to its gradient products, and a tile takes about a
+                                         // microsecond to arrive, so two stages leave the tensor pipe waiting for loads
+constexpr uint32_t kSmem = 2 * kKvTile + kQStages * 2 * kQTile + 2 * 2 * kPTile + 2 * 128 * 4 + 256 + 1024;
 
 struct alignas(64) Params {
     CUtensorMap map_x;            // packed [unit][pad + position][K 128 | V 128], boxes of 128 rows x 64 channels
@@ -243,29 +249,33 @@ __global__ void __launch_bounds__(kThreads, 1) attn_bwd_kv_kernel(const __grid_c
     uint8_t* k_ptr = smem;
     uint8_t* v_ptr = k_ptr + kKvTile;
     uint8_t* qd_ptr = v_ptr + kKvTile;                 // stage x: [Q | dO]
-    uint8_t* p_ptr = qd_ptr + 2 * 2 * kQTile;          // buffer x: [P^T | dS^T]
+    uint8_t* p_ptr = qd_ptr + kQStages * 2 * kQTile;   // buffer x: [P^T | dS^T]
     float* vec = reinterpret_cast<float*>(p_ptr + 2 * 2 * kPTile);   // buffer x: [64 lse * log2 e | 64 delta]
     uint64_t* bars = reinterpret_cast<uint64_t*>(vec + 2 * 128);
-    volatile int* failed = reinterpret_cast<volatile int*>(bars + 12);
+    volatile int* failed = reinterpret_cast<volatile int*>(bars + 16);
     const uint32_t ks = smem_u32(k_ptr), vs = smem_u32(v_ptr), qds = smem_u32(qd_ptr), ps = smem_u32(p_ptr);
     const uint32_t bar0 = smem_u32(bars);
-    auto qd_full = [&](int x) { return bar0 + 8 * x; };          // loader -> MMA: Q, dO tile staged
-    auto s_full = [&](int x) { return bar0 + 16 + 8 * x; };      // MMA -> warps: S^T, dP^T in TMEM
-    auto s_free = [&](int x) { return bar0 + 32 + 8 * x; };      // warps -> MMA: S^T, dP^T read
-    auto p_full = [&](int x) { return bar0 + 48 + 8 * x; };      // warps -> MMA: P^T, dS^T written
-    auto g_done = [&](int x) { return bar0 + 64 + 8 * x; };      // MMA -> loader, warps: gradient products done
-    const uint32_t kv_full = bar0 + 80, acc_done = bar0 + 88;
+    auto qd_full = [&](int x) { return bar0 + 8 * x; };           // loader -> MMA: Q, dO tile staged (three stages)
+    auto qd_free = [&](int x) { return bar0 + 24 + 8 * x; };      // MMA -> loader: gradient products have read the stage
+    auto s_full = [&](int x) { return bar0 + 48 + 8 * x; };       // MMA -> warps: S^T, dP^T in TMEM
+    auto s_free = [&](int x) { return bar0 + 64 + 8 * x; };       // warps -> MMA: S^T, dP^T read
+    auto p_full = [&](int x) { return bar0 + 80 + 8 * x; };       // warps -> MMA: P^T, dS^T written
+    auto g_done = [&](int x) { return bar0 + 96 + 8 * x; };       // MMA -> warps: gradient products have read P^T, dS^T
+    const uint32_t kv_full = bar0 + 112, acc_done = bar0 + 120;
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int jt = blockIdx.x, u = blockIdx.y;
     const int n = u / P.heads, h = u % P.heads;
     const int j0 = jt * 128;
 
-    if (tid == 256) {
-        for (int x = 0; x < 2; ++x) {
+    if (tid == kMmaThread) {
+        for (int x = 0; x < kQStages; ++x) {
             mbar_init(qd_full(x), 1);
+            mbar_init(qd_free(x), 1);
+        }
+        for (int x = 0; x < 2; ++x) {
             mbar_init(s_full(x), 1);
-            mbar_init(s_free(x), 256);
-            mbar_init(p_full(x), 256);
+            mbar_init(s_free(x), kEpiThreads);
+            mbar_init(p_full(x), kEpiThreads);
             mbar_init(g_done(x), 1);
         }
         mbar_init(kv_full, 1);
@@ -290,15 +300,15 @@ __global__ void __launch_bounds__(kThreads, 1) attn_bwd_kv_kernel(const __grid_c
     const int first = 2 * (max(0, j0 - P.c - P.q0) / 128);
     const bool any = first < T && j0 < P.S;
 
-    if (tid == 288 && any) {
+    if (tid == kLoadThread && any) {
         // ---------------- loader
         mbar_expect_tx(kv_full, 2 * kKvTile);
         for (int x = 0; x < 4; ++x)      // K channels 0-63, 64-127, V channels 0-63, 64-127
             tma_load_4d(ks + x * (kKvTile / 2), &P.map_x, 64 * x, P.pad + j0, u, 0, kv_full);
 #pragma unroll 1
         for (int t = first; t < T; ++t) {
-            const int x = (t - first) & 1, use = (t - first) >> 1;
-            if (use >= 1) mbar_wait(g_done(x), (use - 1) & 1, P.status, failed, 40);
+            const int x = (t - first) % kQStages, use = (t - first) / kQStages;
+            if (use >= 1) mbar_wait(qd_free(x), (use - 1) & 1, P.status, failed, 40);
             mbar_expect_tx(qd_full(x), 2 * kQTile);
             const uint32_t dst = qds + x * 2 * kQTile;
             const int row = P.q0 + 64 * t;
@@ -307,93 +317,103 @@ __global__ void __launch_bounds__(kThreads, 1) attn_bwd_kv_kernel(const __grid_c
             tma_load_4d(dst + kQTile, &P.map_do, 0, row, h, n, qd_full(x));
             tma_load_4d(dst + kQTile + kQTile / 2, &P.map_do, 64, row, h, n, qd_full(x));
         }
-    } else if (tid == 256 && any) {
+    } else if (tid == kMmaThread && any) {
         // ---------------- MMA issuer
         const uint32_t idesc_s = instr_desc_bf16(64, false, false);
         const uint32_t idesc_g = instr_desc_bf16(128, false, true);
         const uint64_t ka = smem_desc_sw128(ks, 16, 1024), va = smem_desc_sw128(vs, 16, 1024);
-        auto kstep = [](int kk, uint32_t half_bytes) { return (uint64_t)(((kk >> 2) * half_bytes + (kk & 3) * 32u) >> 4); };
         auto issue_grad = [&](int t) {
-            const int x = (t - first) & 1, use = (t - first) >> 1;
+            const int x = (t - first) & 1, use = (t - first) >> 1, sx = (t - first) % kQStages;
             mbar_wait(p_full(x), use & 1, P.status, failed, 41);
             tc_fence_after();
-            const uint32_t q_addr = qds + x * 2 * kQTile, pt = ps + x * 2 * kPTile;
+            const uint32_t q_addr = qds + sx * 2 * kQTile, pt = ps + x * 2 * kPTile;
             const uint64_t pa = smem_desc(pt, 2048, 128), da = smem_desc(pt + kPTile, 2048, 128);
             const uint64_t qb_mn = smem_desc_sw128(q_addr, kQTile / 2, 1024), dob_mn = smem_desc_sw128(q_addr + kQTile, kQTile / 2, 1024);
-#pragma unroll
-            for (int kk = 0; kk < 4; ++kk) {       // 16 queries per step: two 8-query groups of the A operand, two 8-row groups of the B operand
-                umma_ss(tmem + 256, pa + kk * 256u, dob_mn + kk * 128u, idesc_g, (t != first || kk != 0));
-                umma_ss(tmem + 384, da + kk * 256u, qb_mn + kk * 128u, idesc_g, (t != first || kk != 0));
-            }
+            // 16 queries per step: two 8-query groups of the A operand, two 8-row groups of the B operand
+            umma_ss_k4(tmem + 256, pa, dob_mn, 256u, 128u, idesc_g, t != first);
+            umma_ss_k4(tmem + 384, da, qb_mn, 256u, 128u, idesc_g, t != first);
             umma_commit(g_done(x));
+            umma_commit(qd_free(sx));
         };
         mbar_wait(kv_full, 0, P.status, failed, 42);
 #pragma unroll 1
         for (int t = first; t < T; ++t) {
-            const int x = (t - first) & 1, use = (t - first) >> 1;
-            mbar_wait(qd_full(x), use & 1, P.status, failed, 43);
+            const int x = (t - first) & 1, use = (t - first) >> 1, sx = (t - first) % kQStages;
+            mbar_wait(qd_full(sx), ((t - first) / kQStages) & 1, P.status, failed, 43);
             if (use >= 1) mbar_wait(s_free(x), (use - 1) & 1, P.status, failed, 44);
             tc_fence_after();
-            const uint32_t q_addr = qds + x * 2 * kQTile;
+            const uint32_t q_addr = qds + sx * 2 * kQTile;
             const uint64_t qk = smem_desc_sw128(q_addr, 16, 1024), dok = smem_desc_sw128(q_addr + kQTile, 16, 1024);
-#pragma unroll
-            for (int kk = 0; kk < 8; ++kk) umma_ss(tmem + x * 64, ka + kstep(kk, kKvTile / 2), qk + kstep(kk, kQTile / 2), idesc_s, kk != 0);
-#pragma unroll
-            for (int kk = 0; kk < 8; ++kk) umma_ss(tmem + 128 + x * 64, va + kstep(kk, kKvTile / 2), dok + kstep(kk, kQTile / 2), idesc_s, kk != 0);
+            // 128 channels: 32 bytes per 16-channel step inside a 128-byte row, then the second 64-channel half of each tile
+            umma_ss_k4(tmem + x * 64, ka, qk, 2u, 2u, idesc_s, 0);
+            umma_ss_k4(tmem + x * 64, ka + ((kKvTile / 2) >> 4), qk + ((kQTile / 2) >> 4), 2u, 2u, idesc_s, 1);
+            umma_ss_k4(tmem + 128 + x * 64, va, dok, 2u, 2u, idesc_s, 0);
+            umma_ss_k4(tmem + 128 + x * 64, va + ((kKvTile / 2) >> 4), dok + ((kQTile / 2) >> 4), 2u, 2u, idesc_s, 1);
             umma_commit(s_full(x));
             if (t > first) issue_grad(t - 1);
         }
         issue_grad(T - 1);
         umma_commit(acc_done);
     }
-    if (warp < 8 && any) {
-        // ---------------- P^T and dS^T: a thread owns one key (TMEM lane) and 32 of the tile's 64 queries
-        const int rl = (warp & 3) * 32 + lane, half = warp >> 2;
+    if (warp < kEpiWarps && any) {
+        // ---------------- P^T and dS^T: a thread owns one key (TMEM lane) and 16 of the tile's 64 queries
+        const int rl = (warp & 3) * 32 + lane, part = warp >> 2;
         const int j = j0 + rl;
         const uint32_t lane_base = tmem + ((uint32_t)((warp & 3) * 32) << 16);
         __nv_bfloat16* ds_row = P.ds_t + (int64_t)u * P.ds_z + (int64_t)j * P.ds_row;
+        // per-query vectors of a tile (lse * log2 e, delta): threads 0-127 fetch one value each, a tile ahead, so that
+        // the load's latency is not part of an iteration
+        auto fetch = [&](int t) {
+            const int q = 64 * t + (tid & 63);                       // query within the block
+            if (tid >= 128 || t >= T || q >= P.qb) return 0.f;
+            return tid < 64 ? P.lse[(int64_t)u * P.lse_z + q] * 1.4426950408889634f : P.delta[(int64_t)u * P.delta_z + q];
+        };
+        float next_vec = fetch(first);
 #pragma unroll 1
         for (int t = first; t < T; ++t) {
             const int x = (t - first) & 1, use = (t - first) >> 1;
             float* vb = vec + x * 128;
-            if (tid < 128) {
-                const int q = 64 * t + (tid & 63);                   // query within the block
-                const bool ok = q < P.qb;
-                vb[tid] = tid < 64 ? (ok ? P.lse[(int64_t)u * P.lse_z + q] * 1.4426950408889634f : 0.f)
-                                   : (ok ? P.delta[(int64_t)u * P.delta_z + q] : 0.f);
-            }
-            asm volatile("bar.sync 1, 256;" ::: "memory");
+            if (tid < 128) vb[tid] = next_vec;
+            asm volatile("bar.sync 1, %0;" ::"n"(kEpiThreads) : "memory");
+            next_vec = fetch(t + 1);
             mbar_wait(s_full(x), use & 1, P.status, failed, 45);
             tc_fence_after();
-            uint32_t sv[32], dv[32];
-            tmem_ld32(lane_base + x * 64 + half * 32, sv);
-            tmem_ld32(lane_base + 128 + x * 64 + half * 32, dv);
+            uint32_t sv[16], dv[16];
+            tmem_ld16(lane_base + x * 64 + part * 16, sv);
+            tmem_ld16(lane_base + 128 + x * 64 + part * 16, dv);
             tmem_ld_wait();
             tc_fence_before();
             mbar_arrive(s_free(x));
             if (use >= 1) mbar_wait(g_done(x), (use - 1) & 1, P.status, failed, 46);      // the P^T, dS^T buffer is free again
-            const int qc0 = 64 * t + half * 32;                      // first of this thread's queries, within the block
+            const int qc0 = 64 * t + part * 16;                      // first of this thread's queries, within the block
             // key j is seen by query r of the chunk when j < c + r + 1
             const int lim = j - P.c - P.q0;                          // visible: query (within the block) >= lim
             uint8_t* pdst = p_ptr + x * 2 * kPTile + rl * 16;
+            // tiles that neither the causal limit nor the end of the keys or queries cuts need no tests (the common case)
+            const bool whole = j0 + 128 <= P.S && 64 * t + 64 <= P.qb && j0 + 127 - P.c - P.q0 <= 64 * t;
+            const float4* lv = reinterpret_cast<const float4*>(vb + part * 16);
+            const float4* dl = reinterpret_cast<const float4*>(vb + 64 + part * 16);
 #pragma unroll
-            for (int e = 0; e < 32; e += 8) {
-                uint32_t pk[4], dk[4];
+            for (int e = 0; e < 16; e += 8) {
+                const float4 la = lv[e >> 2], lb = lv[(e >> 2) + 1], da = dl[e >> 2], db = dl[(e >> 2) + 1];
+                const float ls[8] = {la.x, la.y, la.z, la.w, lb.x, lb.y, lb.z, lb.w};
+                const float de[8] = {da.x, da.y, da.z, da.w, db.x, db.y, db.z, db.w};
+                float pv[8], dsv[8];
 #pragma unroll
-                for (int y = 0; y < 8; y += 2) {
-                    const int qa = qc0 + e + y;
-                    const bool on0 = j < P.S && qa < P.qb && qa >= lim, on1 = j < P.S && qa + 1 < P.qb && qa + 1 >= lim;
-                    const float p0 = on0 ? exp2f(__uint_as_float(sv[e + y]) * P.scale2 - vb[half * 32 + e + y]) : 0.f;
-                    const float p1 = on1 ? exp2f(__uint_as_float(sv[e + y + 1]) * P.scale2 - vb[half * 32 + e + y + 1]) : 0.f;
-                    const float d0 = p0 * (__uint_as_float(dv[e + y]) - vb[64 + half * 32 + e + y]) * P.scale;
-                    const float d1 = p1 * (__uint_as_float(dv[e + y + 1]) - vb[64 + half * 32 + e + y + 1]) * P.scale;
-                    pk[y >> 1] = pack_bf16(p0, p1);
-                    dk[y >> 1] = pack_bf16(on0 ? d0 : 0.f, on1 ? d1 : 0.f);
+                for (int y = 0; y < 8; ++y) {
+                    pv[y] = exp2f(fmaf(__uint_as_float(sv[e + y]), P.scale2, -ls[y]));
+                    if (!whole) {
+                        const int qa = qc0 + e + y;
+                        if (!(j < P.S && qa < P.qb && qa >= lim)) pv[y] = 0.f;
+                    }
+                    dsv[y] = pv[y] * (__uint_as_float(dv[e + y]) - de[y]) * P.scale;
                 }
-                const uint32_t g = (uint32_t)((half * 32 + e) >> 3) * 2048u;
-                *reinterpret_cast<uint4*>(pdst + g) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
-                *reinterpret_cast<uint4*>(pdst + kPTile + g) = make_uint4(dk[0], dk[1], dk[2], dk[3]);
-                if (j < P.S) *reinterpret_cast<uint4*>(ds_row + qc0 + e) = make_uint4(dk[0], dk[1], dk[2], dk[3]);
+                const uint4 pk = make_uint4(pack_bf16(pv[0], pv[1]), pack_bf16(pv[2], pv[3]), pack_bf16(pv[4], pv[5]), pack_bf16(pv[6], pv[7]));
+                const uint4 dk = make_uint4(pack_bf16(dsv[0], dsv[1]), pack_bf16(dsv[2], dsv[3]), pack_bf16(dsv[4], dsv[5]), pack_bf16(dsv[6], dsv[7]));
+                const uint32_t g = (uint32_t)((part * 16 + e) >> 3) * 2048u;
+                *reinterpret_cast<uint4*>(pdst + g) = pk;
+                *reinterpret_cast<uint4*>(pdst + kPTile + g) = dk;
+                if (j < P.S) *reinterpret_cast<uint4*>(ds_row + qc0 + e) = dk;
             }
             fence_proxy_async();
             mbar_arrive(p_full(x));
@@ -403,16 +423,15 @@ __global__ void __launch_bounds__(kThreads, 1) attn_bwd_kv_kernel(const __grid_c
         tc_fence_after();
         {
             const bool row_live = j < P.S;
-            float* ok = P.dXK + ((int64_t)u * P.S + (row_live ? j : 0)) * kD + half * 64;
-            float* ov = P.dXV + ((int64_t)u * P.S + (row_live ? j : 0)) * kD + half * 64;
+            float* ok = P.dXK + ((int64_t)u * P.S + (row_live ? j : 0)) * kD + part * 32;
+            float* ov = P.dXV + ((int64_t)u * P.S + (row_live ? j : 0)) * kD + part * 32;
 #pragma unroll 1
-            for (int piece = 0; piece < 4; ++piece) {
-                const int mat = piece >> 1, c0 = (piece & 1) * 32;
+            for (int mat = 0; mat < 2; ++mat) {
                 uint32_t a[32];
-                tmem_ld32(lane_base + (mat ? 384 : 256) + half * 64 + c0, a);     // (the whole warp, whatever its rows)
+                tmem_ld32(lane_base + (mat ? 384 : 256) + part * 32, a);     // (the whole warp, whatever its rows)
                 tmem_ld_wait();
                 if (row_live) {
-                    float4* dst = reinterpret_cast<float4*>((mat ? ok : ov) + c0);
+                    float4* dst = reinterpret_cast<float4*>(mat ? ok : ov);
 #pragma unroll
                     for (int e = 0; e < 8; ++e) {
                         float4 cur = dst[e];

@@ -507,28 +507,6 @@ constexpr uint32_t kPairVTile = 32768;            // 128 cache rows x 128 channe
 constexpr uint32_t kPairOutRow = 272;             // bytes per row of a staged output tile: 256 + 16, so that 16-byte accesses of 8 rows miss each other's banks
 constexpr uint32_t kPairOutTile = kSlots * kPairOutRow;
 
-// Eight MMAs of one K loop (128 channels in steps of 16) from ONE instruction block: descriptors advance by fixed steps,
-// the first MMA overwrites the accumulator when `acc_first` is 0. Keeps the issuing thread's instruction count per MMA
-// below the MMA's own duration at small N.
-__device__ __forceinline__ void umma_ss_k8(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t astep, uint32_t bstep,
-                                           uint32_t idesc, uint32_t acc_first) {
-    asm volatile(
-        "{\n\t.reg .pred p0, p1;\n\t.reg .b64 a, b, sa, sb;\n\t"
-        "setp.ne.b32 p0, %6, 0;\n\tsetp.eq.b32 p1, 0, 0;\n\t"
-        "cvt.u64.u32 sa, %4;\n\tcvt.u64.u32 sb, %5;\n\t"
-        "mov.b64 a, %1;\n\tmov.b64 b, %2;\n\t"
-        "tcgen05.mma.cta_group::1.kind::f16 [%0], a, b, %3, p0;\n\t"
-        "add.u64 a, a, sa;\n\tadd.u64 b, b, sb;\n\ttcgen05.mma.cta_group::1.kind::f16 [%0], a, b, %3, p1;\n\t"
-        "add.u64 a, a, sa;\n\tadd.u64 b, b, sb;\n\ttcgen05.mma.cta_group::1.kind::f16 [%0], a, b, %3, p1;\n\t"
-        "add.u64 a, a, sa;\n\tadd.u64 b, b, sb;\n\ttcgen05.mma.cta_group::1.kind::f16 [%0], a, b, %3, p1;\n\t"
-        "add.u64 a, a, sa;\n\tadd.u64 b, b, sb;\n\ttcgen05.mma.cta_group::1.kind::f16 [%0], a, b, %3, p1;\n\t"
-        "add.u64 a, a, sa;\n\tadd.u64 b, b, sb;\n\ttcgen05.mma.cta_group::1.kind::f16 [%0], a, b, %3, p1;\n\t"
-        "add.u64 a, a, sa;\n\tadd.u64 b, b, sb;\n\ttcgen05.mma.cta_group::1.kind::f16 [%0], a, b, %3, p1;\n\t"
-        "add.u64 a, a, sa;\n\tadd.u64 b, b, sb;\n\ttcgen05.mma.cta_group::1.kind::f16 [%0], a, b, %3, p1;\n\t}" ::"r"(d_tmem),
-        "l"(adesc), "l"(bdesc), "r"(idesc), "r"(astep), "r"(bstep), "r"(acc_first)
-        : "memory");
-}
-
 struct PairLayout {
     uint32_t rows_k, lbo_k, r_bytes, x_bytes, total;
 };
