@@ -4,7 +4,7 @@
 //   cache update (Eq. 4-7 reversed)
 //     R, s        recomputed by the forward's own tcgen05 conv kernel (R left in place)
 //     dw          = [gK | gV] [X_K | X_V]^T                          per unit, K = 2d
-//     dA          row kernel: dA = [R>0] (dw - <dw, w>_row) / s with w = R / s, rounded to bf16
+//     dA          row kernel: dA = [R>0] (dw - <dw, w>_row) / s with w = R / s, rounded to bf16, written in both orientations
 //     dX         += w^T [gK | gV] = R^T ([gK | gV] / s)               per unit, K = M; R is exact in bf16
 //     dG         += sum over units and positions of dA (*) Z          the im2col view of Z is a tensor
 //                                                                     map with overlapping strides
@@ -113,57 +113,61 @@ __global__ void pack_gt_kernel(const __nv_bfloat16* gp, __nv_bfloat16* gt, int M
     for (int r = threadIdx.y; r < 32; r += blockDim.y) gt[plane + (int64_t)(c0 + r) * M + i0 + threadIdx.x] = tile[threadIdx.x][r];
 }
 
-// One block per (unit, slot) row: dA = [R>0] (dw - <dw, w>) / s with w = R / s (Eq. 7 reversed), in bf16,
-// zero from column S up to the row stride; R comes from the recompute in bf16 (rows of Sp, zero beyond S);
-// dbias += sum of dA.
-__global__ void __launch_bounds__(256) da_row_kernel(BwdStep p, const float* dw, __nv_bfloat16* dab, const __nv_bfloat16* rb, int Sp) {
-    __shared__ float red[8];
-    const int64_t row = blockIdx.x;                          // u * M + i
-    const float* dwr = dw + row * Sp;
-    const __nv_bfloat16* Rr = rb + row * Sp;
-    const float inv_s = 1.f / p.s[row];
-    float acc = 0.f;
-    for (int j = threadIdx.x; j < p.S; j += 256) acc = fmaf(__bfloat162float(Rr[j]), dwr[j], acc);
-    for (int of = 16; of > 0; of >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, of);
-    if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = acc;
+// dA = [R>0] (dw - <dw, w>) / s with w = R / s (Eq. 7 reversed), rounded to bf16, in both orientations: dAb[u][i][j]
+// (rows of Sp, zero from column S on) and dAT[u][j][i]. One block per 16 consecutive slots of a unit, so that a
+// thread's piece of the transposed copy is 16 slots = one full 32-byte sector. R comes from the recompute in bf16
+// (rows of Sp, zero beyond S); dbias += sum of dA.
+constexpr int kDaRows = 16;
+__global__ void __launch_bounds__(256) da_rows_kernel(BwdStep p, const float* dw, __nv_bfloat16* dab, __nv_bfloat16* dat, const __nv_bfloat16* rb, int Sp) {
+    __shared__ float dots[kDaRows], bias_sum[kDaRows];
+    const int blocks_per_unit = p.M / kDaRows;
+    const int u = blockIdx.x / blocks_per_unit, i0 = (blockIdx.x % blocks_per_unit) * kDaRows;
+    const int64_t row0 = (int64_t)u * p.M + i0;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    // <dw, w> of the 16 rows: two rows per warp
+    for (int r = warp; r < kDaRows; r += 8) {
+        const float* dwr = dw + (row0 + r) * Sp;
+        const __nv_bfloat16* Rr = rb + (row0 + r) * Sp;
+        float acc = 0.f;
+        for (int j = lane; j < p.S; j += 32) acc = fmaf(__bfloat162float(Rr[j]), dwr[j], acc);
+        for (int of = 16; of > 0; of >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, of);
+        if (lane == 0) { dots[r] = acc / p.s[row0 + r]; bias_sum[r] = 0.f; }
+    }
     __syncthreads();
-    float dot = 0.f;
-    for (int w = 0; w < 8; ++w) dot += red[w];
-    dot *= inv_s;                                            // <dw, w>
-    float bsum = 0.f;
+    float inv_s[kDaRows], dot[kDaRows], bsum[kDaRows];
+#pragma unroll
+    for (int r = 0; r < kDaRows; ++r) { inv_s[r] = 1.f / p.s[row0 + r]; dot[r] = dots[r]; bsum[r] = 0.f; }
+    // a thread takes a position j and all 16 rows: the rows' reads and writes are 2- or 4-byte pieces of lines the
+    // whole warp covers (consecutive j), the transposed write is 32 bytes
     for (int j = threadIdx.x; j < Sp; j += 256) {
-        float da = 0.f;
-        if (j < p.S && __bfloat162float(Rr[j]) > 0.f) da = (dwr[j] - dot) * inv_s;
-        dab[row * Sp + j] = __float2bfloat16_rn(da);
-        bsum += da;
+        __align__(16) __nv_bfloat16 col[kDaRows];
+        float rv[kDaRows], dwv[kDaRows];
+#pragma unroll
+        for (int r = 0; r < kDaRows; ++r) {          // all 32 loads first: they do not depend on one another
+            rv[r] = __bfloat162float(rb[(row0 + r) * Sp + j]);
+            dwv[r] = dw[(row0 + r) * Sp + j];
+        }
+#pragma unroll
+        for (int r = 0; r < kDaRows; ++r) {
+            const float da = (j < p.S && rv[r] > 0.f) ? (dwv[r] - dot[r]) * inv_s[r] : 0.f;
+            col[r] = __float2bfloat16_rn(da);
+            dab[(row0 + r) * Sp + j] = col[r];
+            bsum[r] += da;
+        }
+        uint4* dst = reinterpret_cast<uint4*>(dat + ((int64_t)u * Sp + j) * p.M + i0);
+        dst[0] = *reinterpret_cast<const uint4*>(col);
+        dst[1] = *reinterpret_cast<const uint4*>(col + 8);
     }
     if (p.dbias) {
-        __syncthreads();
-        for (int of = 16; of > 0; of >>= 1) bsum += __shfl_xor_sync(0xffffffffu, bsum, of);
-        if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = bsum;
-        __syncthreads();
-        if (threadIdx.x == 0) {
-            float t = 0.f;
-            for (int w = 0; w < 8; ++w) t += red[w];
-            const int u = (int)(row / p.M), i = (int)(row % p.M);
-            atomicAdd(p.dbias + (p.weights_per_head ? (u % p.heads) * p.M : 0) + i, t);
+#pragma unroll
+        for (int r = 0; r < kDaRows; ++r) {
+            float t = bsum[r];
+            for (int of = 16; of > 0; of >>= 1) t += __shfl_xor_sync(0xffffffffu, t, of);
+            if (lane == 0) atomicAdd(&bias_sum[r], t);
         }
-    }
-}
-
-// dAT[u][j][i] = dAb[u][i][j]: 64 x 64 tiles through shared memory.
-__global__ void __launch_bounds__(256) transpose_kernel(const __nv_bfloat16* in, __nv_bfloat16* out, int M, int Sp) {
-    __shared__ __nv_bfloat16 tile[64][66];
-    const int u = blockIdx.z, i0 = blockIdx.y * 64, j0 = blockIdx.x * 64;
-    const int tx = threadIdx.x & 63, ty = threadIdx.x >> 6;
-    for (int r = ty; r < 64; r += 4) {
-        const int j = j0 + tx;
-        tile[r][tx] = j < Sp ? in[((int64_t)u * M + i0 + r) * Sp + j] : __float2bfloat16_rn(0.f);
-    }
-    __syncthreads();
-    for (int r = ty; r < 64; r += 4) {
-        const int j = j0 + r;
-        if (j < Sp) out[((int64_t)u * Sp + j) * M + i0 + tx] = tile[tx][r];
+        __syncthreads();
+        if (threadIdx.x < kDaRows)
+            atomicAdd(p.dbias + (p.weights_per_head ? (u % p.heads) * p.M : 0) + i0 + threadIdx.x, bias_sum[threadIdx.x]);
     }
 }
 
@@ -523,10 +527,9 @@ int tensor_backward_compress(lococo_handle* h, const BwdStep& p, const CompressP
         if (!gemm::launch(G, m_tiles, s_tiles, U, st)) return -1;
         ++n;
     }
-    da_row_kernel<<<U * M, 256, 0, st>>>(p, dw, dab, wb, L.Sp);
-    transpose_kernel<<<dim3((L.Sp + 63) / 64, M / 64, U), 256, 0, st>>>(dab, dat, M, L.Sp);
+    da_rows_kernel<<<U * (M / kDaRows), 256, 0, st>>>(p, dw, dab, dat, wb, L.Sp);
     if (!launched()) return -1;
-    n += 2;
+    ++n;
 
     const Tensor4 t_wb{wb, {(uint64_t)L.Sp, (uint64_t)M, (uint64_t)U, 1}, {(uint64_t)L.Sp * 2, (uint64_t)M * L.Sp * 2, (uint64_t)U * M * L.Sp * 2}};
     const Tensor4 t_dab{dab, {(uint64_t)L.Sp, (uint64_t)M, (uint64_t)U, 1}, {(uint64_t)L.Sp * 2, (uint64_t)M * L.Sp * 2, (uint64_t)U * M * L.Sp * 2}};
