@@ -67,6 +67,15 @@ struct TcCompressParams {
     int n_tile, tiles, parts, tiles_per_part, halves, stages, rows_pad, slot_blocks;
     int pair;                     // 1: generation-stage form, one CTA per TWO units that share a weight set (compress_pair_body)
     int pairs;                    // CTAs of that form
+    // Tensor maps for staging the key and value tiles with the tensor copy engine (boxes of `rows` = n_tile + k - 1 token
+    // rows x 64 channels, 128-byte swizzle), and for the tile (at most two) that holds both cache and chunk rows a pair of
+    // maps with the box heights of its two parts. tile_maps == 0: every tile is staged by 16-byte async copies instead.
+    int tile_maps;
+    int seam_h1[2];               // cache rows (halo included) of a mixed tile; 0 = unused entry
+};
+enum { kTmKCache = 0, kTmKChunk = 1, kTmVCache = 2, kTmVChunk = 3, kTmSeam = 4, kTileMaps = 12 };   // seam e: 4 + 4 e + {Kc, Kn, Vc, Vn}
+struct alignas(64) TcTileMaps {
+    CUtensorMap m[kTileMaps];
 };
 
 // G [sets][M][C][k] -> per (set, slot block, tap, 128-channel half) a 32 KB image of the
@@ -167,10 +176,13 @@ __device__ __forceinline__ void merge_partials(const TcCompressParams& P, uint32
 // `tmem`: base of 512 TMEM columns the CTA owns. `cache_cg`: read cache rows around L1 (set when the
 // cache was rewritten by other SMs earlier in the SAME kernel; L1 is coherent only across launches).
 // kMerge: whether the kernel is one that may be asked to merge the partial sets itself (P.merge).
+// `tmaps`: the tile maps in kernel parameter space, or nullptr (async-copy staging).
 template <bool kMerge>
-__device__ __forceinline__ void compress_body(const TcCompressParams& P, uint8_t* smem, uint32_t tmem, bool cache_cg, int part,
-                                              int sb, int u) {
+__device__ __forceinline__ void compress_body(const TcCompressParams& P, const TcTileMaps* tmaps, uint8_t* smem_raw, uint32_t tmem,
+                                              bool cache_cg, int part, int sb, int u) {
     const CompressParams& p = P.base;
+    // the tiles are 128-byte swizzled (a function of the shared-memory address): everything starts on a 1024-byte boundary
+    uint8_t* smem = smem_raw + ((1024u - (smem_u32(smem_raw) & 1023u)) & 1023u);
     const int nthr16 = blockDim.x / 16;
     const int n = u / p.heads, h = u % p.heads;
     const int tid = threadIdx.x, warp = tid >> 5;
@@ -178,19 +190,20 @@ __device__ __forceinline__ void compress_body(const TcCompressParams& P, uint8_t
     const int rl = (warp & 3) * 32 + (tid & 31);       // accumulator row = slot within the block
     const int n_tile = P.n_tile, pad = (p.k - 1) / 2, rows = n_tile + p.k - 1;
     const int NS = P.stages;
-    const uint32_t lbo_z = (uint32_t)P.rows_pad * 16u;
+    const uint32_t half_z = (uint32_t)P.rows_pad * 128u;      // one 64-channel half of a tile: rows_pad rows of 128 bytes
     // does this CTA read cache rows (or write the cache itself)? then the earlier kernels come first
     const bool touches_cache = P.direct || part * P.tiles_per_part * n_tile - pad < p.xk.c;
 
     uint8_t* ring_ptr = smem;
     uint8_t* zk_ptr = ring_ptr + (size_t)NS * kStageBytes;
-    uint8_t* zv_ptr = zk_ptr + 16 * lbo_z;
-    uint64_t* bars = reinterpret_cast<uint64_t*>(zv_ptr + 16 * lbo_z);
-    volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(bars + 2 * NS + 2);
+    uint8_t* zv_ptr = zk_ptr + 2 * half_z;
+    uint64_t* bars = reinterpret_cast<uint64_t*>(zv_ptr + 2 * half_z);
+    volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(bars + 2 * NS + 4);
     volatile int* failed = reinterpret_cast<volatile int*>(tmem_slot + 1);
     const uint32_t ring = smem_u32(ring_ptr), zk = smem_u32(zk_ptr), zv = smem_u32(zv_ptr);
     const uint32_t bar_full = smem_u32(bars), bar_empty = bar_full + 8 * NS;
     const uint32_t bar_acc = bar_empty + 8 * NS, bar_blend = bar_acc + 8;
+    const uint32_t bar_k = bar_blend + 8, bar_v = bar_k + 8;     // key tile, value tile staged
 
     if (tid == 128) {
         for (int s = 0; s < NS; ++s) {
@@ -199,6 +212,8 @@ __device__ __forceinline__ void compress_body(const TcCompressParams& P, uint8_t
         }
         mbar_init(bar_acc, 1);
         mbar_init(bar_blend, 1);
+        mbar_init(bar_k, 1);
+        mbar_init(bar_v, 1);
         *failed = 0;
         fence_barrier_init();
     }
@@ -237,41 +252,85 @@ __device__ __forceinline__ void compress_body(const TcCompressParams& P, uint8_t
         if (tid == 160) {
             for (int i = 0; i < npro; ++i) load_stage(g + i, i);
         }
-        // ---- 1. stage the key and value rows j0-pad .. j0+n_tile+pad-1 (zeros outside [0,S))
-        // each thread owns one 8-channel group (q) and every (threads/16)-th row
-        // `rows_of`: 0 all rows, 1 only rows outside the cache (chunk rows and padding), 2 only cache rows
+        // ---- 1. stage the key and value rows j0-pad .. j0+n_tile+pad-1 (zeros outside [0,S)) as two 64-channel halves
+        // of 128-byte rows in the 128-byte swizzle. A tap is a row offset into the tile: the swizzle is a function of the
+        // shared-memory address, so an operand may start at any row.
+        // By the tensor copy engine where the tile's rows are one box of the cache or of the chunk, or (the tile that
+        // holds the seam) one box of each with heights the host prepared; rows outside a tensor arrive as zeros.
+        const int j_first = j0 - pad;
+        const int h1 = p.xk.c > 0 ? max(0, min(rows, p.xk.c - j_first)) : 0;     // rows from the cache at the head of the tile
+        int seam = -1;
+        if (h1 > 0 && h1 < rows) seam = h1 == P.seam_h1[0] ? 0 : (h1 == P.seam_h1[1] ? 1 : -1);
+        const bool by_engine = tmaps != nullptr && P.tile_maps && !cache_cg && (h1 == 0 || h1 == rows || seam >= 0);
+        // one (matrix, source) box: both 64-channel halves
+        auto engine_rows = [&](int map, int y, int dst_row, uint32_t dst, uint32_t bar) {
+            tma_load_4d(dst + dst_row * 128, &tmaps->m[map], 0, y, h, n, bar);
+            tma_load_4d(dst + half_z + dst_row * 128, &tmaps->m[map], 64, y, h, n, bar);
+        };
+        // `which` 0 keys, 1 values; `rows_of`: 0 all rows, 1 only rows outside the cache, 2 only cache rows
+        auto engine_tile = [&](int which, uint32_t dst, uint32_t bar, int rows_of) {
+            if (rows_of != 2) mbar_expect_tx(bar, (uint32_t)rows * 256u);
+            if (h1 == rows) {
+                if (rows_of != 1) engine_rows(kTmKCache + 2 * which, j_first, 0, dst, bar);
+            } else if (h1 == 0) {
+                if (rows_of != 2) engine_rows(kTmKChunk + 2 * which, j_first - p.xk.c, 0, dst, bar);
+            } else {
+                if (rows_of != 1) engine_rows(kTmSeam + 4 * seam + 2 * which, j_first, 0, dst, bar);
+                if (rows_of != 2) engine_rows(kTmSeam + 4 * seam + 2 * which + 1, 0, h1, dst, bar);
+            }
+        };
+        // the same tile by 16-byte async copies: each thread owns one 16-byte piece of a row (q) and every
+        // (threads/16)-th row
         auto stage_tile = [&](const CatView& xv_, uint32_t dst, int first, int step, int rows_of = 0) {
             const int q = first & 15;
             const __nv_bfloat16* cbase = unit_base<__nv_bfloat16>(xv_.cache, n, h) + q * 8;
             const __nv_bfloat16* kbase = unit_base<__nv_bfloat16>(xv_.chunk, n, h) + q * 8;
-            const uint32_t d0 = dst + q * lbo_z;
+            const uint32_t d0 = dst + (uint32_t)(q >> 3) * half_z;
             for (int r = first >> 4; r < rows; r += step) {
-                const int j = j0 - pad + r;
+                const int j = j_first + r;
                 const bool valid = j >= 0 && j < p.S;
                 const bool in_cache = valid && j < xv_.c;
                 if ((rows_of == 1 && in_cache) || (rows_of == 2 && !in_cache)) continue;
                 const __nv_bfloat16* src = !valid ? safe : (in_cache ? cbase + (int64_t)j * xv_.cache.st
                                                                      : kbase + (int64_t)(j - xv_.c) * xv_.chunk.st);
-                if (in_cache && cache_cg) cp_async16_cg(d0 + r * 16, src, 16u);
-                else cp_async16(d0 + r * 16, src, valid ? 16u : 0u);
+                const uint32_t d = d0 + (uint32_t)r * 128u + (uint32_t)(((q & 7) ^ (r & 7)) << 4);
+                if (in_cache && cache_cg) cp_async16_cg(d, src, 16u);
+                else cp_async16(d, src, valid ? 16u : 0u);
             }
         };
-        // the value tile is a conv input only when c_in = 2d; otherwise it is needed by the
-        // blend only and is staged by the epilogue warps while the conv runs
-        if (touches_cache) {
+        // the value tile is a conv input only when c_in = 2d; otherwise the blends alone need it
+        if (by_engine) {
             // chunk rows (and the weight ring's first stages) before the wait for the previous step, cache rows after
-            stage_tile(p.xk, zk, tid, nthr16, 1);
-            if (P.halves == 2) stage_tile(p.xv, zv, tid, nthr16, 1);
-            wait_for_earlier_kernels();
-            stage_tile(p.xk, zk, tid, nthr16, 2);
-            if (P.halves == 2) stage_tile(p.xv, zv, tid, nthr16, 2);
+            if (tid == 192) {
+                engine_tile(0, zk, bar_k, touches_cache ? 1 : 0);
+                engine_tile(1, zv, bar_v, touches_cache ? 1 : 0);
+            }
+            if (touches_cache) {
+                wait_for_earlier_kernels();
+                if (tid == 192) {
+                    engine_tile(0, zk, bar_k, 2);
+                    engine_tile(1, zv, bar_v, 2);
+                }
+            }
         } else {
-            stage_tile(p.xk, zk, tid, nthr16);
-            if (P.halves == 2) stage_tile(p.xv, zv, tid, nthr16);
+            if (touches_cache) {
+                stage_tile(p.xk, zk, tid, nthr16, 1);
+                if (P.halves == 2) stage_tile(p.xv, zv, tid, nthr16, 1);
+                wait_for_earlier_kernels();
+                stage_tile(p.xk, zk, tid, nthr16, 2);
+                if (P.halves == 2) stage_tile(p.xv, zv, tid, nthr16, 2);
+            } else {
+                stage_tile(p.xk, zk, tid, nthr16);
+                if (P.halves == 2) stage_tile(p.xv, zv, tid, nthr16);
+            }
+            cp_async_wait_all();
+            fence_proxy_async();
+            __syncthreads();
+            if (tid == 192) {
+                mbar_arrive(bar_k);
+                if (P.halves == 2) mbar_arrive(bar_v);
+            }
         }
-        cp_async_wait_all();
-        fence_proxy_async();
-        __syncthreads();
 
         // ---- 2. Eq. 6 as an implicit GEMM: one ring stage per (tap, 128-channel half).
         // Producer and MMA issuer are different threads, so the tensor pipe always has
@@ -280,18 +339,21 @@ __device__ __forceinline__ void compress_body(const TcCompressParams& P, uint8_t
             for (int it = npro; it < total; ++it) load_stage(g + it, it);
         } else if (tid == 128) {
             const uint64_t a0 = smem_desc(ring, 2048, 128);
-            const uint64_t bk0 = smem_desc(zk, lbo_z, 128), bv0 = smem_desc(zv, lbo_z, 128);
-            const uint32_t bstep = (2 * lbo_z) >> 4;
+            const uint64_t bk0 = smem_desc_sw128(zk, 16, 1024), bv0 = smem_desc_sw128(zv, 16, 1024);
+            const uint32_t hstep = half_z >> 4;      // second 64-channel half of a tile
+            mbar_wait(bar_k, tile_it & 1, P.status, failed, 5);
+            if (P.halves == 2) mbar_wait(bar_v, tile_it & 1, P.status, failed, 6);
             // stage index and phase, tap and channel half are tracked incrementally: no division here
             uint32_t st = g % NS, ph = (g / NS) & 1, tap = 0, half = 0;
-#pragma unroll 1
             for (int it = 0; it < total; ++it) {
                 mbar_wait(bar_full + 8 * st, ph, P.status, failed, 2);
                 tc_fence_after();
                 const uint64_t ad = a0 + st * (uint32_t)(kStageBytes >> 4);
-                const uint64_t bd = (half == 0 ? bk0 : bv0) + tap;   // tap t = row offset t (16 bytes per row)
+                const uint64_t bd = (half == 0 ? bk0 : bv0) + tap * 8u;   // tap t = row offset t (128 bytes per row)
+                // 16 channels per step: 32 bytes inside the 128-byte row, then the tile's second half
 #pragma unroll
-                for (int kk = 0; kk < 8; ++kk) umma_ss(tmem, ad + kk * 256u, bd + kk * bstep, idesc_conv, (it | kk) != 0);
+                for (int kk = 0; kk < 8; ++kk)
+                    umma_ss(tmem, ad + kk * 256u, bd + (uint32_t)(kk >> 2) * hstep + (uint32_t)(kk & 3) * 2u, idesc_conv, (it | kk) != 0);
                 umma_commit(bar_empty + 8 * st);
                 if (++half == (uint32_t)P.halves) { half = 0; ++tap; }
                 if (++st == (uint32_t)NS) { st = 0; ph ^= 1; }
@@ -301,7 +363,8 @@ __device__ __forceinline__ void compress_body(const TcCompressParams& P, uint8_t
         g += total;
 
         // ---- 3. accumulator -> bias, ReLU, row sum (Eq. 7), bf16 -> A operand of the blends
-        if (P.halves == 1 && (warp < 4 || warp >= 8)) {
+        if (!by_engine && P.halves == 1 && (warp < 4 || warp >= 8)) {
+            // (async-copy staging) the value tile, by the epilogue warps while the conv runs
             stage_tile(p.xv, zv, warp < 4 ? tid : tid - 128, 16);
             cp_async_wait_all();
         }
@@ -347,14 +410,18 @@ __device__ __forceinline__ void compress_body(const TcCompressParams& P, uint8_t
         __syncthreads();
 
         // ---- 4. Eq. 4, Eq. 5 (unnormalised): U_K += R X_K, U_V += R X_V from the staged tiles
+        if (!by_engine && P.halves == 1 && tid == 192) mbar_arrive(bar_v);   // the barrier above covers the warps' copies
         if (tid == 128) {
+            if (P.halves == 1) mbar_wait(bar_v, tile_it & 1, P.status, failed, 7);
             tc_fence_after();
 #pragma unroll 1
             for (int kk = 0; kk < n_tile / 16; ++kk) {
+                // contraction over positions: 16 rows of the tiles per step (MN-major operands, the two 64-channel
+                // blocks half a tile apart), starting `pad` rows in
                 const uint64_t ad = smem_desc(ring + kk * 2 * 2048, 2048, 128);
-                const uint32_t row0 = (uint32_t)(pad + kk * 16) * 16;
-                const uint64_t bk = smem_desc(zk + row0, 128, lbo_z);
-                const uint64_t bv = smem_desc(zv + row0, 128, lbo_z);
+                const uint32_t row0 = (uint32_t)(pad + kk * 16) * 128;
+                const uint64_t bk = smem_desc_sw128(zk + row0, half_z, 1024);
+                const uint64_t bv = smem_desc_sw128(zv + row0, half_z, 1024);
                 const uint32_t acc = (tile_it | kk) != 0;
                 umma_ss(tmem + kColUK, ad, bk, idesc_blend, acc);
                 umma_ss(tmem + kColUV, ad, bv, idesc_blend, acc);
@@ -811,11 +878,15 @@ __device__ __forceinline__ void cta_tmem_release(uint32_t tmem) {
     if (threadIdx.x < 32) tmem_dealloc(tmem, kTmemCols);
 }
 
-__global__ void __launch_bounds__(kThreads, 1) compress_tc_kernel(const __grid_constant__ TcCompressParams P) {
+struct TcCompressLaunch {
+    TcCompressParams c;
+    TcTileMaps t;
+};
+__global__ void __launch_bounds__(kThreads, 1) compress_tc_kernel(const __grid_constant__ TcCompressLaunch P) {
     extern __shared__ __align__(128) uint8_t smem[];
     __shared__ uint32_t tmem_slot;
     const uint32_t tmem = cta_tmem_acquire(&tmem_slot);
-    compress_body<false>(P, smem, tmem, false, blockIdx.x, blockIdx.y, blockIdx.z);
+    compress_body<false>(P.c, &P.t, smem, tmem, false, blockIdx.x, blockIdx.y, blockIdx.z);
     cta_tmem_release(tmem);
 }
 
@@ -1359,6 +1430,7 @@ __device__ __forceinline__ void decode_attention_body(const TcAttnParams& P, uin
 struct TcStepParams {
     TcAttnParams attn;
     TcCompressParams comp;
+    TcTileMaps tiles;
     int qtiles, n_attn_first, n_attn, comp_per_unit;   // comp_per_unit = parts * slot_blocks
     int decode;                                        // 1: chunks of one query, attention by decode_attention_body (a warp per unit)
     // position in the item list of a persistent launch (sequence_tc_kernel)
@@ -1377,7 +1449,7 @@ __device__ __forceinline__ void step_item(const TcStepParams& P, uint8_t* smem, 
             compress_pair_body(P.comp, &P.attn.maps[kMapVCache], smem, tmem, idx);
         } else {
             const int u = idx / P.comp_per_unit, rem = idx % P.comp_per_unit;
-            compress_body<true>(P.comp, smem, tmem, cache_cg, rem % P.comp.parts, rem / P.comp.parts, u);
+            compress_body<true>(P.comp, &P.tiles, smem, tmem, cache_cg, rem % P.comp.parts, rem / P.comp.parts, u);
         }
     } else {
         if (idx >= P.n_attn_first) idx -= n_comp;       // the attention items after the compress CTAs continue the first ones' numbering
@@ -1543,7 +1615,7 @@ __global__ void __launch_bounds__(kAttnThreads, 1) sequence_tc_kernel(const __gr
         }
         // within a unit: compress CTAs first (the longest), then the attention tiles, longest first
         // (cache rows rewritten by other SMs earlier in this same kernel are read around L1)
-        if (r < P.comp_per_unit) compress_body<false>(P.comp, smem, tmem, n > 0, r % P.comp.parts, r / P.comp.parts, u);
+        if (r < P.comp_per_unit) compress_body<false>(P.comp, nullptr, smem, tmem, n > 0, r % P.comp.parts, r / P.comp.parts, u);
         else attention_body(P.attn, Q.steps[n].attn.maps, true, smem, tmem, P.qtiles - 1 - (r - P.comp_per_unit), u);
         __syncthreads();
         if (threadIdx.x == 0) {
@@ -1577,9 +1649,10 @@ int parts_cap(int units, int slot_blocks) {
     return (600 + pairs - 1) / pairs;
 }
 
+int tile_rows_alloc(int n_tile, int k) { return (n_tile + k - 1 + 7) / 8 * 8; }    // halves of a tile stay on 1024-byte boundaries
+
 size_t smem_bytes(int n_tile, int k, int stages) {
-    const int rows_pad = (n_tile + k - 1) | 1;
-    return (size_t)stages * kStageBytes + 2 * 16 * (size_t)rows_pad * 16 + (2 * stages + 2) * 8 + 16;
+    return 1024 + (size_t)stages * kStageBytes + 2 * 256 * (size_t)tile_rows_alloc(n_tile, k) + (2 * stages + 4) * 8 + 16;
 }
 
 // Tile width and CTA count: fewest waves of 148 SMs, then least padded work.
@@ -1606,7 +1679,7 @@ bool make_plan(int S, int k, int halves, int units, int slot_blocks, bool fused,
             const double cost = (fused ? ctas * cta_us / 148.0 + 0.5 * cta_us : waves * cta_us) + (stages < 4 ? 0.05 : 0.0);
             if (cost < best) {
                 best = cost;
-                *out = Plan{n_tile, tiles, parts_eff, tpp, stages, (n_tile + k - 1) | 1, smem_bytes(n_tile, k, stages), cta_us};
+                *out = Plan{n_tile, tiles, parts_eff, tpp, stages, tile_rows_alloc(n_tile, k), smem_bytes(n_tile, k, stages), cta_us};
             }
         }
     }
@@ -1661,6 +1734,74 @@ int tensor_pack_weights(lococo_handle* h, const void* G, cudaStream_t st) {
 bool tensor_compress_supported(const lococo_handle* h, const CompressParams& p) {
     Plan pl;
     return h->use_tensor && p.S >= 1 && make_plan(p.S, p.k, p.c_in / 128, p.units, p.M / kSlots, false, &pl);
+}
+
+
+// ---- tensor maps
+using EncodeTiledFn = CUresult (*)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
+                                   const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                   CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+static EncodeTiledFn encode_tiled() {
+    static EncodeTiledFn fn = [] {
+        void* sym = nullptr;
+        cudaDriverEntryPointQueryResult res;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &sym, cudaEnableDefault, &res) != cudaSuccess ||
+            res != cudaDriverEntryPointSuccess) {
+            cudaGetLastError();
+            sym = nullptr;
+        }
+        return reinterpret_cast<EncodeTiledFn>(sym);
+    }();
+    return fn;
+}
+
+// View [batch, heads, tokens, 128] of bf16, `tokens` rows valid (rows beyond, or before row 0, read as zeros): boxes of
+// `box_rows` tokens x 64 channels in the 128-byte swizzle.
+static bool make_rows_map(CUtensorMap* map, const View& v, int tokens, int heads, int batch, int box_rows) {
+    EncodeTiledFn fn = encode_tiled();
+    if (!fn || tokens < 1 || box_rows < 1 || box_rows > 256) return false;
+    const cuuint64_t dims[4] = {(cuuint64_t)kD, (cuuint64_t)tokens, (cuuint64_t)heads, (cuuint64_t)batch};
+    cuuint64_t strides[3] = {(cuuint64_t)v.st * 2, (cuuint64_t)v.sh * 2, (cuuint64_t)v.sb * 2};
+    // a dimension of extent 1 never uses its stride: give it a harmless one
+    if (heads == 1) strides[1] = strides[0] * (cuuint64_t)tokens;
+    if (batch == 1) strides[2] = strides[1] * (cuuint64_t)heads;
+    for (cuuint64_t st : strides)
+        if (st == 0 || st % 16 != 0 || st >= ((cuuint64_t)1 << 40)) return false;
+    if (v.st < 0 || v.sh < 0 || v.sb < 0 || reinterpret_cast<uintptr_t>(v.ptr) % 16 != 0) return false;
+    const cuuint32_t box[4] = {64, (cuuint32_t)box_rows, 1, 1};
+    const cuuint32_t estr[4] = {1, 1, 1, 1};
+    return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, v.ptr, dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+              CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+static bool make_tile_map(CUtensorMap* map, const View& v, int tokens, int heads, int batch) {
+    return make_rows_map(map, v, tokens, heads, batch, 128);
+}
+
+// The tile maps of a compress launch whose tiling is already in P: whole-tile boxes of the cache and of the chunk, and
+// for each tile that holds the seam a pair of boxes with the heights of its two parts. Any refusal: async copies.
+static void fill_tile_maps(TcCompressParams* P, TcTileMaps* T) {
+    const CompressParams& p = P->base;
+    const int batch = p.units / p.heads, pad = (p.k - 1) / 2, rows = P->n_tile + p.k - 1, c = p.xk.c, b = p.S - c;
+    P->tile_maps = 0;
+    P->seam_h1[0] = P->seam_h1[1] = 0;
+    if (b < 1) return;
+    bool ok = make_rows_map(&T->m[kTmKChunk], p.xk.chunk, b, p.heads, batch, rows) &&
+              make_rows_map(&T->m[kTmVChunk], p.xv.chunk, b, p.heads, batch, rows);
+    if (ok && c > 0)
+        ok = make_rows_map(&T->m[kTmKCache], p.xk.cache, c, p.heads, batch, rows) &&
+             make_rows_map(&T->m[kTmVCache], p.xv.cache, c, p.heads, batch, rows);
+    int seams = 0;
+    for (int t = 0; ok && c > 0 && t < P->tiles; ++t) {
+        const int h1 = std::max(0, std::min(rows, c - (t * P->n_tile - pad)));
+        if (h1 == 0 || h1 == rows || h1 == P->seam_h1[0] || h1 == P->seam_h1[1]) continue;
+        if (seams == 2) break;                       // (cannot happen with one seam; such a tile would be staged by async copies)
+        CUtensorMap* m = &T->m[kTmSeam + 4 * seams];
+        ok = make_rows_map(m + 0, p.xk.cache, c, p.heads, batch, h1) && make_rows_map(m + 1, p.xk.chunk, b, p.heads, batch, rows - h1) &&
+             make_rows_map(m + 2, p.xv.cache, c, p.heads, batch, h1) && make_rows_map(m + 3, p.xv.chunk, b, p.heads, batch, rows - h1);
+        P->seam_h1[seams++] = h1;
+    }
+    if (ok) P->tile_maps = 1;
+    else P->seam_h1[0] = P->seam_h1[1] = 0;
 }
 
 static bool build_compress_params(lococo_handle* h, const CompressParams& p, bool fused, TcCompressParams* out,
@@ -1742,9 +1883,12 @@ int tensor_compress(lococo_handle* h, const CompressParams& p, cudaStream_t st) 
     static bool attr_set[64] = {};
     if (!smem_limit_set(compress_tc_kernel, kMaxSmem, attr_set)) return -1;
     dim3 grid(P.parts, P.slot_blocks, p.units);
+    TcCompressLaunch launch{};
+    launch.c = P;
+    fill_tile_maps(&launch.c, &launch.t);
     prof_begin(p.prof, 0, st);
     // the full 227 KB keeps one CTA per SM, so a CTA always finds its 512 TMEM columns free
-    compress_tc_kernel<<<grid, kThreads, kMaxSmem, st>>>(P);
+    compress_tc_kernel<<<grid, kThreads, kMaxSmem, st>>>(launch);
     const bool ok = cudaGetLastError() == cudaSuccess;
     prof_end(p.prof, st);
     if (!ok) return -1;
@@ -1753,42 +1897,6 @@ int tensor_compress(lococo_handle* h, const CompressParams& p, cudaStream_t st) 
 }
 
 // ---- tensor maps of the attention operands
-using EncodeTiledFn = CUresult (*)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
-                                   const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
-                                   CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
-static EncodeTiledFn encode_tiled() {
-    static EncodeTiledFn fn = [] {
-        void* sym = nullptr;
-        cudaDriverEntryPointQueryResult res;
-        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &sym, cudaEnableDefault, &res) != cudaSuccess ||
-            res != cudaDriverEntryPointSuccess) {
-            cudaGetLastError();
-            sym = nullptr;
-        }
-        return reinterpret_cast<EncodeTiledFn>(sym);
-    }();
-    return fn;
-}
-
-// View [batch, heads, tokens, 128] of bf16, `tokens` rows valid (rows beyond read as zeros): boxes of
-// 128 tokens x 64 channels in the 128-byte swizzle.
-static bool make_tile_map(CUtensorMap* map, const View& v, int tokens, int heads, int batch) {
-    EncodeTiledFn fn = encode_tiled();
-    if (!fn || tokens < 1) return false;
-    const cuuint64_t dims[4] = {(cuuint64_t)kD, (cuuint64_t)tokens, (cuuint64_t)heads, (cuuint64_t)batch};
-    cuuint64_t strides[3] = {(cuuint64_t)v.st * 2, (cuuint64_t)v.sh * 2, (cuuint64_t)v.sb * 2};
-    // a dimension of extent 1 never uses its stride: give it a harmless one
-    if (heads == 1) strides[1] = strides[0] * (cuuint64_t)tokens;
-    if (batch == 1) strides[2] = strides[1] * (cuuint64_t)heads;
-    for (cuuint64_t st : strides)
-        if (st == 0 || st % 16 != 0 || st >= ((cuuint64_t)1 << 40)) return false;
-    if (v.st < 0 || v.sh < 0 || v.sb < 0 || reinterpret_cast<uintptr_t>(v.ptr) % 16 != 0) return false;
-    const cuuint32_t box[4] = {64, 128, 1, 1};
-    const cuuint32_t estr[4] = {1, 1, 1, 1};
-    return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, v.ptr, dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
-              CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
-}
-
 static void fill_attention_maps(TcAttnParams* P) {
     const AttnParams& a = P->base;
     const int batch = a.units / a.heads;
@@ -1806,6 +1914,7 @@ static bool build_step_params(lococo_handle* h, const AttnParams& a, const Compr
     TcStepParams P{};
     double comp_us = 0.0;
     if (!build_compress_params(h, p, true, &P.comp, &comp_us)) return false;
+    fill_tile_maps(&P.comp, &P.tiles);
     P.attn.base = a;
     P.attn.status = P.comp.status;
     fill_attention_maps(&P.attn);
