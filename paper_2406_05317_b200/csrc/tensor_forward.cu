@@ -537,7 +537,7 @@ __device__ __forceinline__ void compress_body(const TcCompressParams& P, const T
     tc_fence_before();
     __syncthreads();
     if (tid == 128) {
-        for (int s = 0; s < 2 * NS + 2; ++s) mbar_inval(bar_full + 8 * s);
+        for (int s = 0; s < 2 * NS + 4; ++s) mbar_inval(bar_full + 8 * s);
     }
 }
 
