@@ -381,6 +381,23 @@ __device__ __forceinline__ void compress_body(const TcCompressParams& P, const T
                 tmem_ld32(lane_addr + c0, v);
                 tmem_ld_wait();
                 const bool ragged = j0 + c0 + 32 > p.S;
+                if (p.prot == 0 && !ragged && rstore == nullptr) {
+                    // the common case, with as few instructions as it takes: round first, then clamp (rounding is monotonic
+                    // and keeps zero, so max(round(x), 0) = round(max(x, 0))), two values per instruction
+#pragma unroll
+                    for (int e = 0; e < 32; e += 8) {
+                        uint32_t pk[4];
+#pragma unroll
+                        for (int x = 0; x < 8; x += 2) {
+                            const __nv_bfloat162 pr = __hmax2(__floats2bfloat162_rn(__uint_as_float(v[e + x]) + bias_i, __uint_as_float(v[e + x + 1]) + bias_i),
+                                                              __floats2bfloat162_rn(0.f, 0.f));
+                            pk[x >> 1] = *reinterpret_cast<const uint32_t*>(&pr);
+                            ssum += __low2float(pr) + __high2float(pr);
+                        }
+                        *reinterpret_cast<uint4*>(ring_ptr + ((c0 + e) >> 3) * 2048 + rl * 16) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
+                    }
+                    continue;
+                }
 #pragma unroll
                 for (int e = 0; e < 32; e += 8) {
                     uint32_t pk[4];
