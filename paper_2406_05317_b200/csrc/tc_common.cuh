@@ -80,6 +80,18 @@ __device__ __forceinline__ void tma_load_4d(uint32_t dst_smem, const void* tenso
         "l"(tensor_map), "r"(x), "r"(y), "r"(z), "r"(w), "r"(bar)
         : "memory");
 }
+// Tiled copy shared -> global through the tensor copy engine, rank 4, one box of the tensor map at coordinates
+// (x, y, z, w), all of them inside the tensor and x times the element size a multiple of 16 bytes. The copy belongs to
+// the thread's current bulk group; the shared-memory source must stay untouched until the group's reads are done.
+__device__ __forceinline__ void tma_store_4d(const void* tensor_map, uint32_t src_smem, int x, int y, int z, int w) {
+    asm volatile("cp.async.bulk.tensor.4d.global.shared::cta.tile.bulk_group [%0, {%2, %3, %4, %5}], [%1];" ::"l"(tensor_map),
+                 "r"(src_smem), "r"(x), "r"(y), "r"(z), "r"(w)
+                 : "memory");
+}
+// Closes the thread's bulk group and waits until its copies have read their shared-memory sources.
+__device__ __forceinline__ void bulk_stores_read() {
+    asm volatile("cp.async.bulk.commit_group;\n\tcp.async.bulk.wait_group.read 0;" ::: "memory");
+}
 // Makes a tensor map that was written to global memory before this kernel started (by a copy on the
 // same stream) the one the copy engine uses, whatever an earlier kernel read from that address.
 __device__ __forceinline__ void tensormap_acquire(const void* tensor_map) {

@@ -72,8 +72,9 @@ struct TcCompressParams {
     // maps with the box heights of its two parts. tile_maps == 0: every tile is staged by 16-byte async copies instead.
     int tile_maps;
     int seam_h1[2];               // cache rows (halo included) of a mixed tile; 0 = unused entry
+    int out_maps;                 // 1: maps of the output cache (boxes of 128 slots x 64 channels) for the direct write
 };
-enum { kTmKCache = 0, kTmKChunk = 1, kTmVCache = 2, kTmVChunk = 3, kTmSeam = 4, kTileMaps = 12 };   // seam e: 4 + 4 e + {Kc, Kn, Vc, Vn}
+enum { kTmKCache = 0, kTmKChunk = 1, kTmVCache = 2, kTmVChunk = 3, kTmSeam = 4, kTmKOut = 12, kTmVOut = 13, kTileMaps = 14 };   // seam e: 4 + 4 e + {Kc, Kn, Vc, Vn}
 struct alignas(64) TcTileMaps {
     CUtensorMap m[kTileMaps];
 };
@@ -472,21 +473,44 @@ __device__ __forceinline__ void compress_body(const TcCompressParams& P, const T
         const float inv = 1.f / tot;
         if (eg == 0) p.s[(int64_t)u * p.M + slot] = tot;
         const uint32_t lane_addr = tmem + ((uint32_t)((warp & 3) * 32) << 16);
+        // With maps of the output cache the rows leave through the copy engine: a thread (a slot) puts its 64-byte pieces
+        // into four swizzled boxes of 128 slots x 64 channels in the idle ring, and one lane sends the boxes off. A warp
+        // storing its 32 slots' pieces to memory itself pays for 32 separate segments per instruction.
+        const bool by_store_engine = tmaps != nullptr && P.out_maps;
+        uint8_t* boxes = ring_ptr + 2048;                      // [K | V][channels 0-63 | 64-127][128 slots][128 bytes]
 #pragma unroll 1
         for (int piece = eg; piece < 2 * (kD / 32); piece += 3) {
             const int mat = piece & 1, c0 = (piece >> 1) * 32;
-            const View& out = mat ? p.v_out : p.k_out;
-            __nv_bfloat16* orow = unit_base_mut<__nv_bfloat16>(out, n, h) + (int64_t)slot * out.st + c0;
             uint32_t a[32];
             tmem_ld32(lane_addr + (mat ? kColUV : kColUK) + c0, a);
             tmem_ld_wait();
+            uint4 o[4];
 #pragma unroll
             for (int e = 0; e < 32; e += 8)
-                *reinterpret_cast<uint4*>(orow + e) =
-                    make_uint4(pack_bf16(__uint_as_float(a[e]) * inv, __uint_as_float(a[e + 1]) * inv),
-                               pack_bf16(__uint_as_float(a[e + 2]) * inv, __uint_as_float(a[e + 3]) * inv),
-                               pack_bf16(__uint_as_float(a[e + 4]) * inv, __uint_as_float(a[e + 5]) * inv),
-                               pack_bf16(__uint_as_float(a[e + 6]) * inv, __uint_as_float(a[e + 7]) * inv));
+                o[e >> 3] = make_uint4(pack_bf16(__uint_as_float(a[e]) * inv, __uint_as_float(a[e + 1]) * inv),
+                                       pack_bf16(__uint_as_float(a[e + 2]) * inv, __uint_as_float(a[e + 3]) * inv),
+                                       pack_bf16(__uint_as_float(a[e + 4]) * inv, __uint_as_float(a[e + 5]) * inv),
+                                       pack_bf16(__uint_as_float(a[e + 6]) * inv, __uint_as_float(a[e + 7]) * inv));
+            if (by_store_engine) {
+                uint8_t* row = boxes + (mat * 2 + (c0 >> 6)) * 16384 + rl * 128;
+#pragma unroll
+                for (int x = 0; x < 4; ++x) *reinterpret_cast<uint4*>(row + (((((c0 & 63) >> 3) + x) ^ (rl & 7)) << 4)) = o[x];
+            } else {
+                const View& out = mat ? p.v_out : p.k_out;
+                __nv_bfloat16* orow = unit_base_mut<__nv_bfloat16>(out, n, h) + (int64_t)slot * out.st + c0;
+#pragma unroll
+                for (int x = 0; x < 4; ++x) *reinterpret_cast<uint4*>(orow + 8 * x) = o[x];
+            }
+        }
+        if (by_store_engine) {
+            fence_proxy_async();
+            __syncthreads();
+            if (tid == 0) {
+#pragma unroll
+                for (int x = 0; x < 4; ++x)
+                    tma_store_4d(&tmaps->m[x < 2 ? kTmKOut : kTmVOut], smem_u32(boxes) + x * 16384, 64 * (x & 1), sb * kSlots, h, n);
+                bulk_stores_read();
+            }
         }
     } else
     // ---- partial blends and row sums of this CTA's tiles
@@ -1800,6 +1824,7 @@ static void fill_tile_maps(TcCompressParams* P, TcTileMaps* T) {
     const CompressParams& p = P->base;
     const int batch = p.units / p.heads, pad = (p.k - 1) / 2, rows = P->n_tile + p.k - 1, c = p.xk.c, b = p.S - c;
     P->tile_maps = 0;
+    P->out_maps = 0;
     P->seam_h1[0] = P->seam_h1[1] = 0;
     if (b < 1) return;
     bool ok = make_rows_map(&T->m[kTmKChunk], p.xk.chunk, b, p.heads, batch, rows) &&
@@ -1819,6 +1844,9 @@ static void fill_tile_maps(TcCompressParams* P, TcTileMaps* T) {
     }
     if (ok) P->tile_maps = 1;
     else P->seam_h1[0] = P->seam_h1[1] = 0;
+    // the output cache, for the CTAs that write their rows themselves
+    P->out_maps = make_rows_map(&T->m[kTmKOut], p.k_out, p.M, p.heads, batch, kSlots) &&
+                  make_rows_map(&T->m[kTmVOut], p.v_out, p.M, p.heads, batch, kSlots);
 }
 
 static bool build_compress_params(lococo_handle* h, const CompressParams& p, bool fused, TcCompressParams* out,
