@@ -636,8 +636,8 @@ __host__ __device__ inline PairLayout pair_layout(int S, int n_tile, int k) {
 
 // `vmap`: tensor map of the value cache ([batch, heads, c rows, 128] in boxes of 128 rows x 64 channels), in kernel
 // parameter space.
-__device__ __forceinline__ void compress_pair_body(const TcCompressParams& P, const CUtensorMap* vmap, uint8_t* smem_raw,
-                                                   uint32_t tmem, int pair) {
+__device__ __forceinline__ void compress_pair_body(const TcCompressParams& P, const CUtensorMap* vmap, const TcTileMaps* tmaps,
+                                                   uint8_t* smem_raw, uint32_t tmem, int pair) {
     const CompressParams& p = P.base;
     const int tid = threadIdx.x, warp = tid >> 5;
     const int eg = warp >> 2;                          // epilogue group: which column chunks
@@ -818,6 +818,7 @@ __device__ __forceinline__ void compress_pair_body(const TcCompressParams& P, co
     // cache rows. A thread owns a slot; the rows are staged in shared memory so that the stores to the cache are
     // whole 256-byte rows (a warp storing 32 rows' pieces directly pays for 32 separate segments per instruction).
     const int n_tail = p.S - p.xk.c;                     // chunk rows: positions c .. S-1 (<= 16 of them)
+    const bool by_store_engine = tmaps != nullptr && P.out_maps;   // the cache rows leave as boxes through the copy engine
     float rtail[2][16];
 #pragma unroll
     for (int x = 0; x < 2; ++x) {
@@ -871,14 +872,37 @@ __device__ __forceinline__ void compress_pair_body(const TcCompressParams& P, co
                     }
                 }
             }
-            uint8_t* orow = x_ptr + (x * 2 + mat) * kPairOutTile + rl * kPairOutRow + c0 * 2;
+            uint4 o[4];
 #pragma unroll
             for (int e = 0; e < 32; e += 8)
-                *reinterpret_cast<uint4*>(orow + e * 2) =
-                    make_uint4(pack_bf16(acc[e] * inv, acc[e + 1] * inv), pack_bf16(acc[e + 2] * inv, acc[e + 3] * inv),
-                               pack_bf16(acc[e + 4] * inv, acc[e + 5] * inv), pack_bf16(acc[e + 6] * inv, acc[e + 7] * inv));
+                o[e >> 3] = make_uint4(pack_bf16(acc[e] * inv, acc[e + 1] * inv), pack_bf16(acc[e + 2] * inv, acc[e + 3] * inv),
+                                       pack_bf16(acc[e + 4] * inv, acc[e + 5] * inv), pack_bf16(acc[e + 6] * inv, acc[e + 7] * inv));
+            if (by_store_engine) {
+                // swizzled boxes of 128 slots x 64 channels: [unit][K | V][channels 0-63 | 64-127]
+                uint8_t* row = x_ptr + ((x * 2 + mat) * 2 + (c0 >> 6)) * 16384 + rl * 128;
+#pragma unroll
+                for (int y = 0; y < 4; ++y) *reinterpret_cast<uint4*>(row + (((((c0 & 63) >> 3) + y) ^ (rl & 7)) << 4)) = o[y];
+            } else {
+                uint8_t* orow = x_ptr + (x * 2 + mat) * kPairOutTile + rl * kPairOutRow + c0 * 2;
+#pragma unroll
+                for (int y = 0; y < 4; ++y) *reinterpret_cast<uint4*>(orow + 16 * y) = o[y];
+            }
         }
     }
+    if (by_store_engine) {
+        // the copy engine takes the boxes to the cache
+        fence_proxy_async();
+        __syncthreads();
+        if (tid == 0) {
+            for (int x = 0; x < nu; ++x) {
+                const int u = units[x], n = u / p.heads, h = u % p.heads;
+#pragma unroll
+                for (int y = 0; y < 4; ++y)
+                    tma_store_4d(&tmaps->m[y < 2 ? kTmKOut : kTmVOut], smem_u32(x_ptr) + (x * 4 + y) * 16384, 64 * (y & 1), 0, h, n);
+            }
+            bulk_stores_read();
+        }
+    } else {
     __syncthreads();
 #pragma unroll 1
     for (int x = 0; x < nu; ++x) {
@@ -894,6 +918,7 @@ __device__ __forceinline__ void compress_pair_body(const TcCompressParams& P, co
                     *reinterpret_cast<const uint4*>(tile + row * kPairOutRow + piece16 * 16);
             }
         }
+    }
     }
     tc_fence_before();
     __syncthreads();
@@ -1487,7 +1512,7 @@ __device__ __forceinline__ void step_item(const TcStepParams& P, uint8_t* smem, 
     if (is_comp) {
         idx -= P.n_attn_first;
         if (P.comp.pair) {
-            compress_pair_body(P.comp, &P.attn.maps[kMapVCache], smem, tmem, idx);
+            compress_pair_body(P.comp, &P.attn.maps[kMapVCache], &P.tiles, smem, tmem, idx);
         } else {
             const int u = idx / P.comp_per_unit, rem = idx % P.comp_per_unit;
             compress_body<true>(P.comp, &P.tiles, smem, tmem, cache_cg, rem % P.comp.parts, rem / P.comp.parts, u);
