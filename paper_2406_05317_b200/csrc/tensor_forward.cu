@@ -206,16 +206,11 @@ __device__ __forceinline__ void compress_body(const TcCompressParams& P, const T
     const uint32_t bar_acc = bar_empty + 8 * NS, bar_blend = bar_acc + 8;
     const uint32_t bar_k = bar_blend + 8, bar_v = bar_k + 8;     // key tile, value tile staged
 
-    if (tid == 128) {
-        for (int s = 0; s < NS; ++s) {
-            mbar_init(bar_full + 8 * s, 1);
-            mbar_init(bar_empty + 8 * s, 1);
-        }
-        mbar_init(bar_acc, 1);
-        mbar_init(bar_blend, 1);
-        mbar_init(bar_k, 1);
-        mbar_init(bar_v, 1);
-        *failed = 0;
+    if (warp == 4) {
+        // every barrier here has one arrival per phase; a lane sets up one of them
+        const int lane = tid & 31;
+        if (lane < 2 * NS + 4) mbar_init(bar_full + 8 * lane, 1);
+        if (lane == 0) *failed = 0;
         fence_barrier_init();
     }
     tc_fence_before();
@@ -240,6 +235,8 @@ __device__ __forceinline__ void compress_body(const TcCompressParams& P, const T
 #pragma unroll 1
     for (int tile = tile_begin; tile < tile_end; ++tile, ++tile_it) {
         const int j0 = tile * n_tile;
+        // columns of this tile that hold positions below S, as a multiple of 16: the last tile's MMAs are that narrow
+        const int n_use = min(n_tile, (p.S - j0 + 15) & ~15);
         // The weight producer (one thread of warp 5) runs ahead of everything else: a tile's
         // first ring stages need no wait, the ring being drained at every tile boundary.
         const int total = p.k * P.halves;
@@ -342,6 +339,7 @@ __device__ __forceinline__ void compress_body(const TcCompressParams& P, const T
             const uint64_t a0 = smem_desc(ring, 2048, 128);
             const uint64_t bk0 = smem_desc_sw128(zk, 16, 1024), bv0 = smem_desc_sw128(zv, 16, 1024);
             const uint32_t hstep = half_z >> 4;      // second 64-channel half of a tile
+            const uint32_t idesc_tile = n_use == n_tile ? idesc_conv : instr_desc_bf16(n_use, false, false);
             mbar_wait(bar_k, tile_it & 1, P.status, failed, 5);
             if (P.halves == 2) mbar_wait(bar_v, tile_it & 1, P.status, failed, 6);
             // stage index and phase, tap and channel half are tracked incrementally: no division here
@@ -354,7 +352,7 @@ __device__ __forceinline__ void compress_body(const TcCompressParams& P, const T
                 // 16 channels per step: 32 bytes inside the 128-byte row, then the tile's second half
 #pragma unroll
                 for (int kk = 0; kk < 8; ++kk)
-                    umma_ss(tmem, ad + kk * 256u, bd + (uint32_t)(kk >> 2) * hstep + (uint32_t)(kk & 3) * 2u, idesc_conv, (it | kk) != 0);
+                    umma_ss(tmem, ad + kk * 256u, bd + (uint32_t)(kk >> 2) * hstep + (uint32_t)(kk & 3) * 2u, idesc_tile, (it | kk) != 0);
                 umma_commit(bar_empty + 8 * st);
                 if (++half == (uint32_t)P.halves) { half = 0; ++tap; }
                 if (++st == (uint32_t)NS) { st = 0; ph ^= 1; }
@@ -376,8 +374,10 @@ __device__ __forceinline__ void compress_body(const TcCompressParams& P, const T
             const uint32_t lane_addr = tmem + ((uint32_t)((warp & 3) * 32) << 16);
             float* rstore = P.R_store ? P.R_store + ((int64_t)u * p.M + slot) * p.S : nullptr;
             const bool keep = slot < p.prot;
+            // (columns from n_use on were not written; they are read, as zeros, only by the copy of R for the backward pass)
+            const int n_read = p.R16 ? n_tile : n_use;
 #pragma unroll 1
-            for (int c0 = eg * 32; c0 < n_tile; c0 += 96) {
+            for (int c0 = eg * 32; c0 < n_read; c0 += 96) {
                 uint32_t v[32];
                 tmem_ld32(lane_addr + c0, v);
                 tmem_ld_wait();
@@ -433,7 +433,7 @@ __device__ __forceinline__ void compress_body(const TcCompressParams& P, const T
             if (P.halves == 1) mbar_wait(bar_v, tile_it & 1, P.status, failed, 7);
             tc_fence_after();
 #pragma unroll 1
-            for (int kk = 0; kk < n_tile / 16; ++kk) {
+            for (int kk = 0; kk < n_use / 16; ++kk) {
                 // contraction over positions: 16 rows of the tiles per step (MN-major operands, the two 64-channel
                 // blocks half a tile apart), starting `pad` rows in
                 const uint64_t ad = smem_desc(ring + kk * 2 * 2048, 2048, 128);
@@ -575,10 +575,11 @@ __device__ __forceinline__ void compress_body(const TcCompressParams& P, const T
             merge_partials(P, tmem, sb, u, part, own_s);
         }
     }
-    tc_fence_before();
-    __syncthreads();
-    if (tid == 128) {
-        for (int s = 0; s < 2 * NS + 4; ++s) mbar_inval(bar_full + 8 * s);
+    if (!kMerge) {
+        // (a kernel whose CTA goes on to other work in this shared memory; a CTA that ends here leaves its barriers as they are)
+        tc_fence_before();
+        __syncthreads();
+        if (warp == 4 && (tid & 31) < 2 * NS + 4) mbar_inval(bar_full + 8 * (tid & 31));
     }
 }
 
@@ -1074,17 +1075,11 @@ __device__ __forceinline__ void attention_body(const TcAttnParams& P, const CUte
     constexpr int kMma = 256;                                   // lane 0 of warp 8
     constexpr int kLoad = 288;                                  // lane 0 of warp 9: issues the tensor copies
 
-    if (tid == kMma) {
-        for (int b = 0; b < 2; ++b) {
-            mbar_init(k_full(b), 1);
-            mbar_init(v_full(b), 1);
-            mbar_init(s_full(b), 1);
-            mbar_init(s_free(b), 256);
-            mbar_init(p_full(b), 256);
-            mbar_init(pv_done(b), 1);
-        }
-        mbar_init(q_full, 1);
-        *failed = 0;
+    if (warp == kMma / 32) {
+        // a lane sets up one of the thirteen barriers: s_free and p_full (words 4-7) count the 256 softmax threads
+        const int lane = tid & 31;
+        if (lane < 13) mbar_init(bar0 + 8 * lane, lane >= 4 && lane < 8 ? 256 : 1);
+        if (lane == 0) *failed = 0;
         fence_barrier_init();
     }
     tc_fence_before();
@@ -1364,10 +1359,11 @@ __device__ __forceinline__ void attention_body(const TcAttnParams& P, const CUte
         }
         if (live && p.lse && half == 0) p.lse[(int64_t)u * p.lse_stride + row] = (m_used + log2f(ltot)) * 0.6931471805599453f;
     }
-    tc_fence_before();
-    __syncthreads();
-    if (tid == kMma) {
-        for (int s = 0; s < 13; ++s) mbar_inval(bar0 + 8 * s);
+    if (maps_fresh) {
+        // (the persistent kernel: its CTA goes on to other work in this shared memory)
+        tc_fence_before();
+        __syncthreads();
+        if (warp == kMma / 32 && (tid & 31) < 13) mbar_inval(bar0 + 8 * (tid & 31));
     }
 }
 
