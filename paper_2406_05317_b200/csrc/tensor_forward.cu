@@ -170,6 +170,84 @@ __device__ __forceinline__ void merge_partials(const TcCompressParams& P, uint32
     }
 }
 
+// The same merge with the stored sets brought in by the copy engine instead of by the threads' own loads (which leave
+// a thread waiting for an L2 round trip per piece: 6.5 us for two stored sets). A (matrix, 32-channel chunk) piece of a
+// stored set is 16 KB of contiguous memory. Each of the three warp groups runs its pieces through a ring of three such
+// buffers of its own: its first thread asks for the next pieces while the group adds up the ones that have arrived.
+// Arithmetic and order of the sums as in merge_partials. `stage`: 3 x 3 x 16 KB of idle shared memory, 128-byte aligned;
+// `bars`: nine barriers, already set up (one arrival each).
+constexpr uint32_t kMergePiece = 32 * kSlots * 4;                 // bytes
+constexpr uint32_t kMergeStage = 9 * kMergePiece;
+__device__ __forceinline__ void merge_partials_staged(const TcCompressParams& P, uint32_t tmem, int sb, int u, int own, float own_s,
+                                                      uint8_t* stage, uint32_t bars, volatile int* failed) {
+    const CompressParams& p = P.base;
+    const int n = u / p.heads, h = u % p.heads;
+    const int warp = threadIdx.x >> 5;
+    const int eg = warp >> 2, rl = (warp & 3) * 32 + (threadIdx.x & 31);
+    const int slot = sb * kSlots + rl;
+    const int64_t base = ((int64_t)u * P.slot_blocks + sb) * P.part_stride;
+    const uint32_t lane_addr = tmem + ((uint32_t)((warp & 3) * 32) << 16);
+    const bool leader = rl == 0;
+    const int stored = P.parts - 1;                               // sets that come from memory
+    const int n_pieces = (2 * (kD / 32) - eg + 2) / 3;            // pieces eg, eg + 3, ... below 8
+    const int n_jobs = n_pieces * stored;
+    const float* gbuf = reinterpret_cast<const float*>(stage + eg * 3 * kMergePiece);
+    const uint32_t gbuf_a = smem_u32(gbuf), gbar = bars + eg * 24;
+    // job j: stored set number (j % stored) of the group's piece number (j / stored), into buffer j % 3
+    auto request = [&](int j) {
+        const int piece = eg + 3 * (j / stored), k = j % stored;
+        const int pt = k < own ? k : k + 1, mat = piece & 1, c0 = (piece >> 1) * 32;
+        const uint32_t b = gbar + 8 * (j % 3);
+        mbar_expect_tx(b, kMergePiece);
+        bulk_load(gbuf_a + (j % 3) * kMergePiece, P.part_U + ((base + pt) * 2 + mat) * (int64_t)(kSlots * kD) + c0 * kSlots, kMergePiece, b);
+    };
+    if (leader) {
+        // the sets were written by other CTAs' ordinary stores (seen through the acquire and the CTA barrier before this
+        // call): ordered before the copy engine's reads of them
+        asm volatile("fence.proxy.async;" ::: "memory");
+        for (int j = 0; j < 3 && j < n_jobs; ++j) request(j);
+    }
+    float tot = 0.f;
+    for (int pt = 0; pt < P.parts; ++pt) tot += pt == own ? own_s : __ldcg(P.part_s + (base + pt) * kSlots + rl);
+    tot = slot < p.prot ? 1.f : tot + p.eps;   // a protected slot's row is e_i: denominator exactly 1
+    const float inv = 1.f / tot;
+    if (eg == 0) p.s[(int64_t)u * p.M + slot] = tot;
+    int j = 0;
+#pragma unroll 1
+    for (int piece = eg; piece < 2 * (kD / 32); piece += 3) {
+        const int mat = piece & 1, c0 = (piece >> 1) * 32;
+        uint32_t mine[32];
+        tmem_ld32(lane_addr + (mat ? kColUV : kColUK) + c0, mine);
+        float acc[32];
+#pragma unroll
+        for (int e = 0; e < 32; ++e) acc[e] = 0.f;
+#pragma unroll 1
+        for (int pt = 0; pt < P.parts; ++pt) {
+            if (pt == own) {
+                tmem_ld_wait();
+#pragma unroll
+                for (int e = 0; e < 32; ++e) acc[e] += __uint_as_float(mine[e]);
+                continue;
+            }
+            mbar_wait(gbar + 8 * (j % 3), (j / 3) & 1, P.status, failed, 14);
+            const float* v = gbuf + (j % 3) * (kMergePiece / 4) + rl;
+#pragma unroll
+            for (int e = 0; e < 32; ++e) acc[e] += v[e * kSlots];
+            // the group is done with the buffer: its next use may be asked for
+            asm volatile("bar.sync %0, 128;" ::"r"(3 + eg) : "memory");
+            if (leader && j + 3 < n_jobs) request(j + 3);
+            ++j;
+        }
+        const View& out = mat ? p.v_out : p.k_out;
+        __nv_bfloat16* orow = unit_base_mut<__nv_bfloat16>(out, n, h) + (int64_t)slot * out.st + c0;
+#pragma unroll
+        for (int e = 0; e < 32; e += 8)
+            *reinterpret_cast<uint4*>(orow + e) =
+                make_uint4(pack_bf16(acc[e] * inv, acc[e + 1] * inv), pack_bf16(acc[e + 2] * inv, acc[e + 3] * inv),
+                           pack_bf16(acc[e + 4] * inv, acc[e + 5] * inv), pack_bf16(acc[e + 6] * inv, acc[e + 7] * inv));
+    }
+}
+
 // Work of one CTA of exactly 384 threads: tiles [part*tiles_per_part, ...) of slot block sb of unit u.
 // Thread 128 issues the MMAs, thread 160 feeds the weight ring, every thread stages rows, and all
 // twelve warps share the two epilogues: warp w owns accumulator rows (TMEM lanes) 32*(w%4)..+31
@@ -569,10 +647,19 @@ __device__ __forceinline__ void compress_body(const TcCompressParams& P, const T
                 counts[0] = 0;     // nobody touches the counts again before the next step
                 counts[1] = 0;
             }
+            // idle shared memory for the stored sets' pieces, where there is enough of it (past the row sums)
+            uint8_t* stage = ring_ptr + 8192;
+            const uint32_t mbars = smem_u32(ring_ptr + 2048);
+            const bool staged = (size_t)NS * kStageBytes + 4 * (size_t)half_z >= 8192 + (size_t)kMergeStage;
+            if (staged && tid == 32) {
+                for (int i = 0; i < 9; ++i) mbar_init(mbars + 8 * i, 1);
+                fence_barrier_init();
+            }
             __syncthreads();
             __threadfence();
             const float own_s = sums[rl] + sums[kSlots + rl] + sums[2 * kSlots + rl];
-            merge_partials(P, tmem, sb, u, part, own_s);
+            if (staged) merge_partials_staged(P, tmem, sb, u, part, own_s, stage, mbars, failed);
+            else merge_partials(P, tmem, sb, u, part, own_s);
         }
     }
     if (!kMerge) {
