@@ -2,11 +2,13 @@
 //
 // compress_tc_kernel fuses Algorithm 2's Steps 4 and 5 for one tile of positions:
 //   1. the [cache; chunk] key and value rows of the tile (plus a (k-1)/2 halo) are staged
-//      once in shared memory, un-swizzled, as [8-channel group][row][8 channels];
+//      once in shared memory by the tensor copy engine, as two 64-channel halves of 128-byte
+//      rows in the 128-byte swizzle;
 //   2. Eq. 6 runs as an implicit GEMM on the tensor cores: for every tap t,
 //      D[slot, pos] += G_t[slot, ch] * Z[pos + t, ch]; a tap is a row offset into the
-//      staged tile, which the un-swizzled layout allows at 16-byte granularity; the
-//      per-tap weight tiles stream from L2 through a ring fed by bulk async copies;
+//      staged tile (the swizzle is a function of the shared-memory address, so an operand
+//      may start at any row); the per-tap weight tiles stream from L2 through a ring fed by
+//      bulk async copies;
 //   3. the accumulator leaves TMEM once: bias, ReLU, the running row sum of Eq. 7, bf16
 //      rounding, and the result is written back to shared memory as the A operand of
 //   4. Eq. 4 / Eq. 5: U_K += R * X_K and U_V += R * X_V, which read the SAME staged tiles,
@@ -613,7 +615,9 @@ __device__ __forceinline__ void compress_body(const TcCompressParams& P, const T
         }
         if (!last) {
             // stored channel-major ([channel][slot]) so that a warp's 32 lanes write 128 contiguous bytes;
-            // the eight (matrix, 32-channel chunk) pieces go round the three groups
+            // the eight (matrix, 32-channel chunk) pieces go round the three groups. (Putting the set together in
+            // shared memory first and sending it off as bulk copies, or as 16-byte stores by all threads, was 2-3 %
+            // slower for a whole sequence: these stores leave straight from the accumulators and nothing waits for them.)
 #pragma unroll 1
             for (int piece = eg; piece < 2 * (kD / 32); piece += 3) {
                 const int mat = piece & 1, c0 = (piece >> 1) * 32;
