@@ -102,86 +102,22 @@ __global__ void pack_image_kernel(const __nv_bfloat16* __restrict__ G, __nv_bflo
 }
 
 // cache rows of slot block sb of unit u = (sum of the partial blends) / (sum of the partial row sums + eps), by the CTA
-// (384 threads) that holds partial set `own` in its TMEM accumulators and its row sum in `own_s`; the other sets
-// come from the workspace. The arithmetic is finalize_tile's, term for term, the sets added in their order. The
-// threads are laid out as in the compress epilogues: a thread owns one slot (a warp 32 consecutive slots) and takes
-// the eight (matrix, 32-channel chunk) pieces in turn with the two other warp groups. The stored sets are
-// channel-major, so the warp's loads of one channel are 128 contiguous bytes; the loads of two sets (32 channels
-// each) are in flight at once, around L1 (other SMs wrote them moments ago). The thread then holds 32 consecutive
-// channels of its slot: 64 bytes of the slot-major cache row.
-__device__ __forceinline__ void merge_partials(const TcCompressParams& P, uint32_t tmem, int sb, int u, int own, float own_s) {
-    const CompressParams& p = P.base;
-    const int n = u / p.heads, h = u % p.heads;
-    const int warp = threadIdx.x >> 5;
-    const int eg = warp >> 2, rl = (warp & 3) * 32 + (threadIdx.x & 31);
-    const int slot = sb * kSlots + rl;
-    const int64_t base = ((int64_t)u * P.slot_blocks + sb) * P.part_stride;
-    const uint32_t lane_addr = tmem + ((uint32_t)((warp & 3) * 32) << 16);
-    float tot = 0.f;
-    for (int pt = 0; pt < P.parts; ++pt) tot += pt == own ? own_s : __ldcg(P.part_s + (base + pt) * kSlots + rl);
-    tot = slot < p.prot ? 1.f : tot + p.eps;   // a protected slot's row is e_i: denominator exactly 1
-    const float inv = 1.f / tot;
-    if (eg == 0) p.s[(int64_t)u * p.M + slot] = tot;
-#pragma unroll 1
-    for (int piece = eg; piece < 2 * (kD / 32); piece += 3) {
-        const int mat = piece & 1, c0 = (piece >> 1) * 32;
-        uint32_t mine[32];
-        tmem_ld32(lane_addr + (mat ? kColUV : kColUK) + c0, mine);
-        const float* src = P.part_U + (base * 2 + mat) * (int64_t)(kSlots * kD) + c0 * kSlots + rl;
-        float acc[32];
-#pragma unroll
-        for (int e = 0; e < 32; ++e) acc[e] = 0.f;
-        bool first = true;
-        for (int pt = 0; pt < P.parts;) {
-            // the next two stored sets from pt on, then every set up to the second of them, in order
-            int i0 = pt;
-            if (i0 == own) ++i0;
-            int i1 = i0 + 1;
-            if (i1 == own) ++i1;
-            float v0[32], v1[32];
-#pragma unroll
-            for (int e = 0; e < 32; ++e) {
-                v0[e] = i0 < P.parts ? __ldcg(src + (int64_t)i0 * (2 * kSlots * kD) + e * kSlots) : 0.f;
-                v1[e] = i1 < P.parts ? __ldcg(src + (int64_t)i1 * (2 * kSlots * kD) + e * kSlots) : 0.f;
-            }
-            if (first) {
-                tmem_ld_wait();
-                first = false;
-            }
-            for (int x = pt; x <= i1 && x < P.parts; ++x) {
-                if (x == own) {
-#pragma unroll
-                    for (int e = 0; e < 32; ++e) acc[e] += __uint_as_float(mine[e]);
-                } else if (x == i0) {
-#pragma unroll
-                    for (int e = 0; e < 32; ++e) acc[e] += v0[e];
-                } else {
-#pragma unroll
-                    for (int e = 0; e < 32; ++e) acc[e] += v1[e];
-                }
-            }
-            pt = i1 + 1;
-        }
-        const View& out = mat ? p.v_out : p.k_out;
-        __nv_bfloat16* orow = unit_base_mut<__nv_bfloat16>(out, n, h) + (int64_t)slot * out.st + c0;
-#pragma unroll
-        for (int e = 0; e < 32; e += 8)
-            *reinterpret_cast<uint4*>(orow + e) =
-                make_uint4(pack_bf16(acc[e] * inv, acc[e + 1] * inv), pack_bf16(acc[e + 2] * inv, acc[e + 3] * inv),
-                           pack_bf16(acc[e + 4] * inv, acc[e + 5] * inv), pack_bf16(acc[e + 6] * inv, acc[e + 7] * inv));
-    }
-}
-
-// The same merge with the stored sets brought in by the copy engine instead of by the threads' own loads (which leave
-// a thread waiting for an L2 round trip per piece: 6.5 us for two stored sets). A (matrix, 32-channel chunk) piece of a
-// stored set is 16 KB of contiguous memory. Each of the three warp groups runs its pieces through a ring of three such
-// buffers of its own: its first thread asks for the next pieces while the group adds up the ones that have arrived.
-// Arithmetic and order of the sums as in merge_partials. `stage`: 3 x 3 x 16 KB of idle shared memory, 128-byte aligned;
-// `bars`: nine barriers, already set up (one arrival each).
+// (384 threads) that holds partial set `own` in its TMEM accumulators and its row sum in `own_s`; the other sets come
+// from the workspace. The arithmetic is finalize_tile's, term for term, the sets added in their order. The threads are
+// laid out as in the compress epilogues: a thread owns one slot (a warp 32 consecutive slots) and takes the eight
+// (matrix, 32-channel chunk) pieces in turn with the two other warp groups; it ends up with 32 consecutive channels of
+// its slot, 64 bytes of the slot-major cache row. The stored sets are channel-major and come in through the copy
+// engine (a thread's own loads of them, 32 channels x 2 sets in flight around L1, left it waiting for an L2 round trip
+// per piece: 6.5 us for two stored sets). A (matrix, 32-channel chunk) piece of a stored set is 16 KB of contiguous
+// memory. Each of the three warp groups runs its pieces through a ring of three such buffers of its own: its first
+// thread asks for the next pieces while the group adds up the ones that have arrived. `stage`: 3 x 3 x 16 KB of idle
+// shared memory, 128-byte aligned (the host sets P.merge only where the ring and the tiles have room for it, which is
+// every plan: at least two 32 KB stages and, where fewer than four fit, tiles of more than 99 KB); `bars`: nine
+// barriers, already set up (one arrival each).
 constexpr uint32_t kMergePiece = 32 * kSlots * 4;                 // bytes
 constexpr uint32_t kMergeStage = 9 * kMergePiece;
-__device__ __forceinline__ void merge_partials_staged(const TcCompressParams& P, uint32_t tmem, int sb, int u, int own, float own_s,
-                                                      uint8_t* stage, uint32_t bars, volatile int* failed) {
+__device__ __forceinline__ void merge_partials(const TcCompressParams& P, uint32_t tmem, int sb, int u, int own, float own_s,
+                                               uint8_t* stage, uint32_t bars, volatile int* failed) {
     const CompressParams& p = P.base;
     const int n = u / p.heads, h = u % p.heads;
     const int warp = threadIdx.x >> 5;
@@ -651,19 +587,17 @@ __device__ __forceinline__ void compress_body(const TcCompressParams& P, const T
                 counts[0] = 0;     // nobody touches the counts again before the next step
                 counts[1] = 0;
             }
-            // idle shared memory for the stored sets' pieces, where there is enough of it (past the row sums)
+            // idle shared memory for the stored sets' pieces (past the row sums)
             uint8_t* stage = ring_ptr + 8192;
             const uint32_t mbars = smem_u32(ring_ptr + 2048);
-            const bool staged = (size_t)NS * kStageBytes + 4 * (size_t)half_z >= 8192 + (size_t)kMergeStage;
-            if (staged && tid == 32) {
+            if (tid == 32) {
                 for (int i = 0; i < 9; ++i) mbar_init(mbars + 8 * i, 1);
                 fence_barrier_init();
             }
             __syncthreads();
             __threadfence();
             const float own_s = sums[rl] + sums[kSlots + rl] + sums[2 * kSlots + rl];
-            if (staged) merge_partials_staged(P, tmem, sb, u, part, own_s, stage, mbars, failed);
-            else merge_partials(P, tmem, sb, u, part, own_s);
+            merge_partials(P, tmem, sb, u, part, own_s, stage, mbars, failed);
         }
     }
     if (!kMerge) {
@@ -2104,7 +2038,10 @@ int tensor_chunk_step(lococo_handle* h, const AttnParams& a, const CompressParam
     const bool own_output = p.W_out == nullptr && p.k_out.ptr != p.xk.cache.ptr && p.v_out.ptr != p.xv.cache.ptr;
     P.comp.direct = own_output && P.comp.parts == 1;
     // several CTAs per (unit, slot block): the one that stores the last partial set sums them and writes the rows
-    P.comp.merge = own_output && P.comp.parts > 1 && p.R16 == nullptr;
+    // (the merging CTA stages the stored sets in its idle ring and tiles: every plan has the room, and one that did not
+    // would leave the sum to the finalize pass)
+    const bool merge_room = (size_t)P.comp.stages * kStageBytes + 4 * 128 * (size_t)P.comp.rows_pad >= 8192 + (size_t)kMergeStage;
+    P.comp.merge = own_output && P.comp.parts > 1 && p.R16 == nullptr && merge_room;
     // generation stage: chunks so short that a unit's positions are one small tile. Two units per compress CTA share
     // every weight stage, and a chunk of one query is attended to by a warp instead of a 128-row MMA tile.
     const int n_tile16 = (p.S + 15) / 16 * 16;
