@@ -93,6 +93,13 @@ def test_cfg4_slice(api, orc, path):
     check_sequence(api, orc, wl.CONFIGS["cfg4"].slice(heads=2, B=1024, L=3072), path)
 
 
+@pytest.mark.parametrize("B", [256, 320])
+def test_two_position_tiles_per_unit(api, orc, B):
+    # S = 384 or 448: two compress CTAs per unit, so the one that arrives last merges ONE stored set with its own
+    # (the shortest run of the merge's buffer ring); 448 = 2 x 224 has no ragged last tile, 384 has one
+    check_sequence(api, orc, wl.CONFIGS["cfg2"].slice(heads=3, B=B, L=4 * B + 96), 0)
+
+
 def test_tensor_path_ragged_chunks_direct_cache_write(api, orc):
     # tensor-core path with sizes that are multiples of nothing the kernels tile by: B = 100, a short last
     # chunk, a first compress step on a partly filled cache (c = 100), several sequences; with this many
